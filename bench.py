@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of tree-decode attention over prefix-shared KV.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
+
+A step is one pass of the whole path over the workload's tree: tree flatten (all pages kept),
+then for each layer the append of one new token per leaf and tree-decode attention for every
+leaf.  The metric is leaf-queries/s = leaves / (time of one step over all layers), summed over
+GPUs (independent replicas, no collective).  One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "tree_decode_attention_leaf_queries_per_s"
+UNIT = "leaf-queries/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (0 = its own)")
+    ap.add_argument("--chunk-pages", type=int, default=None)
+    ap.add_argument("--kernel", type=int, default=None)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time budget of the oracle sample")
+    return ap.parse_args()
+
+
+def workload_description(wl, layers):
+    from workloads import tree_stats
+    g, st = wl.geometry, tree_stats(wl.tree)
+    return {
+        "workload": wl.name,
+        "tree": f"{st['n_leaves']} leaves, {st['n_nodes']} nodes, {st['unique_tokens']} unique tokens, "
+                f"{st['path_tokens']} path tokens",
+        "heads": f"{g.num_q_heads}q/{g.num_kv_heads}kv x {g.head_dim}",
+        "layers": layers,
+        "page_size": g.page_size,
+        "topology_seed": wl.topology_seed,
+        "value_seed": wl.value_seed,
+    }
+
+
+# ----------------------------------------------------------------------------- oracle timing
+def oracle_sample(wl, layers, budget_s, max_leaves=None):
+    """Time the oracle, as it stands, on a bounded sample: whole leaves of layer 0, as many as
+    fit the budget.  Returns (leaf-queries/s for a full step over `layers` layers, threads, text)."""
+    from oracle.tree_attention import tree_decode_attention
+    from workloads import node_kv_bits, query_bits
+    tree, g = wl.tree, wl.geometry
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([int(p.get("num_threads", 1)) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = 1
+    qb = query_bits(wl.value_seed, 0, tree.n_leaves, g.num_q_heads, g.head_dim)
+    empty = np.zeros((0, g.num_kv_heads, g.head_dim), np.uint16)
+    k_nodes = [empty] * tree.n_nodes
+    v_nodes = [empty] * tree.n_nodes
+    order = np.random.default_rng(0).permutation(tree.n_leaves)
+    if max_leaves:
+        order = order[:max_leaves]
+    done, spent = 0, 0.0
+    for l in order:
+        v = int(tree.leaf_node[l])
+        while v >= 0:  # inputs are generated outside the timed part
+            if k_nodes[v] is empty and tree.tokens[v] > 0:
+                k_nodes[v], v_nodes[v] = node_kv_bits(wl.value_seed, v, int(tree.tokens[v]), g.num_kv_heads,
+                                                      g.head_dim, 0)
+            v = int(tree.parent[v])
+        t0 = time.perf_counter()
+        tree_decode_attention(tree.parent, tree.tokens, tree.leaf_node, k_nodes, v_nodes, qb,
+                              g.num_q_heads, g.num_kv_heads, leaves=[int(l)])
+        spent += time.perf_counter() - t0
+        done += 1
+        if spent >= budget_s:
+            break
+    per_leaf_layer = spent / done
+    value = 1.0 / (per_leaf_layer * layers)
+    text = (f"{done} of {tree.n_leaves} leaves of {wl.name}, layer 0 only ({spent:.1f} s of oracle time); "
+            f"a full step is {layers} layers x {tree.n_leaves} leaves, scaled linearly")
+    return value, threads, text, spent
+
+
+def run_reference(args):
+    """The reference arm: the fp64 CPU oracle timed on the host cores, rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from workloads import make_workload
+    wl = make_workload(args.workload)
+    layers = args.layers or wl.geometry.num_layers
+    per_step_budget = max(0.5, min(6.0, 90.0 / max(1, args.steps + args.warmup)))
+    vals, spent_all = [], []
+    threads, text = 1, ""
+    for i in range(args.warmup + args.steps):
+        value, threads, text, spent = oracle_sample(wl, layers, per_step_budget)
+        if i >= args.warmup:
+            vals.append(value)
+            spent_all.append(spent)
+    value = len(vals) / sum(1.0 / v for v in vals)
+    ms = 1000.0 * wl.tree.n_leaves / value
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_description(wl, layers),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": "each step: " + text},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, power = [], [], []
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.file.read().splitlines():
+            f = [x.strip() for x in row.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.file.name)
+        except OSError:
+            pass
+        if sm:
+            out.update({"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                        "samples": len(sm), "power_w_max": max(power)})
+        return out
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------- ours
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from workloads import make_workload
+    from workloads.loader import DecodeJob
+    import paper_2502_13575_b200 as ets
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    wl = make_workload(args.workload)
+    g, tree = wl.geometry, wl.tree
+    layers = args.layers or g.num_layers
+    K, W = args.steps, args.warmup
+    headroom = K + W + 2
+    job = DecodeJob(wl, headroom=headroom, device=local, layers=layers, chunk_pages=args.chunk_pages,
+                    kernel=args.kernel, host_buffers=not args.no_e2e)
+    ctx = job.ctx
+    stats = ctx.get_stats()
+    L = tree.n_leaves
+    kv_bytes_tok = g.kv_bytes_per_token
+    qo_bytes = 2 * L * g.num_q_heads * g.head_dim * 2
+
+    def timed_loop(step_fn, sync_each):
+        job.reset_lengths()
+        for _ in range(W):
+            step_fn()
+            if sync_each:
+                torch.cuda.synchronize()
+        u_tokens = []
+        barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            step_fn()
+            u_tokens.append(job.unique_tokens())
+            if sync_each:
+                torch.cuda.synchronize()   # the host reads this step's result
+        e1.record()
+        torch.cuda.synchronize()
+        barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1))
+        return ms, float(np.mean(u_tokens))
+
+    # ---- device-resident throughput (the headline value) with clocks sampled during the region
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms_total, u_mean = timed_loop(job.step, sync_each=False)
+    clocks = sampler.stop() if rank == 0 else {}
+    ctx.poll_status()
+    ms_step = ms_total / K
+    value = world * L / (ms_step / 1000.0)
+
+    # ---- same loop with the attention and merge kernels bracketed by events on their stream
+    ctx.set_option(ets.ETS_OPT_TIMING, 1)
+    job.reset_lengths()
+    for _ in range(W):
+        job.step()
+    torch.cuda.synchronize()
+    ctx.timing_read()
+    u_tok2 = []
+    for _ in range(K):
+        job.step()
+        u_tok2.append(job.unique_tokens())
+    torch.cuda.synchronize()
+    attn_ms, merge_ms, n_calls = ctx.timing_read()
+    ctx.set_option(ets.ETS_OPT_TIMING, 0)
+    attn_ms_per_launch = attn_ms / max(n_calls, 1)
+    merge_ms_per_launch = merge_ms / max(n_calls, 1)
+    alg_bytes_launch = float(np.mean(u_tok2)) * kv_bytes_tok + qo_bytes
+    achieved = alg_bytes_launch / (attn_ms_per_launch * 1e-3) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+    traffic = None
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        try:
+            traffic = json.load(open(traffic_file)).get(args.workload)
+        except Exception:
+            traffic = None
+    roofline = {
+        "bound": "hbm", "kernel": "node-partial attention", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth", "traffic": traffic,
+        "algorithmic_bytes_per_launch": alg_bytes_launch, "us_per_launch": attn_ms_per_launch * 1e3,
+        "merge_us_per_launch": merge_ms_per_launch * 1e3, "launches_timed": int(n_calls),
+        "frac_of_nominal_8TBps": achieved / 8000.0,
+        "whole_step_gbs": (u_mean * kv_bytes_tok + qo_bytes) * layers / (ms_step * 1e-3) / 1e9,
+    }
+
+    # ---- end to end: host buffers through the *_host entry points, result read every step
+    e2e = None
+    if not args.no_e2e:
+        ms_e2e, _ = timed_loop(job.step_host, sync_each=True)
+        e2e = {"value": world * L / (ms_e2e / K / 1000.0), "unit": UNIT,
+               "h2d_bytes_per_step": job.h2d_bytes_per_step, "d2h_bytes_per_step": job.d2h_bytes_per_step,
+               "ms_per_step": ms_e2e / K}
+    ctx.poll_status()
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        v, threads, text, _ = oracle_sample(wl, layers, args.cpu_seconds)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": text}
+
+    if rank == 0:
+        cfg = workload_description(wl, layers)
+        cfg.update({"cache": "inputs larger than L2: every step streams %.2f GB of KV" %
+                             (u_mean * kv_bytes_tok * layers / 1e9),
+                    "parallelism": f"replicas x{world}, no collective",
+                    "segments": stats["n_segments"], "chunks": stats["n_chunks"], "items": stats["n_items"]})
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": cfg, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": K * layers * 3, "roofline": roofline, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

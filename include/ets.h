@@ -1,0 +1,231 @@
+/*
+ * ets.h - C ABI of the tree-decode attention library for prefix-shared paged KV.
+ *
+ * Problem statement (paper: "ETS: Efficient Tree Search for Inference-Time Scaling",
+ * arXiv 2502.13575).  A PRM-guided search keeps a tree of reasoning-step nodes; a
+ * trajectory is a root-to-leaf path, and trajectories that pass through the same node
+ * share that node's KV cache (Section 4.1; Appendix B, the node/leaf formulation of
+ * Eq. 5).  Decoding is memory-bandwidth bound and its cost is the KV that must be loaded
+ * per step (Sections 1 and 3); turning KV sharing into fewer loads needs an attention
+ * kernel that reads each shared segment once (Section 3, item 1).  This library is that
+ * step: every live leaf issues one grouped-query decode query, and its attention spans
+ * the concatenated K/V of its root-to-leaf path,
+ *
+ *     out[l,a,:] = sum_t softmax_t( sm_scale * <q[l,a,:], K_l[t, a/G, :]> ) * V_l[t, a/G, :]
+ *     lse[l,a]   = log sum_t exp( sm_scale * <q[l,a,:], K_l[t, a/G, :]> )
+ *
+ * with G = num_q_heads / num_kv_heads, no mask and no positional transform, while the
+ * tree's unique K/V is streamed from device memory once per (node, kv head), not once
+ * per leaf.  The paper itself ships no kernel and prints no attention formula; the
+ * formula above is textbook softmax attention.
+ *
+ * Conventions
+ *   - Every function returns an int32 status: ETS_OK or a negative ETS_ERR_* code.
+ *     Nothing throws, aborts or traps the device.  ets_last_error() gives a message.
+ *   - A failed call leaves the context as it was before the call.
+ *   - "HOST" / "DEVICE" below says where a pointer must point.  The library never takes
+ *     ownership of caller memory and never allocates device memory after ets_create.
+ *   - All device work is enqueued on the cuda_stream argument (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream).  Calls on one context must be issued from
+ *     one host thread at a time and, if several streams are used, ordered by the caller.
+ *   - bf16 tensors are dense, row-major, innermost index last.
+ */
+#ifndef ETS_H_
+#define ETS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ETS_OK                   0
+#define ETS_ERR_INVALID_ARG     -1  /* null pointer, negative size, index out of range      */
+#define ETS_ERR_BAD_TREE        -2  /* parent/leaf arrays do not describe a valid forest    */
+#define ETS_ERR_POOL_EXHAUSTED  -3  /* not enough pages, or a workspace bound was exceeded  */
+#define ETS_ERR_UNSUPPORTED     -4  /* geometry the kernels do not cover                    */
+#define ETS_ERR_STATE           -5  /* call order: no tree yet, host-only context, ...      */
+#define ETS_ERR_CUDA            -6  /* a CUDA runtime call failed                           */
+#define ETS_ERR_DEVICE_TIMEOUT  -7  /* a bounded device-side wait ran out                   */
+
+typedef struct ets_ctx ets_ctx; /* opaque, library-owned */
+
+/* Geometry and capacity bounds, fixed for the life of a context. */
+typedef struct ets_config {
+    int32_t num_q_heads;        /* Hq; multiple of num_kv_heads; Hq/Hkv in {1,2,4,8,16}     */
+    int32_t num_kv_heads;       /* Hkv                                                       */
+    int32_t head_dim;           /* d: 64 or 128                                              */
+    int32_t page_size;          /* tokens per page: 16                                       */
+    int32_t num_layers;         /* independent K/V pools sharing one set of tables           */
+    int32_t max_nodes;          /* bound on n_nodes of any tree                              */
+    int32_t max_leaves;         /* bound on n_leaves of any tree                             */
+    int32_t max_path_tokens;    /* bound on the token capacity summed along one path         */
+    int64_t max_path_entries;   /* bound on the sum over leaves of nodes on their path       */
+    int64_t pages_per_layer;    /* pool capacity in pages (same for every layer)             */
+    int32_t max_append_tokens;  /* bound on tokens per ets_kv_append*_host call (0: leaves)  */
+    int32_t device;             /* CUDA device ordinal; -1 = host-only context (tables only) */
+    float   sm_scale;           /* 0 -> 1/sqrt(head_dim)                                     */
+    int32_t flags;              /* reserved, must be 0                                       */
+} ets_config;
+
+/*
+ * Byte sizes of the three caller-provided DEVICE buffers for a configuration:
+ * the K pool and the V pool (num_layers * pages_per_layer pages each; a page holds
+ * page_size tokens of all KV heads, bf16, in a layout private to the library) and the
+ * workspace (tables, partial results, staging).  All three must be 1024-byte aligned
+ * (any cudaMalloc / torch allocation is).  Pool contents need no initialisation.
+ */
+int32_t ets_pool_bytes(const ets_config* cfg, size_t* k_bytes, size_t* v_bytes,
+                       size_t* workspace_bytes);
+
+/*
+ * Create a context over caller-owned DEVICE buffers that must outlive it.  With
+ * cfg->device == -1 the three pointers may be NULL and only the host-side calls
+ * (ets_tree_build, ets_tree_export, ets_work_export, ets_get_stats) are usable.
+ */
+int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* workspace,
+                   ets_ctx** out);
+int32_t ets_destroy(ets_ctx* ctx);
+
+/*
+ * Tree flatten (host).  Section 4.1: the tree of step nodes, whose shared nodes mean shared
+ * KV; Section 2.2: shared KV segments are stored once and referenced.  Replaces the current
+ * topology.
+ *   parent[n_nodes]      HOST  parent index in [-1, i): -1 = a root, parents precede children
+ *   cap_tokens[n_nodes]  HOST  tokens the node holds or will hold; it reserves
+ *                              ceil(cap/page_size) pages
+ *   keep_pages_of        HOST  nullable; keep_pages_of[i] = node index of the PREVIOUS build whose
+ *                              pages, contents and length node i inherits (clipped to its new
+ *                              capacity), or -1.  An old node may be named once.
+ *   leaf_node[n_leaves]  HOST  node each live leaf sits at; may repeat, may be internal
+ * Page rule (bit-exact, see ets_tree_export): free pages form a min-heap of ids; pages of
+ * old nodes that nobody keeps are freed first; then nodes in index order take their kept pages
+ * and pop the lowest free ids.  Every layer uses the same ids.
+ * The tables are uploaded asynchronously on cuda_stream; decode/append calls that should see
+ * the new tree must be ordered after it on that stream.
+ * Errors: ETS_ERR_BAD_TREE, ETS_ERR_POOL_EXHAUSTED (pages or a config bound), ETS_ERR_INVALID_ARG.
+ */
+int32_t ets_tree_build(ets_ctx* ctx, int32_t n_nodes, const int32_t* parent,
+                       const int32_t* cap_tokens, const int32_t* keep_pages_of,
+                       int32_t n_leaves, const int32_t* leaf_node, void* cuda_stream);
+
+/*
+ * Flattened tables, for bit-exact checks.  Counts are always written; each non-NULL HOST
+ * pointer receives the table (the caller sizes them from a first call with NULL pointers).
+ *   node_page_off[n_nodes+1], page_ids[n_pages]         pages of each node, in token order
+ *   node_leaf_off[n_nodes+1], node_leaves[n_group]      leaves below each node, ascending
+ *   leaf_path_off[n_leaves+1], leaf_path[n_path]        path of each leaf, root first
+ *   leaf_path_pos[n_path]                               leaf's position in that node's group
+ *   node_depth[n_nodes], node_len[n_nodes]              depth (root 0), current token count
+ */
+typedef struct ets_tables_host {
+    int32_t n_nodes, n_leaves;
+    int64_t n_pages, n_group, n_path;
+    int32_t *node_page_off, *page_ids, *node_leaf_off, *node_leaves;
+    int32_t *leaf_path_off, *leaf_path, *leaf_path_pos, *node_depth, *node_len;
+} ets_tables_host;
+int32_t ets_tree_export(const ets_ctx* ctx, ets_tables_host* out);
+
+/*
+ * The private work decomposition, exported for invariant checks only (its content is an
+ * implementation choice and may change): runs of chained nodes with one query group are
+ * fused into segments; segments are cut into chunks of pages; a work item is one
+ * (chunk, kv head, tile of the group's leaves).
+ *   unit[n_units*4]     per page slot: page id, node, first token index within the node, 0
+ *   item[n_items*8]     unit_begin, unit_count, kv_head, leaf_list_begin (into node_leaves),
+ *                       n_leaves_in_tile, partial_slot_of_first_leaf, chunk id, 0
+ *   leaf_slot_off[n_leaves+1], leaf_slots[n_leaf_slots]  partial slots to merge per leaf
+ */
+typedef struct ets_work_host {
+    int64_t n_units, n_items, n_leaf_slots, n_partial_slots;
+    int32_t *unit, *item, *leaf_slot_off, *leaf_slots;
+} ets_work_host;
+int32_t ets_work_export(const ets_ctx* ctx, ets_work_host* out);
+
+/*
+ * KV append.  Section 1: each trajectory needs KV state for every token it has generated;
+ * Section 3, item 3: KV of earlier steps is reused by later ones.  Appends n_new[i] tokens to
+ * node node_id[i] of one layer (distinct nodes per call), growing its length there; fails with
+ * ETS_ERR_POOL_EXHAUSTED if a node would exceed its cap_tokens.
+ *   node_id[n_items], n_new[n_items]  HOST
+ *   k_new, v_new   bf16 [sum(n_new), num_kv_heads, head_dim], items packed in order.
+ *                  DEVICE for ets_kv_append; HOST for ets_kv_append_host (copied through a
+ *                  staging area of max_append_tokens tokens; pinned memory makes the copy async)
+ * Asynchronous on cuda_stream; host arrays may be reused when the call returns, k_new/v_new
+ * after the stream has passed the call.
+ */
+int32_t ets_kv_append(ets_ctx* ctx, int32_t layer, int32_t n_items, const int32_t* node_id,
+                      const int32_t* n_new, const void* k_new, const void* v_new,
+                      void* cuda_stream);
+int32_t ets_kv_append_host(ets_ctx* ctx, int32_t layer, int32_t n_items, const int32_t* node_id,
+                           const int32_t* n_new, const void* k_new, const void* v_new,
+                           void* cuda_stream);
+/*
+ * Token lengths are tracked per (layer, node): within one decode step layer l has already
+ * received the new token while deeper layers have not, and each layer's attention must see
+ * exactly its own tokens.  ets_tree_export reports layer 0; this reads any layer's lengths
+ * into node_len[n_nodes] (HOST).
+ */
+int32_t ets_get_node_len(const ets_ctx* ctx, int32_t layer, int32_t* node_len);
+
+/*
+ * Tree-decode attention: node-partial attention over every (segment chunk, kv head, leaf tile)
+ * followed by the log-sum-exp merge along each leaf's path (the formula at the top of this
+ * file).
+ *   q    bf16 [n_leaves, num_q_heads, head_dim]
+ *   out  bf16 [n_leaves, num_q_heads, head_dim]   (fp32 result rounded to nearest even)
+ *   lse  fp32 [n_leaves, num_q_heads], natural log; nullable
+ * DEVICE pointers for ets_tree_attn_decode; HOST pointers for ets_tree_attn_decode_host, which
+ * copies q in and out/lse back on the same stream (the results are valid once the stream has
+ * passed the call).  A leaf whose path holds no token yields zeros and lse = -inf.
+ * Errors: ETS_ERR_STATE (no tree), ETS_ERR_INVALID_ARG, ETS_ERR_CUDA.
+ */
+int32_t ets_tree_attn_decode(ets_ctx* ctx, int32_t layer, const void* q, void* out, float* lse,
+                             void* cuda_stream);
+int32_t ets_tree_attn_decode_host(ets_ctx* ctx, int32_t layer, const void* q, void* out,
+                                  float* lse, void* cuda_stream);
+
+/*
+ * Read one node's current K and V rows of one layer back in token order:
+ * bf16 [node_len, num_kv_heads, head_dim] each, DEVICE pointers (either may be NULL).
+ */
+int32_t ets_kv_read_debug(ets_ctx* ctx, int32_t layer, int32_t node, void* k_out, void* v_out,
+                          void* cuda_stream);
+
+/* Counters of the current tree.  "KV size" follows Section 3: the unique KV state of the tree. */
+typedef struct ets_stats {
+    int64_t n_nodes, n_leaves;
+    int64_t unique_tokens;      /* sum over nodes of current length (layer 0)                */
+    int64_t unique_kv_bytes;    /* unique_tokens * 2 * Hkv * d * 2, one layer                */
+    int64_t path_tokens;        /* sum over leaves of tokens on their path: what a kernel    */
+                                /* without prefix sharing would read                         */
+    int64_t pages_used, pages_free;
+    int64_t n_segments, n_chunks, n_items, n_units, n_partial_slots;
+    int64_t attended_tokens;    /* current tokens of nodes that have a leaf below them       */
+} ets_stats;
+int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
+
+/* Tuning and instrumentation knobs; unknown keys give ETS_ERR_INVALID_ARG. */
+#define ETS_OPT_CHUNK_PAGES   1  /* pages per chunk (0 = automatic); applies at the next build   */
+#define ETS_OPT_KERNEL        2  /* 0 automatic, 1 scalar-FMA kernel only                       */
+#define ETS_OPT_TIMING        3  /* 1: bracket the attention and merge kernels with events      */
+int32_t ets_set_option(ets_ctx* ctx, int32_t key, int64_t value);
+
+/* With ETS_OPT_TIMING on: waits for the recorded events, returns and clears the sums. */
+int32_t ets_timing_read(ets_ctx* ctx, double* attn_ms, double* merge_ms, int64_t* n_calls);
+
+/*
+ * Synchronise cuda_stream and report the device-side status word: ETS_OK, or
+ * ETS_ERR_DEVICE_TIMEOUT / ETS_ERR_INVALID_ARG if a kernel gave up on a bounded wait or
+ * skipped an out-of-range table entry.  Clears the word.
+ */
+int32_t ets_poll_status(ets_ctx* ctx, void* cuda_stream);
+
+const char* ets_last_error(const ets_ctx* ctx);
+const char* ets_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ETS_H_ */

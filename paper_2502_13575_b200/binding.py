@@ -1,0 +1,292 @@
+"""ctypes binding of the C ABI declared in include/ets.h.
+
+Argument marshalling only: every step of the path (tree flatten, KV append, node-partial
+attention, log-sum-exp merge) runs inside libets_b200.so.  Functions carry the C names.
+PyTorch is used for device memory and streams, nothing else.  If the shared library is
+missing this module raises at import time; there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+ETS_OK = 0
+ETS_ERR_INVALID_ARG = -1
+ETS_ERR_BAD_TREE = -2
+ETS_ERR_POOL_EXHAUSTED = -3
+ETS_ERR_UNSUPPORTED = -4
+ETS_ERR_STATE = -5
+ETS_ERR_CUDA = -6
+ETS_ERR_DEVICE_TIMEOUT = -7
+
+ETS_OPT_CHUNK_PAGES = 1
+ETS_OPT_KERNEL = 2
+ETS_OPT_TIMING = 3
+
+_ERR_NAMES = {
+    -1: "ETS_ERR_INVALID_ARG", -2: "ETS_ERR_BAD_TREE", -3: "ETS_ERR_POOL_EXHAUSTED",
+    -4: "ETS_ERR_UNSUPPORTED", -5: "ETS_ERR_STATE", -6: "ETS_ERR_CUDA", -7: "ETS_ERR_DEVICE_TIMEOUT",
+}
+
+
+class EtsError(RuntimeError):
+    def __init__(self, code: int, message: str = ""):
+        self.code = int(code)
+        super().__init__(f"{_ERR_NAMES.get(self.code, self.code)}: {message}")
+
+
+class ets_config(C.Structure):
+    _fields_ = [
+        ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+        ("page_size", C.c_int32), ("num_layers", C.c_int32), ("max_nodes", C.c_int32),
+        ("max_leaves", C.c_int32), ("max_path_tokens", C.c_int32),
+        ("max_path_entries", C.c_int64), ("pages_per_layer", C.c_int64),
+        ("max_append_tokens", C.c_int32), ("device", C.c_int32), ("sm_scale", C.c_float),
+        ("flags", C.c_int32),
+    ]
+
+
+_I32P = C.POINTER(C.c_int32)
+
+
+class ets_tables_host(C.Structure):
+    _fields_ = [
+        ("n_nodes", C.c_int32), ("n_leaves", C.c_int32),
+        ("n_pages", C.c_int64), ("n_group", C.c_int64), ("n_path", C.c_int64),
+        ("node_page_off", _I32P), ("page_ids", _I32P), ("node_leaf_off", _I32P), ("node_leaves", _I32P),
+        ("leaf_path_off", _I32P), ("leaf_path", _I32P), ("leaf_path_pos", _I32P),
+        ("node_depth", _I32P), ("node_len", _I32P),
+    ]
+
+
+class ets_work_host(C.Structure):
+    _fields_ = [
+        ("n_units", C.c_int64), ("n_items", C.c_int64), ("n_leaf_slots", C.c_int64),
+        ("n_partial_slots", C.c_int64),
+        ("unit", _I32P), ("item", _I32P), ("leaf_slot_off", _I32P), ("leaf_slots", _I32P),
+    ]
+
+
+class ets_stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "n_nodes", "n_leaves", "unique_tokens", "unique_kv_bytes", "path_tokens", "pages_used",
+        "pages_free", "n_segments", "n_chunks", "n_items", "n_units", "n_partial_slots",
+        "attended_tokens")]
+
+
+# every symbol include/ets.h declares, with its C signature
+_SIGNATURES = {
+    "ets_pool_bytes": (C.c_int32, [C.POINTER(ets_config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "ets_create": (C.c_int32, [C.POINTER(ets_config), C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p)]),
+    "ets_destroy": (C.c_int32, [C.c_void_p]),
+    "ets_tree_build": (C.c_int32, [C.c_void_p, C.c_int32, _I32P, _I32P, _I32P, C.c_int32, _I32P, C.c_void_p]),
+    "ets_tree_export": (C.c_int32, [C.c_void_p, C.POINTER(ets_tables_host)]),
+    "ets_work_export": (C.c_int32, [C.c_void_p, C.POINTER(ets_work_host)]),
+    "ets_kv_append": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, _I32P, _I32P, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ets_kv_append_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, _I32P, _I32P, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ets_get_node_len": (C.c_int32, [C.c_void_p, C.c_int32, _I32P]),
+    "ets_tree_attn_decode": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ets_tree_attn_decode_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ets_kv_read_debug": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ets_get_stats": (C.c_int32, [C.c_void_p, C.POINTER(ets_stats)]),
+    "ets_set_option": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int64]),
+    "ets_timing_read": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "ets_poll_status": (C.c_int32, [C.c_void_p, C.c_void_p]),
+    "ets_last_error": (C.c_char_p, [C.c_void_p]),
+    "ets_version": (C.c_char_p, []),
+}
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2502_13575_b200.build` "
+            "(there is no fallback path)")
+    lib = C.CDLL(path)
+    for name, (res, args) in _SIGNATURES.items():
+        fn = getattr(lib, name)  # AttributeError if the library does not export it
+        fn.restype = res
+        fn.argtypes = args
+    return lib
+
+
+lib = _load()
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(_I32P)
+
+
+def _dev_ptr(t) -> Optional[int]:
+    """Device (or host) address of a torch tensor / numpy array / raw int; None passes NULL."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        assert t.flags["C_CONTIGUOUS"]
+        return t.ctypes.data
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        if torch.cuda.is_available():
+            return torch.cuda.current_stream().cuda_stream or None
+        return None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def make_config(num_q_heads: int, num_kv_heads: int, head_dim: int, *, num_layers: int = 1,
+                max_nodes: int, max_leaves: int, max_path_tokens: int, max_path_entries: int,
+                pages_per_layer: int, page_size: int = 16, max_append_tokens: int = 0,
+                device: int = 0, sm_scale: float = 0.0) -> ets_config:
+    return ets_config(num_q_heads, num_kv_heads, head_dim, page_size, num_layers, max_nodes, max_leaves,
+                      max_path_tokens, max_path_entries, pages_per_layer, max_append_tokens, device,
+                      sm_scale, 0)
+
+
+def ets_version() -> str:
+    return lib.ets_version().decode()
+
+
+def ets_pool_bytes(cfg: ets_config):
+    k, v, w = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    rc = lib.ets_pool_bytes(C.byref(cfg), C.byref(k), C.byref(v), C.byref(w))
+    if rc != ETS_OK:
+        raise EtsError(rc, "ets_pool_bytes")
+    return k.value, v.value, w.value
+
+
+class EtsContext:
+    """Owns the device buffers (torch allocations) and the opaque ets_ctx handle.  Method names
+    are the C entry points without the `ets_` prefix; each one is a single C call."""
+
+    def __init__(self, cfg: ets_config):
+        self.cfg = cfg
+        self._h = C.c_void_p()
+        kb, vb, wb = ets_pool_bytes(cfg)
+        self.k_pool = self.v_pool = self.workspace = None
+        if cfg.device >= 0:
+            import torch
+            dev = torch.device("cuda", cfg.device)
+            self.k_pool = torch.empty(kb, dtype=torch.uint8, device=dev)
+            self.v_pool = torch.empty(vb, dtype=torch.uint8, device=dev)
+            self.workspace = torch.empty(wb, dtype=torch.uint8, device=dev)
+        rc = lib.ets_create(C.byref(cfg), _dev_ptr(self.k_pool), _dev_ptr(self.v_pool),
+                            _dev_ptr(self.workspace), C.byref(self._h))
+        if rc != ETS_OK:
+            raise EtsError(rc, "ets_create")
+
+    # -- plumbing
+    def _check(self, rc: int):
+        if rc != ETS_OK:
+            raise EtsError(rc, lib.ets_last_error(self._h).decode())
+
+    def close(self):
+        if self._h:
+            lib.ets_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- C entry points
+    def tree_build(self, parent, cap_tokens, leaf_node, keep_pages_of=None, stream=None):
+        parent, cap, leaves = _i32(parent), _i32(cap_tokens), _i32(leaf_node)
+        keep = None if keep_pages_of is None else _i32(keep_pages_of)
+        if cap.shape != parent.shape or (keep is not None and keep.shape != parent.shape):
+            raise EtsError(ETS_ERR_INVALID_ARG, "array lengths differ")
+        self._check(lib.ets_tree_build(self._h, parent.shape[0], _p(parent), _p(cap), _p(keep),
+                                       leaves.shape[0], _p(leaves), _stream_ptr(stream)))
+
+    def tree_export(self) -> Dict[str, np.ndarray]:
+        t = ets_tables_host()
+        self._check(lib.ets_tree_export(self._h, C.byref(t)))
+        sizes = {
+            "node_page_off": t.n_nodes + 1, "page_ids": t.n_pages, "node_leaf_off": t.n_nodes + 1,
+            "node_leaves": t.n_group, "leaf_path_off": t.n_leaves + 1, "leaf_path": t.n_path,
+            "leaf_path_pos": t.n_path, "node_depth": t.n_nodes, "node_len": t.n_nodes,
+        }
+        out = {k: np.zeros(n, dtype=np.int32) for k, n in sizes.items()}
+        for k, a in out.items():
+            setattr(t, k, _p(a))
+        self._check(lib.ets_tree_export(self._h, C.byref(t)))
+        return out
+
+    def work_export(self) -> Dict[str, np.ndarray]:
+        w = ets_work_host()
+        self._check(lib.ets_work_export(self._h, C.byref(w)))
+        n_leaves = self.get_stats()["n_leaves"]
+        out = {
+            "unit": np.zeros(w.n_units * 4, np.int32), "item": np.zeros(w.n_items * 8, np.int32),
+            "leaf_slot_off": np.zeros(n_leaves + 1, np.int32), "leaf_slots": np.zeros(w.n_leaf_slots, np.int32),
+        }
+        for k, a in out.items():
+            setattr(w, k, _p(a))
+        self._check(lib.ets_work_export(self._h, C.byref(w)))
+        out["unit"] = out["unit"].reshape(-1, 4)
+        out["item"] = out["item"].reshape(-1, 8)
+        out["n_partial_slots"] = int(w.n_partial_slots)
+        return out
+
+    def get_node_len(self, layer: int = 0) -> np.ndarray:
+        n = self.get_stats()["n_nodes"]
+        a = np.zeros(n, np.int32)
+        self._check(lib.ets_get_node_len(self._h, layer, _p(a)))
+        return a
+
+    def kv_append(self, layer: int, node_id, n_new, k_new, v_new, stream=None):
+        node_id, n_new = _i32(node_id), _i32(n_new)
+        self._check(lib.ets_kv_append(self._h, layer, node_id.shape[0], _p(node_id), _p(n_new),
+                                      _dev_ptr(k_new), _dev_ptr(v_new), _stream_ptr(stream)))
+
+    def kv_append_host(self, layer: int, node_id, n_new, k_new, v_new, stream=None):
+        node_id, n_new = _i32(node_id), _i32(n_new)
+        self._check(lib.ets_kv_append_host(self._h, layer, node_id.shape[0], _p(node_id), _p(n_new),
+                                           _dev_ptr(k_new), _dev_ptr(v_new), _stream_ptr(stream)))
+
+    def tree_attn_decode(self, layer: int, q, out, lse=None, stream=None):
+        self._check(lib.ets_tree_attn_decode(self._h, layer, _dev_ptr(q), _dev_ptr(out), _dev_ptr(lse),
+                                             _stream_ptr(stream)))
+
+    def tree_attn_decode_host(self, layer: int, q, out, lse=None, stream=None):
+        self._check(lib.ets_tree_attn_decode_host(self._h, layer, _dev_ptr(q), _dev_ptr(out), _dev_ptr(lse),
+                                                  _stream_ptr(stream)))
+
+    def kv_read_debug(self, layer: int, node: int, k_out, v_out, stream=None):
+        self._check(lib.ets_kv_read_debug(self._h, layer, node, _dev_ptr(k_out), _dev_ptr(v_out),
+                                          _stream_ptr(stream)))
+
+    def get_stats(self) -> Dict[str, int]:
+        s = ets_stats()
+        self._check(lib.ets_get_stats(self._h, C.byref(s)))
+        return {n: int(getattr(s, n)) for n, _ in ets_stats._fields_}
+
+    def set_option(self, key: int, value: int):
+        self._check(lib.ets_set_option(self._h, key, value))
+
+    def timing_read(self):
+        a, m, n = C.c_double(), C.c_double(), C.c_int64()
+        self._check(lib.ets_timing_read(self._h, C.byref(a), C.byref(m), C.byref(n)))
+        return a.value, m.value, n.value
+
+    def poll_status(self, stream=None):
+        self._check(lib.ets_poll_status(self._h, _stream_ptr(stream)))

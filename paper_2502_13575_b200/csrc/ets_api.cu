@@ -1,0 +1,636 @@
+// C ABI of the library (see include/ets.h): context, workspace carving, table upload,
+// launches.  No torch types, no exceptions across the boundary.
+#include "../../include/ets.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "ets_device.cuh"
+#include "ets_flatten.hpp"
+
+static_assert(ETS_ERR_INVALID_ARG == ets::F_INVALID && ETS_ERR_BAD_TREE == ets::F_BAD_TREE &&
+                  ETS_ERR_POOL_EXHAUSTED == ets::F_EXHAUSTED, "status codes out of sync");
+static_assert(sizeof(ets::Item) == 32 && sizeof(ets::DevItem) == 32, "item layout");
+
+namespace {
+
+constexpr int kStages = 3;        // pinned staging buffers for table uploads
+constexpr int kDescSlots = 8;     // pinned/device descriptor slots for appends
+constexpr int kTimingCap = 8192;  // decode calls that can be timed between two reads
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {  // byte offsets inside the workspace
+    size_t blob, blob_cap;
+    size_t desc, desc_slot_bytes;
+    size_t part_ml, part_o;
+    size_t q_stage, out_stage, lse_stage, k_stage, v_stage;
+    size_t status;
+    size_t total;
+    int64_t max_partial_slots, max_items, max_units;
+    int32_t max_append_tokens;
+};
+
+bool config_ok(const ets_config* c, std::string& why) {
+    if (!c) { why = "null config"; return false; }
+    if (c->num_q_heads <= 0 || c->num_kv_heads <= 0 || c->num_q_heads % c->num_kv_heads) {
+        why = "num_q_heads must be a positive multiple of num_kv_heads"; return false;
+    }
+    if (c->num_layers <= 0 || c->max_nodes <= 0 || c->max_leaves <= 0 || c->pages_per_layer <= 0 ||
+        c->max_path_entries <= 0 || c->max_path_tokens <= 0 || c->max_append_tokens < 0) {
+        why = "capacity bounds must be positive"; return false;
+    }
+    if (c->flags != 0) { why = "flags must be 0"; return false; }
+    if (c->pages_per_layer > 0x7fffffffLL) { why = "pages_per_layer too large"; return false; }
+    return true;
+}
+
+int32_t config_supported(const ets_config* c, std::string& why) {
+    int g = c->num_q_heads / c->num_kv_heads;
+    if (c->head_dim != 64 && c->head_dim != 128) { why = "head_dim must be 64 or 128"; return ETS_ERR_UNSUPPORTED; }
+    if (c->page_size <= 0) { why = "page_size must be positive"; return ETS_ERR_UNSUPPORTED; }
+    // the kernels are written for 16-token pages; a host-only context may flatten with any size
+    if (c->device >= 0 && c->page_size != ets::kPageTokens) { why = "page_size must be 16"; return ETS_ERR_UNSUPPORTED; }
+    if (!(g == 1 || g == 2 || g == 4 || g == 8 || g == 16)) {
+        why = "num_q_heads/num_kv_heads must be 1, 2, 4, 8 or 16"; return ETS_ERR_UNSUPPORTED;
+    }
+    return ETS_OK;
+}
+
+Layout make_layout(const ets_config* c) {
+    Layout L{};
+    const int64_t path_pages = (int64_t)c->max_leaves * ((c->max_path_tokens + c->page_size - 1) / c->page_size) +
+                               c->max_path_entries;
+    L.max_partial_slots = c->max_path_entries + (path_pages + 7) / 8;
+    L.max_items = L.max_partial_slots * c->num_kv_heads;
+    L.max_units = c->pages_per_layer;
+    L.max_append_tokens = c->max_append_tokens > 0 ? c->max_append_tokens : c->max_leaves;
+    const size_t A = 1024;
+    size_t blob = 0;
+    blob += align_up((size_t)L.max_units * 16, 256);
+    blob += align_up((size_t)L.max_items * 32, 256);
+    blob += align_up(((size_t)c->max_nodes + 1) * 4, 256);          // node_page_off
+    blob += align_up((size_t)c->pages_per_layer * 4, 256);          // page_ids
+    blob += align_up((size_t)c->max_path_entries * 4, 256);         // node_leaves
+    blob += align_up(((size_t)c->max_leaves + 1) * 4, 256);         // leaf_slot_off
+    blob += align_up((size_t)L.max_partial_slots * 4, 256);         // leaf_slots
+    blob += align_up((size_t)c->num_layers * c->max_nodes * 4, 256);  // node_len
+    L.blob_cap = align_up(blob, A);
+    size_t off = 0;
+    L.blob = off; off += L.blob_cap;
+    L.desc_slot_bytes = align_up((size_t)c->max_nodes * 16, 256);
+    L.desc = off; off += align_up(L.desc_slot_bytes * kDescSlots, A);
+    const size_t rows = (size_t)L.max_partial_slots * c->num_q_heads;
+    L.part_ml = off; off += align_up(rows * 8, A);
+    L.part_o = off; off += align_up(rows * c->head_dim * 4, A);
+    const size_t qbytes = (size_t)c->max_leaves * c->num_q_heads * c->head_dim * 2;
+    L.q_stage = off; off += align_up(qbytes, A);
+    L.out_stage = off; off += align_up(qbytes, A);
+    L.lse_stage = off; off += align_up((size_t)c->max_leaves * c->num_q_heads * 4, A);
+    const size_t kvb = (size_t)L.max_append_tokens * c->num_kv_heads * c->head_dim * 2;
+    L.k_stage = off; off += align_up(kvb, A);
+    L.v_stage = off; off += align_up(kvb, A);
+    L.status = off; off += A;
+    L.total = off;
+    return L;
+}
+
+struct BlobOffsets {  // offsets of the packed tables of the current tree inside the device blob
+    size_t units, items, node_page_off, page_ids, node_leaves, leaf_slot_off, leaf_slots, node_len, total;
+    int32_t len_stride;
+};
+
+}  // namespace
+
+struct ets_ctx {
+    ets_config cfg{};
+    ets::FlattenParams fp{};
+    Layout lay{};
+    ets::Tree tree;
+    bool has_tree = false;
+    bool host_only = true;
+    int sm_count = 148;
+    char* k_pool = nullptr;
+    char* v_pool = nullptr;
+    char* ws = nullptr;
+    size_t layer_pool_bytes = 0;
+    float scale_log2 = 0.f;
+    BlobOffsets bo{};
+    // pinned staging for table uploads
+    char* stage_host[kStages] = {nullptr, nullptr, nullptr};
+    cudaEvent_t stage_ev[kStages] = {nullptr, nullptr, nullptr};
+    bool stage_used[kStages] = {false, false, false};
+    int stage_next = 0;
+    // pinned descriptor slots for appends
+    int4* desc_host[kDescSlots] = {};
+    cudaEvent_t desc_ev[kDescSlots] = {};
+    bool desc_used[kDescSlots] = {};
+    int desc_next = 0;
+    int32_t* status_host = nullptr;  // pinned, target of the status read-back
+    // options
+    int32_t opt_chunk_pages = 0;
+    int32_t opt_kernel = 0;
+    bool opt_timing = false;
+    // timing
+    std::vector<cudaEvent_t> tev;   // 3 per timed call
+    int64_t timed_calls = 0;
+    double acc_attn_ms = 0, acc_merge_ms = 0;
+    int64_t acc_calls = 0;
+    std::string err;
+};
+
+namespace {
+
+int32_t fail(ets_ctx* c, int32_t code, const std::string& msg) {
+    if (c) c->err = msg;
+    return code;
+}
+
+int32_t cuda_fail(ets_ctx* c, cudaError_t e, const char* what) {
+    return fail(c, ETS_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define ETS_CUDA(ctx, call)                                        \
+    do {                                                           \
+        cudaError_t e__ = (call);                                  \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call); \
+    } while (0)
+
+BlobOffsets pack_offsets(const ets_ctx* c, const ets::Tree& t) {
+    BlobOffsets b{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
+    b.units = take(t.unit.size() * 4);
+    b.items = take(t.items.size() * sizeof(ets::Item));
+    b.node_page_off = take(t.node_page_off.size() * 4);
+    b.page_ids = take(t.page_ids.size() * 4);
+    b.node_leaves = take(t.node_leaves.size() * 4);
+    b.leaf_slot_off = take(t.leaf_slot_off.size() * 4);
+    b.leaf_slots = take(t.leaf_slots.size() * 4);
+    b.len_stride = t.n_nodes > 0 ? t.n_nodes : 1;
+    b.node_len = take((size_t)c->cfg.num_layers * b.len_stride * 4);
+    b.total = off;
+    return b;
+}
+
+void pack_blob(const ets_ctx* c, const ets::Tree& t, const BlobOffsets& b, char* dst) {
+    auto put = [&](size_t off, const void* src, size_t bytes) { if (bytes) std::memcpy(dst + off, src, bytes); };
+    put(b.units, t.unit.data(), t.unit.size() * 4);
+    put(b.items, t.items.data(), t.items.size() * sizeof(ets::Item));
+    put(b.node_page_off, t.node_page_off.data(), t.node_page_off.size() * 4);
+    put(b.page_ids, t.page_ids.data(), t.page_ids.size() * 4);
+    put(b.node_leaves, t.node_leaves.data(), t.node_leaves.size() * 4);
+    put(b.leaf_slot_off, t.leaf_slot_off.data(), t.leaf_slot_off.size() * 4);
+    put(b.leaf_slots, t.leaf_slots.data(), t.leaf_slots.size() * 4);
+    for (int l = 0; l < c->cfg.num_layers; ++l)
+        put(b.node_len + (size_t)l * b.len_stride * 4, t.len[l].data(), t.len[l].size() * 4);
+}
+
+template <typename T>
+const T* blob_ptr(const ets_ctx* c, size_t off) { return reinterpret_cast<const T*>(c->ws + c->lay.blob + off); }
+
+}  // namespace
+
+extern "C" {
+
+const char* ets_version(void) { return "ets-b200 0.1"; }
+
+const char* ets_last_error(const ets_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int32_t ets_pool_bytes(const ets_config* cfg, size_t* k_bytes, size_t* v_bytes, size_t* workspace_bytes) {
+    std::string why;
+    if (!config_ok(cfg, why)) return ETS_ERR_INVALID_ARG;
+    if (int32_t rc = config_supported(cfg, why)) return rc;
+    const size_t pool = (size_t)cfg->num_layers * (size_t)cfg->pages_per_layer * cfg->num_kv_heads *
+                        ets::tile_bytes(cfg->head_dim);
+    if (k_bytes) *k_bytes = pool;
+    if (v_bytes) *v_bytes = pool;
+    if (workspace_bytes) *workspace_bytes = make_layout(cfg).total;
+    return ETS_OK;
+}
+
+int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* workspace, ets_ctx** out) {
+    if (!out) return ETS_ERR_INVALID_ARG;
+    *out = nullptr;
+    std::string why;
+    if (!config_ok(cfg, why)) return ETS_ERR_INVALID_ARG;
+    if (int32_t rc = config_supported(cfg, why)) return rc;
+    const bool host_only = cfg->device < 0;
+    if (!host_only) {
+        if (!k_pool || !v_pool || !workspace) return ETS_ERR_INVALID_ARG;
+        if (((uintptr_t)k_pool | (uintptr_t)v_pool | (uintptr_t)workspace) & 1023) return ETS_ERR_INVALID_ARG;
+    }
+    ets_ctx* c = new (std::nothrow) ets_ctx();
+    if (!c) return ETS_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->host_only = host_only;
+    c->lay = make_layout(cfg);
+    c->k_pool = (char*)k_pool;
+    c->v_pool = (char*)v_pool;
+    c->ws = (char*)workspace;
+    c->layer_pool_bytes = (size_t)cfg->pages_per_layer * cfg->num_kv_heads * ets::tile_bytes(cfg->head_dim);
+    const float sm = cfg->sm_scale != 0.f ? cfg->sm_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+    c->scale_log2 = sm * 1.4426950408889634f;
+    c->fp.num_kv_heads = cfg->num_kv_heads;
+    c->fp.gqa = cfg->num_q_heads / cfg->num_kv_heads;
+    c->fp.page_size = cfg->page_size;
+    c->fp.num_layers = cfg->num_layers;
+    c->fp.max_nodes = cfg->max_nodes;
+    c->fp.max_leaves = cfg->max_leaves;
+    c->fp.max_path_entries = cfg->max_path_entries;
+    c->fp.max_partial_slots = c->lay.max_partial_slots;
+    c->fp.max_items = c->lay.max_items;
+    c->fp.rows_per_item = 16;
+    if (!host_only) {
+        cudaError_t e = cudaSetDevice(cfg->device);
+        cudaDeviceProp prop{};
+        if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, cfg->device);
+        if (e == cudaSuccess) {
+            c->sm_count = prop.multiProcessorCount;
+            for (int i = 0; i < kStages && e == cudaSuccess; ++i) {
+                e = cudaHostAlloc((void**)&c->stage_host[i], c->lay.blob_cap, cudaHostAllocDefault);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->stage_ev[i], cudaEventDisableTiming);
+            }
+            for (int i = 0; i < kDescSlots && e == cudaSuccess; ++i) {
+                e = cudaHostAlloc((void**)&c->desc_host[i], c->lay.desc_slot_bytes, cudaHostAllocDefault);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->desc_ev[i], cudaEventDisableTiming);
+            }
+            if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->status_host, 64, cudaHostAllocDefault);
+            if (e == cudaSuccess) e = cudaMemset(c->ws + c->lay.status, 0, 1024);
+        }
+        if (e != cudaSuccess) {
+            ets_destroy(c);
+            return ETS_ERR_CUDA;
+        }
+    }
+    c->fp.n_workers = c->sm_count;
+    ets::tree_init(c->tree, c->fp, cfg->pages_per_layer);
+    *out = c;
+    return ETS_OK;
+}
+
+int32_t ets_destroy(ets_ctx* c) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    if (!c->host_only) {
+        cudaSetDevice(c->cfg.device);
+        cudaDeviceSynchronize();
+        for (int i = 0; i < kStages; ++i) {
+            if (c->stage_host[i]) cudaFreeHost(c->stage_host[i]);
+            if (c->stage_ev[i]) cudaEventDestroy(c->stage_ev[i]);
+        }
+        for (int i = 0; i < kDescSlots; ++i) {
+            if (c->desc_host[i]) cudaFreeHost(c->desc_host[i]);
+            if (c->desc_ev[i]) cudaEventDestroy(c->desc_ev[i]);
+        }
+        if (c->status_host) cudaFreeHost(c->status_host);
+        for (cudaEvent_t e : c->tev) cudaEventDestroy(e);
+    }
+    delete c;
+    return ETS_OK;
+}
+
+int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    switch (key) {
+        case ETS_OPT_CHUNK_PAGES:
+            if (value < 0 || value > 4096) return fail(c, ETS_ERR_INVALID_ARG, "chunk pages out of range");
+            c->opt_chunk_pages = (int32_t)value;
+            return ETS_OK;
+        case ETS_OPT_KERNEL:
+            if (value < 0 || value > 1) return fail(c, ETS_ERR_INVALID_ARG, "unknown kernel selector");
+            c->opt_kernel = (int32_t)value;
+            return ETS_OK;
+        case ETS_OPT_TIMING:
+            if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+            c->opt_timing = value != 0;
+            return ETS_OK;
+        default:
+            return fail(c, ETS_ERR_INVALID_ARG, "unknown option");
+    }
+}
+
+int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const int32_t* cap_tokens,
+                       const int32_t* keep_pages_of, int32_t n_leaves, const int32_t* leaf_node,
+                       void* cuda_stream) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    ets::FlattenParams fp = c->fp;
+    fp.chunk_pages = c->opt_chunk_pages;
+    ets::Tree next;
+    std::string err;
+    int32_t rc = ets::tree_build(c->tree, fp, n_nodes, parent, cap_tokens, keep_pages_of, n_leaves, leaf_node,
+                                 next, err);
+    if (rc != ETS_OK) return fail(c, rc, err);
+    if ((int64_t)(next.unit.size() / 4) > c->lay.max_units)
+        return fail(c, ETS_ERR_POOL_EXHAUSTED, "page slots exceed the workspace bound");
+    BlobOffsets bo = pack_offsets(c, next);
+    if (bo.total > c->lay.blob_cap) return fail(c, ETS_ERR_POOL_EXHAUSTED, "tables exceed the workspace bound");
+    if (!c->host_only) {
+        cudaStream_t s = (cudaStream_t)cuda_stream;
+        ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+        const int i = c->stage_next;
+        if (c->stage_used[i]) ETS_CUDA(c, cudaEventSynchronize(c->stage_ev[i]));
+        pack_blob(c, next, bo, c->stage_host[i]);
+        ETS_CUDA(c, cudaMemcpyAsync(c->ws + c->lay.blob, c->stage_host[i], bo.total, cudaMemcpyHostToDevice, s));
+        ETS_CUDA(c, cudaEventRecord(c->stage_ev[i], s));
+        c->stage_used[i] = true;
+        c->stage_next = (i + 1) % kStages;
+    }
+    c->tree = std::move(next);
+    c->bo = bo;
+    c->has_tree = true;
+    return ETS_OK;
+}
+
+int32_t ets_tree_export(const ets_ctx* c, ets_tables_host* o) {
+    if (!c || !o) return ETS_ERR_INVALID_ARG;
+    const ets::Tree& t = c->tree;
+    o->n_nodes = t.n_nodes;
+    o->n_leaves = t.n_leaves;
+    o->n_pages = (int64_t)t.page_ids.size();
+    o->n_group = (int64_t)t.node_leaves.size();
+    o->n_path = (int64_t)t.leaf_path.size();
+    auto cp = [](int32_t* dst, const std::vector<int32_t>& v) { if (dst && !v.empty()) std::memcpy(dst, v.data(), v.size() * 4); };
+    cp(o->node_page_off, t.node_page_off);
+    cp(o->page_ids, t.page_ids);
+    cp(o->node_leaf_off, t.node_leaf_off);
+    cp(o->node_leaves, t.node_leaves);
+    cp(o->leaf_path_off, t.leaf_path_off);
+    cp(o->leaf_path, t.leaf_path);
+    cp(o->leaf_path_pos, t.leaf_path_pos);
+    cp(o->node_depth, t.depth);
+    if (!t.len.empty()) cp(o->node_len, t.len[0]);
+    return ETS_OK;
+}
+
+int32_t ets_work_export(const ets_ctx* c, ets_work_host* o) {
+    if (!c || !o) return ETS_ERR_INVALID_ARG;
+    const ets::Tree& t = c->tree;
+    o->n_units = (int64_t)t.unit.size() / 4;
+    o->n_items = (int64_t)t.items.size();
+    o->n_leaf_slots = (int64_t)t.leaf_slots.size();
+    o->n_partial_slots = t.n_partial_slots;
+    if (o->unit && !t.unit.empty()) std::memcpy(o->unit, t.unit.data(), t.unit.size() * 4);
+    if (o->item && !t.items.empty()) std::memcpy(o->item, t.items.data(), t.items.size() * sizeof(ets::Item));
+    if (o->leaf_slot_off) std::memcpy(o->leaf_slot_off, t.leaf_slot_off.data(), t.leaf_slot_off.size() * 4);
+    if (o->leaf_slots && !t.leaf_slots.empty()) std::memcpy(o->leaf_slots, t.leaf_slots.data(), t.leaf_slots.size() * 4);
+    return ETS_OK;
+}
+
+int32_t ets_get_node_len(const ets_ctx* c, int32_t layer, int32_t* node_len) {
+    if (!c || !node_len || layer < 0 || layer >= c->cfg.num_layers) return ETS_ERR_INVALID_ARG;
+    const auto& v = c->tree.len[layer];
+    if (!v.empty()) std::memcpy(node_len, v.data(), v.size() * 4);
+    return ETS_OK;
+}
+
+int32_t ets_get_stats(const ets_ctx* c, ets_stats* o) {
+    if (!c || !o) return ETS_ERR_INVALID_ARG;
+    const ets::Tree& t = c->tree;
+    std::memset(o, 0, sizeof(*o));
+    o->n_nodes = t.n_nodes;
+    o->n_leaves = t.n_leaves;
+    std::vector<int64_t> cum((size_t)t.n_nodes, 0);
+    for (int32_t i = 0; i < t.n_nodes; ++i) {
+        const int32_t len = t.len[0][i];
+        o->unique_tokens += len;
+        cum[i] = len + (t.parent[i] >= 0 ? cum[t.parent[i]] : 0);
+        if (t.node_leaf_off[i + 1] > t.node_leaf_off[i]) o->attended_tokens += len;
+    }
+    for (int32_t l = 0; l < t.n_leaves; ++l) o->path_tokens += cum[t.leaf_node[l]];
+    o->unique_kv_bytes = o->unique_tokens * 2 * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
+    o->pages_used = (int64_t)t.page_ids.size();
+    o->pages_free = (int64_t)t.free_heap.size();
+    o->n_segments = t.n_segments;
+    o->n_chunks = t.n_chunks;
+    o->n_items = (int64_t)t.items.size();
+    o->n_units = (int64_t)t.unit.size() / 4;
+    o->n_partial_slots = t.n_partial_slots;
+    return ETS_OK;
+}
+
+static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int32_t* node_id,
+                           const int32_t* n_new, const void* k_new, const void* v_new, bool host_src,
+                           cudaStream_t s) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+    if (!c->has_tree) return fail(c, ETS_ERR_STATE, "no tree built");
+    if (layer < 0 || layer >= c->cfg.num_layers || n_items < 0) return fail(c, ETS_ERR_INVALID_ARG, "layer or count");
+    if (n_items == 0) return ETS_OK;
+    if (!node_id || !n_new || !k_new || !v_new) return fail(c, ETS_ERR_INVALID_ARG, "null array");
+    if (((uintptr_t)k_new | (uintptr_t)v_new) & 15) return fail(c, ETS_ERR_INVALID_ARG, "k_new/v_new must be 16-byte aligned");
+    if (n_items > c->cfg.max_nodes) return fail(c, ETS_ERR_INVALID_ARG, "more items than nodes");
+    ets::Tree& t = c->tree;
+    std::vector<int32_t>& len = t.len[layer];
+    // validate everything before touching any state
+    int64_t total = 0;
+    int32_t max_new = 0;
+    std::vector<char> seen;
+    seen.assign((size_t)t.n_nodes, 0);
+    for (int32_t i = 0; i < n_items; ++i) {
+        const int32_t v = node_id[i];
+        if (v < 0 || v >= t.n_nodes) return fail(c, ETS_ERR_INVALID_ARG, "node_id out of range");
+        if (n_new[i] < 0) return fail(c, ETS_ERR_INVALID_ARG, "n_new < 0");
+        if (seen[v]) return fail(c, ETS_ERR_INVALID_ARG, "node named twice in one append");
+        seen[v] = 1;
+        if ((int64_t)len[v] + n_new[i] > t.cap[v]) return fail(c, ETS_ERR_POOL_EXHAUSTED, "append beyond cap_tokens");
+        total += n_new[i];
+        max_new = n_new[i] > max_new ? n_new[i] : max_new;
+    }
+    if (host_src && total > c->lay.max_append_tokens)
+        return fail(c, ETS_ERR_POOL_EXHAUSTED, "more tokens than max_append_tokens in a host append");
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    const int slot = c->desc_next;
+    if (c->desc_used[slot]) ETS_CUDA(c, cudaEventSynchronize(c->desc_ev[slot]));
+    int4* d = c->desc_host[slot];
+    int32_t src = 0;
+    for (int32_t i = 0; i < n_items; ++i) {
+        d[i] = make_int4(node_id[i], len[node_id[i]], n_new[i], src);
+        src += n_new[i];
+    }
+    char* desc_dev = c->ws + c->lay.desc + (size_t)slot * c->lay.desc_slot_bytes;
+    ETS_CUDA(c, cudaMemcpyAsync(desc_dev, d, (size_t)n_items * 16, cudaMemcpyHostToDevice, s));
+    ETS_CUDA(c, cudaEventRecord(c->desc_ev[slot], s));
+    c->desc_used[slot] = true;
+    c->desc_next = (slot + 1) % kDescSlots;
+    const void* ksrc = k_new;
+    const void* vsrc = v_new;
+    if (host_src) {
+        const size_t bytes = (size_t)total * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
+        ETS_CUDA(c, cudaMemcpyAsync(c->ws + c->lay.k_stage, k_new, bytes, cudaMemcpyHostToDevice, s));
+        ETS_CUDA(c, cudaMemcpyAsync(c->ws + c->lay.v_stage, v_new, bytes, cudaMemcpyHostToDevice, s));
+        ksrc = c->ws + c->lay.k_stage;
+        vsrc = c->ws + c->lay.v_stage;
+    }
+    ets::AppendArgs a{};
+    a.desc = reinterpret_cast<const int4*>(desc_dev);
+    a.k_new = reinterpret_cast<const __nv_bfloat16*>(ksrc);
+    a.v_new = reinterpret_cast<const __nv_bfloat16*>(vsrc);
+    a.k_pool = c->k_pool + (size_t)layer * c->layer_pool_bytes;
+    a.v_pool = c->v_pool + (size_t)layer * c->layer_pool_bytes;
+    a.node_page_off = blob_ptr<int32_t>(c, c->bo.node_page_off);
+    a.page_ids = blob_ptr<int32_t>(c, c->bo.page_ids);
+    a.node_len = const_cast<int32_t*>(blob_ptr<int32_t>(c, c->bo.node_len)) + (size_t)layer * c->bo.len_stride;
+    a.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
+    a.n_nodes = t.n_nodes;
+    a.n_pages_total = (int32_t)t.page_ids.size();
+    a.pages_per_layer = c->cfg.pages_per_layer;
+    a.Hkv = c->cfg.num_kv_heads;
+    a.D = c->cfg.head_dim;
+    ets::launch_kv_append(a, n_items, max_new, s);
+    ETS_CUDA(c, cudaGetLastError());
+    for (int32_t i = 0; i < n_items; ++i) len[node_id[i]] += n_new[i];
+    return ETS_OK;
+}
+
+int32_t ets_kv_append(ets_ctx* c, int32_t layer, int32_t n_items, const int32_t* node_id, const int32_t* n_new,
+                      const void* k_new, const void* v_new, void* cuda_stream) {
+    return append_impl(c, layer, n_items, node_id, n_new, k_new, v_new, false, (cudaStream_t)cuda_stream);
+}
+
+int32_t ets_kv_append_host(ets_ctx* c, int32_t layer, int32_t n_items, const int32_t* node_id,
+                           const int32_t* n_new, const void* k_new, const void* v_new, void* cuda_stream) {
+    return append_impl(c, layer, n_items, node_id, n_new, k_new, v_new, true, (cudaStream_t)cuda_stream);
+}
+
+static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse, cudaStream_t s) {
+    const ets::Tree& t = c->tree;
+    if (t.n_leaves == 0) return ETS_OK;
+    ets::DecodeArgs a{};
+    a.units = blob_ptr<int4>(c, c->bo.units);
+    a.items = blob_ptr<ets::DevItem>(c, c->bo.items);
+    a.node_leaves = blob_ptr<int32_t>(c, c->bo.node_leaves);
+    a.node_len = blob_ptr<int32_t>(c, c->bo.node_len) + (size_t)layer * c->bo.len_stride;
+    a.leaf_slot_off = blob_ptr<int32_t>(c, c->bo.leaf_slot_off);
+    a.leaf_slots = blob_ptr<int32_t>(c, c->bo.leaf_slots);
+    a.q = reinterpret_cast<const __nv_bfloat16*>(q);
+    a.out = reinterpret_cast<__nv_bfloat16*>(out);
+    a.lse = lse;
+    a.k_pool = c->k_pool + (size_t)layer * c->layer_pool_bytes;
+    a.v_pool = c->v_pool + (size_t)layer * c->layer_pool_bytes;
+    a.part_ml = reinterpret_cast<float2*>(c->ws + c->lay.part_ml);
+    a.part_o = reinterpret_cast<float*>(c->ws + c->lay.part_o);
+    a.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
+    a.n_items = (int32_t)t.items.size();
+    a.n_leaves = t.n_leaves;
+    a.n_units = (int32_t)(t.unit.size() / 4);
+    a.Hq = c->cfg.num_q_heads;
+    a.Hkv = c->cfg.num_kv_heads;
+    a.G = c->cfg.num_q_heads / c->cfg.num_kv_heads;
+    a.pages_per_layer = c->cfg.pages_per_layer;
+    a.scale_log2 = c->scale_log2;
+
+    cudaEvent_t* ev = nullptr;
+    if (c->opt_timing) {
+        if (c->timed_calls >= kTimingCap) {  // drain so that the pool can be reused
+            double x, y; int64_t n;
+            ets_timing_read(c, &x, &y, &n);
+            c->acc_attn_ms += x; c->acc_merge_ms += y; c->acc_calls += n;
+        }
+        while ((int64_t)c->tev.size() < 3 * (c->timed_calls + 1)) {
+            cudaEvent_t e;
+            ETS_CUDA(c, cudaEventCreate(&e));
+            c->tev.push_back(e);
+        }
+        ev = &c->tev[3 * c->timed_calls];
+        ETS_CUDA(c, cudaEventRecord(ev[0], s));
+    }
+    ets::launch_partial_fma(a, c->cfg.head_dim, s);
+    if (ev) ETS_CUDA(c, cudaEventRecord(ev[1], s));
+    ets::launch_merge(a, c->cfg.head_dim, s);
+    if (ev) {
+        ETS_CUDA(c, cudaEventRecord(ev[2], s));
+        c->timed_calls++;
+    }
+    ETS_CUDA(c, cudaGetLastError());
+    return ETS_OK;
+}
+
+static int32_t decode_check(ets_ctx* c, int32_t layer, const void* q, void* out) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+    if (!c->has_tree) return fail(c, ETS_ERR_STATE, "no tree built");
+    if (layer < 0 || layer >= c->cfg.num_layers) return fail(c, ETS_ERR_INVALID_ARG, "layer out of range");
+    if (c->tree.n_leaves > 0 && (!q || !out)) return fail(c, ETS_ERR_INVALID_ARG, "null q or out");
+    return ETS_OK;
+}
+
+int32_t ets_tree_attn_decode(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse, void* cuda_stream) {
+    if (int32_t rc = decode_check(c, layer, q, out)) return rc;
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, ETS_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    return decode_impl(c, layer, q, out, lse, (cudaStream_t)cuda_stream);
+}
+
+int32_t ets_tree_attn_decode_host(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse,
+                                  void* cuda_stream) {
+    if (int32_t rc = decode_check(c, layer, q, out)) return rc;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    const size_t rows = (size_t)c->tree.n_leaves * c->cfg.num_q_heads;
+    const size_t qbytes = rows * c->cfg.head_dim * 2;
+    if (rows == 0) return ETS_OK;
+    char* qd = c->ws + c->lay.q_stage;
+    char* od = c->ws + c->lay.out_stage;
+    float* ld = reinterpret_cast<float*>(c->ws + c->lay.lse_stage);
+    ETS_CUDA(c, cudaMemcpyAsync(qd, q, qbytes, cudaMemcpyHostToDevice, s));
+    if (int32_t rc = decode_impl(c, layer, qd, od, lse ? ld : nullptr, s)) return rc;
+    ETS_CUDA(c, cudaMemcpyAsync(out, od, qbytes, cudaMemcpyDeviceToHost, s));
+    if (lse) ETS_CUDA(c, cudaMemcpyAsync(lse, ld, rows * 4, cudaMemcpyDeviceToHost, s));
+    return ETS_OK;
+}
+
+int32_t ets_kv_read_debug(ets_ctx* c, int32_t layer, int32_t node, void* k_out, void* v_out, void* cuda_stream) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+    if (!c->has_tree) return fail(c, ETS_ERR_STATE, "no tree built");
+    if (layer < 0 || layer >= c->cfg.num_layers || node < 0 || node >= c->tree.n_nodes)
+        return fail(c, ETS_ERR_INVALID_ARG, "layer or node out of range");
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    const int32_t* pages = blob_ptr<int32_t>(c, c->bo.page_ids) + c->tree.node_page_off[node];
+    ets::launch_kv_read(c->k_pool + (size_t)layer * c->layer_pool_bytes,
+                        c->v_pool + (size_t)layer * c->layer_pool_bytes, pages, c->tree.len[layer][node],
+                        c->cfg.num_kv_heads, c->cfg.head_dim, (__nv_bfloat16*)k_out, (__nv_bfloat16*)v_out,
+                        (cudaStream_t)cuda_stream);
+    ETS_CUDA(c, cudaGetLastError());
+    return ETS_OK;
+}
+
+int32_t ets_timing_read(ets_ctx* c, double* attn_ms, double* merge_ms, int64_t* n_calls) {
+    if (!c || !attn_ms || !merge_ms || !n_calls) return ETS_ERR_INVALID_ARG;
+    if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+    double a = c->acc_attn_ms, m = c->acc_merge_ms;
+    int64_t n = c->acc_calls;
+    c->acc_attn_ms = c->acc_merge_ms = 0;
+    c->acc_calls = 0;
+    for (int64_t i = 0; i < c->timed_calls; ++i) {
+        cudaEvent_t* ev = &c->tev[3 * i];
+        ETS_CUDA(c, cudaEventSynchronize(ev[2]));
+        float x = 0, y = 0;
+        ETS_CUDA(c, cudaEventElapsedTime(&x, ev[0], ev[1]));
+        ETS_CUDA(c, cudaEventElapsedTime(&y, ev[1], ev[2]));
+        a += x; m += y; ++n;
+    }
+    c->timed_calls = 0;
+    *attn_ms = a; *merge_ms = m; *n_calls = n;
+    return ETS_OK;
+}
+
+int32_t ets_poll_status(ets_ctx* c, void* cuda_stream) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    ETS_CUDA(c, cudaMemcpyAsync(c->status_host, c->ws + c->lay.status, 4, cudaMemcpyDeviceToHost, s));
+    ETS_CUDA(c, cudaMemsetAsync(c->ws + c->lay.status, 0, 4, s));
+    ETS_CUDA(c, cudaStreamSynchronize(s));
+    const int32_t v = *c->status_host;
+    if (v == 0) return ETS_OK;
+    if (v == -7) return fail(c, ETS_ERR_DEVICE_TIMEOUT, "a device-side wait ran out");
+    return fail(c, ETS_ERR_INVALID_ARG, "a kernel skipped an out-of-range table entry");
+}
+
+}  // extern "C"

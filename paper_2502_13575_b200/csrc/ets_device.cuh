@@ -1,0 +1,76 @@
+// Device-side declarations shared by the kernels and the API file.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace ets {
+
+// In-page layout of one (page, kv head) tile: 16 tokens x D bf16, stored as the shared-memory
+// image that both the tensor-core paths and the scalar path consume, so that one linear bulk
+// copy of the tile needs no rearrangement:
+//   byte(t, e) = (t/8) * (D/64)*1024          8-token group
+//              + (e/64) * 1024                 64-element half of the head dimension
+//              + (t%8) * 128                   row inside the 8x128B swizzle atom
+//              + (((e%64)/8) ^ (t%8)) * 16     16-byte chunk, XOR-swizzled by the row
+//              + (e%8) * 2
+// i.e. rows of 128 bytes in 1024-byte atoms with the 128-byte swizzle pattern.
+constexpr int kPageTokens = 16;
+
+__host__ __device__ inline size_t tile_bytes(int D) { return (size_t)kPageTokens * D * 2; }
+
+__host__ __device__ inline uint32_t tile_offset(int D, int t, int e) {
+    uint32_t r = (uint32_t)t & 7u;
+    return (uint32_t)(t >> 3) * (uint32_t)(D / 64) * 1024u + (uint32_t)(e >> 6) * 1024u + r * 128u +
+           ((((uint32_t)(e & 63) >> 3) ^ r) << 4) + (uint32_t)(e & 7) * 2u;
+}
+
+struct DevItem {
+    int32_t unit_begin, unit_count, kv_head, leaf_list_begin;
+    int32_t n_leaves_tile, slot_first, chunk, reserved;
+};
+
+// Everything a decode launch needs; passed by value.
+struct DecodeArgs {
+    const int4* units;
+    const DevItem* items;
+    const int32_t* node_leaves;
+    const int32_t* node_len;       // this layer's lengths
+    const int32_t* leaf_slot_off;
+    const int32_t* leaf_slots;
+    const __nv_bfloat16* q;
+    __nv_bfloat16* out;
+    float* lse;
+    const char* k_pool;            // this layer's pools
+    const char* v_pool;
+    float2* part_ml;               // [slot][Hq]  (m in log2 units, l)
+    float* part_o;                 // [slot][Hq][D]
+    int32_t* status;
+    int32_t n_items, n_leaves, n_units;
+    int32_t Hq, Hkv, G;
+    int64_t pages_per_layer;
+    float scale_log2;              // sm_scale * log2(e)
+};
+
+struct AppendArgs {
+    const int4* desc;              // per item: node, start, n_new, src token offset
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    char* k_pool;
+    char* v_pool;
+    const int32_t* node_page_off;
+    const int32_t* page_ids;
+    int32_t* node_len;
+    int32_t* status;
+    int32_t n_nodes, n_pages_total;
+    int64_t pages_per_layer;
+    int32_t Hkv, D;
+};
+
+void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_t s);
+void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* page_ids_of_node, int n_tokens,
+                    int Hkv, int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s);
+void launch_partial_fma(const DecodeArgs& a, int D, cudaStream_t s);
+void launch_merge(const DecodeArgs& a, int D, cudaStream_t s);
+
+}  // namespace ets

@@ -1,0 +1,63 @@
+// Host-side tree flattener: page tables, query groups, leaf paths and the work
+// decomposition for the attention kernels.  Pure C++ (no CUDA), so it can be exercised
+// on a machine without a GPU.
+//
+// Semantics follow Section 4.1 and Appendix B of the paper: a node lies on a leaf's
+// path iff the leaf descends from it, and all leaves through a node share its KV.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+namespace ets {
+
+struct FlattenParams {
+    int32_t num_kv_heads = 1;
+    int32_t gqa = 1;            // query heads per kv head
+    int32_t page_size = 16;
+    int32_t num_layers = 1;
+    int32_t max_nodes = 0;
+    int32_t max_leaves = 0;
+    int64_t max_path_entries = 0;
+    int64_t max_partial_slots = 0;
+    int64_t max_items = 0;
+    int32_t chunk_pages = 0;    // 0 = automatic
+    int32_t rows_per_item = 16; // query rows (leaves * gqa) one work item covers
+    int32_t n_workers = 148;    // CTAs the attention kernel keeps resident (for chunk sizing)
+};
+
+// One work item, as uploaded to the device (8 x int32).
+struct Item {
+    int32_t unit_begin, unit_count, kv_head, leaf_list_begin;
+    int32_t n_leaves_tile, slot_first, chunk, reserved;
+};
+
+struct Tree {
+    int32_t n_nodes = 0, n_leaves = 0;
+    std::vector<int32_t> parent, cap, leaf_node, depth;
+    std::vector<int32_t> node_page_off, page_ids;
+    std::vector<int32_t> node_leaf_off, node_leaves;
+    std::vector<int32_t> leaf_path_off, leaf_path, leaf_path_pos;
+    std::vector<std::vector<int32_t>> len;  // [layer][node]
+    std::vector<int32_t> free_heap;         // min-heap of free page ids (std::greater)
+    // work decomposition
+    std::vector<int32_t> unit;              // 4 per unit: page, node, tok0, 0
+    std::vector<Item> items;
+    std::vector<int32_t> leaf_slot_off, leaf_slots;
+    int64_t n_segments = 0, n_chunks = 0, n_partial_slots = 0;
+    int32_t chunk_pages_used = 0;
+};
+
+// Status codes mirror ets.h (kept numerically identical by a static_assert in the API file).
+enum : int32_t { F_OK = 0, F_INVALID = -1, F_BAD_TREE = -2, F_EXHAUSTED = -3 };
+
+// Fresh state: all pages free, no nodes.
+void tree_init(Tree& t, const FlattenParams& p, int64_t pages_per_layer);
+
+// Builds `next` from `prev` (which is left untouched).  On failure `next` is unspecified and
+// `err` holds a message.
+int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, const int32_t* parent,
+                   const int32_t* cap_tokens, const int32_t* keep_pages_of, int32_t n_leaves,
+                   const int32_t* leaf_node, Tree& next, std::string& err);
+
+}  // namespace ets

@@ -1,0 +1,265 @@
+// KV append / read-back, the scalar-FMA node-partial attention kernel and the
+// log-sum-exp merge kernel.
+#include "ets_device.cuh"
+
+namespace ets {
+
+// ------------------------------------------------------------------------------------
+// KV append: scatter new token rows [token, kv head, D] into (page, slot) tiles.
+// One block handles 8 tokens of one item; a thread moves 16-byte chunks.
+// ------------------------------------------------------------------------------------
+constexpr int kAppendTokPerBlock = 8;
+
+__global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
+    const int4 d = a.desc[blockIdx.y];
+    const int node = d.x, start = d.y, n_new = d.z, src_off = d.w;
+    const int t0 = blockIdx.x * kAppendTokPerBlock;
+    if (t0 >= n_new) return;
+    if (node < 0 || node >= a.n_nodes) {
+        if (threadIdx.x == 0) atomicExch(a.status, -1);
+        return;
+    }
+    const int chunks_per_head = a.D / 8;
+    const int chunks_per_tok = a.Hkv * chunks_per_head;
+    const int n_tok = min(kAppendTokPerBlock, n_new - t0);
+    const size_t tb = tile_bytes(a.D);
+    const int page_base = a.node_page_off[node];
+    const int page_cnt = a.node_page_off[node + 1] - page_base;
+    for (int i = threadIdx.x; i < n_tok * chunks_per_tok; i += blockDim.x) {
+        const int t = t0 + i / chunks_per_tok;
+        const int ci = i % chunks_per_tok;
+        const int h = ci / chunks_per_head;
+        const int c = ci % chunks_per_head;
+        const int pos = start + t;
+        const int pslot = pos / kPageTokens;
+        if (pslot >= page_cnt) {  // beyond the node's reserved pages: refuse, flag, keep going
+            atomicExch(a.status, -1);
+            continue;
+        }
+        const int page = a.page_ids[page_base + pslot];
+        if (page < 0 || (int64_t)page >= a.pages_per_layer) {
+            atomicExch(a.status, -1);
+            continue;
+        }
+        const size_t src = ((size_t)(src_off + t) * a.Hkv + h) * a.D + (size_t)c * 8;
+        const size_t dst = ((size_t)page * a.Hkv + h) * tb + tile_offset(a.D, pos % kPageTokens, c * 8);
+        *reinterpret_cast<uint4*>(a.k_pool + dst) = *reinterpret_cast<const uint4*>(a.k_new + src);
+        *reinterpret_cast<uint4*>(a.v_pool + dst) = *reinterpret_cast<const uint4*>(a.v_new + src);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) a.node_len[node] = start + n_new;
+}
+
+void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_t s) {
+    if (n_items <= 0 || max_new <= 0) return;
+    dim3 grid((max_new + kAppendTokPerBlock - 1) / kAppendTokPerBlock, n_items);
+    kv_append_kernel<<<grid, 256, 0, s>>>(a);
+}
+
+// ------------------------------------------------------------------------------------
+// Read one node's rows back in token order (debug / tests).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) kv_read_kernel(const char* k_pool, const char* v_pool,
+                                                      const int32_t* pages, int n_tokens, int Hkv, int D,
+                                                      __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
+    const int chunks_per_head = D / 8;
+    const int chunks_per_tok = Hkv * chunks_per_head;
+    const size_t tb = tile_bytes(D);
+    const int64_t total = (int64_t)n_tokens * chunks_per_tok;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int t = (int)(i / chunks_per_tok);
+        const int ci = (int)(i % chunks_per_tok);
+        const int h = ci / chunks_per_head;
+        const int c = ci % chunks_per_head;
+        const int page = pages[t / kPageTokens];
+        const size_t src = ((size_t)page * Hkv + h) * tb + tile_offset(D, t % kPageTokens, c * 8);
+        const size_t dst = ((size_t)t * Hkv + h) * D + (size_t)c * 8;
+        if (k_out) *reinterpret_cast<uint4*>(k_out + dst) = *reinterpret_cast<const uint4*>(k_pool + src);
+        if (v_out) *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(v_pool + src);
+    }
+}
+
+void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* pages, int n_tokens, int Hkv,
+                    int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s) {
+    if (n_tokens <= 0) return;
+    int64_t total = (int64_t)n_tokens * Hkv * (D / 8);
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 4096) blocks = 4096;
+    kv_read_kernel<<<blocks, 256, 0, s>>>(k_pool, v_pool, pages, n_tokens, Hkv, D, k_out, v_out);
+}
+
+// ------------------------------------------------------------------------------------
+// Scalar-FMA node-partial attention.  One block per work item, 4 warps; warp w takes page
+// slots w, w+4, ... of the chunk.  A lane owns D/32 consecutive features of every row; the
+// q.k dot products are finished with warp shuffles.  Scores are kept in log2 units.
+// Generic fallback: any group width, any supported head_dim, no tensor cores.
+// ------------------------------------------------------------------------------------
+constexpr int kFmaWarps = 4;
+constexpr int kMaxRows = 16;
+
+template <int D>
+__global__ void __launch_bounds__(kFmaWarps * 32) attn_partial_fma_kernel(DecodeArgs a) {
+    constexpr int EPL = D / 32;  // features per lane
+    __shared__ float sm_m[kFmaWarps][kMaxRows];
+    __shared__ float sm_l[kFmaWarps][kMaxRows];
+    __shared__ float sm_o[kFmaWarps][kMaxRows][D];
+
+    const DevItem it = a.items[blockIdx.x];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = a.G;
+    const int rows = it.n_leaves_tile * G;
+    const int h = it.kv_head;
+    const int e0 = lane * EPL;
+
+    float q[kMaxRows][EPL];
+    float o[kMaxRows][EPL];
+    float m[kMaxRows], l[kMaxRows];
+#pragma unroll
+    for (int r = 0; r < kMaxRows; ++r) {
+        m[r] = -INFINITY;
+        l[r] = 0.f;
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) { q[r][j] = 0.f; o[r][j] = 0.f; }
+        if (r < rows) {
+            const int leaf = a.node_leaves[it.leaf_list_begin + r / G];
+            const __nv_bfloat16* qp = a.q + ((size_t)leaf * a.Hq + h * G + r % G) * D + e0;
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) q[r][j] = __bfloat162float(qp[j]);
+        }
+    }
+
+    const size_t tb = tile_bytes(D);
+    for (int u = warp; u < it.unit_count; u += kFmaWarps) {
+        const int4 un = a.units[it.unit_begin + u];
+        if (un.x < 0 || (int64_t)un.x >= a.pages_per_layer) {
+            if (lane == 0) atomicExch(a.status, -1);
+            continue;
+        }
+        int valid = a.node_len[un.y] - un.z;
+        valid = valid < 0 ? 0 : (valid > kPageTokens ? kPageTokens : valid);
+        const char* kt = a.k_pool + ((size_t)un.x * a.Hkv + h) * tb;
+        const char* vt = a.v_pool + ((size_t)un.x * a.Hkv + h) * tb;
+        for (int t = 0; t < valid; ++t) {
+            const uint32_t off = tile_offset(D, t, e0);
+            float kf[EPL], vf[EPL];
+            const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(kt + off);
+            const __nv_bfloat16* vp = reinterpret_cast<const __nv_bfloat16*>(vt + off);
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) { kf[j] = __bfloat162float(kp[j]); vf[j] = __bfloat162float(vp[j]); }
+#pragma unroll
+            for (int r = 0; r < kMaxRows; ++r) {
+                if (r < rows) {
+                    float s = 0.f;
+#pragma unroll
+                    for (int j = 0; j < EPL; ++j) s = fmaf(q[r][j], kf[j], s);
+#pragma unroll
+                    for (int x = 16; x > 0; x >>= 1) s += __shfl_xor_sync(0xffffffffu, s, x);
+                    s *= a.scale_log2;
+                    const float mn = fmaxf(m[r], s);
+                    const float corr = exp2f(m[r] - mn);
+                    const float p = exp2f(s - mn);
+                    l[r] = l[r] * corr + p;
+#pragma unroll
+                    for (int j = 0; j < EPL; ++j) o[r][j] = o[r][j] * corr + p * vf[j];
+                    m[r] = mn;
+                }
+            }
+        }
+    }
+
+    // combine the four warps' partials
+#pragma unroll
+    for (int r = 0; r < kMaxRows; ++r) {
+        if (r < rows) {
+            if (lane == 0) { sm_m[warp][r] = m[r]; sm_l[warp][r] = l[r]; }
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) sm_o[warp][r][e0 + j] = o[r][j];
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < rows * D; i += blockDim.x) {
+        const int r = i / D, e = i % D;
+        float ms = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kFmaWarps; ++w) ms = fmaxf(ms, sm_m[w][r]);
+        float acc = 0.f, ls = 0.f;
+#pragma unroll
+        for (int w = 0; w < kFmaWarps; ++w) {
+            const float wgt = sm_l[w][r] > 0.f ? exp2f(sm_m[w][r] - ms) : 0.f;
+            acc += wgt * sm_o[w][r][e];
+            ls += wgt * sm_l[w][r];
+        }
+        const int slot = it.slot_first + r / G;
+        const size_t row = (size_t)slot * a.Hq + h * G + r % G;
+        a.part_o[row * D + e] = acc;
+        if (e == 0) a.part_ml[row] = make_float2(ms, ls);
+    }
+}
+
+void launch_partial_fma(const DecodeArgs& a, int D, cudaStream_t s) {
+    if (a.n_items <= 0) return;
+    if (D == 128) attn_partial_fma_kernel<128><<<a.n_items, kFmaWarps * 32, 0, s>>>(a);
+    else attn_partial_fma_kernel<64><<<a.n_items, kFmaWarps * 32, 0, s>>>(a);
+}
+
+// ------------------------------------------------------------------------------------
+// Log-sum-exp merge along each leaf's path.  One warp per (leaf, query head); a lane owns
+// D/32 consecutive features.  With partials (m_j, l_j, o_j) in log2 units:
+//   m* = max_j m_j, l* = sum_j l_j 2^(m_j-m*), out = sum_j o_j 2^(m_j-m*) / l*,
+//   lse = (m* + log2 l*) ln 2.  Empty partials (l_j = 0) are skipped.
+// ------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(128) lse_merge_kernel(DecodeArgs a) {
+    constexpr int EPL = D / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * 4 + warp;
+    if (row >= (int64_t)a.n_leaves * a.Hq) return;
+    const int leaf = (int)(row / a.Hq), head = (int)(row % a.Hq);
+    const int s0 = a.leaf_slot_off[leaf], s1 = a.leaf_slot_off[leaf + 1];
+
+    float ms = -INFINITY;
+    for (int j = s0 + lane; j < s1; j += 32) {
+        const float2 ml = a.part_ml[(size_t)a.leaf_slots[j] * a.Hq + head];
+        if (ml.y > 0.f) ms = fmaxf(ms, ml.x);
+    }
+#pragma unroll
+    for (int x = 16; x > 0; x >>= 1) ms = fmaxf(ms, __shfl_xor_sync(0xffffffffu, ms, x));
+
+    float acc[EPL];
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) acc[j] = 0.f;
+    float ls = 0.f;
+    for (int j = s0; j < s1; ++j) {
+        const size_t prow = (size_t)a.leaf_slots[j] * a.Hq + head;
+        const float2 ml = a.part_ml[prow];
+        if (!(ml.y > 0.f)) continue;
+        const float w = exp2f(ml.x - ms);
+        ls += w * ml.y;
+        const float* po = a.part_o + prow * D + lane * EPL;
+        if constexpr (EPL == 4) {
+            const float4 v = *reinterpret_cast<const float4*>(po);
+            acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
+        } else {
+            const float2 v = *reinterpret_cast<const float2*>(po);
+            acc[0] += w * v.x; acc[1] += w * v.y;
+        }
+    }
+    const float inv = ls > 0.f ? 1.f / ls : 0.f;
+    __nv_bfloat16* op = a.out + (size_t)row * D + lane * EPL;
+#pragma unroll
+    for (int j = 0; j < EPL; j += 2) {
+        __nv_bfloat162 pk = __floats2bfloat162_rn(acc[j] * inv, acc[j + 1] * inv);
+        *reinterpret_cast<__nv_bfloat162*>(op + j) = pk;
+    }
+    if (a.lse && lane == 0) a.lse[row] = ls > 0.f ? (ms + log2f(ls)) * 0.6931471805599453f : -INFINITY;
+}
+
+void launch_merge(const DecodeArgs& a, int D, cudaStream_t s) {
+    const int64_t rows = (int64_t)a.n_leaves * a.Hq;
+    if (rows <= 0) return;
+    const int blocks = (int)((rows + 3) / 4);
+    if (D == 128) lse_merge_kernel<128><<<blocks, 128, 0, s>>>(a);
+    else lse_merge_kernel<64><<<blocks, 128, 0, s>>>(a);
+}
+
+}  // namespace ets

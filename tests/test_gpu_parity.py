@@ -1,0 +1,234 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded inputs.  Bar: |gpu - oracle| <= 2e-3 + 1e-2 |oracle| element-wise on the bf16 output
+(bf16 inputs, fp32 accumulation); tables and KV bytes bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2502_13575_b200 as ets
+from paper_2502_13575_b200.runner import context_for_tree
+from oracle.flatten import ReferenceFlattener
+from workloads import Geometry, Tree, make_workload, random_small_tree, node_kv_bits
+from _harness import run_and_check, node_values, fill_layer, bits_to_dev, dev_to_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def _read_node(ctx, layer, node, n_tok, geom):
+    k = torch.empty((n_tok, geom.num_kv_heads, geom.head_dim), dtype=torch.bfloat16, device="cuda")
+    v = torch.empty_like(k)
+    ctx.kv_read_debug(layer, node, k, v)
+    torch.cuda.synchronize()
+    return dev_to_bits(k), dev_to_bits(v)
+
+
+def test_kv_append_round_trip_is_bit_exact():
+    wl = make_workload("cfg2")
+    g, tree = wl.geometry, wl.tree
+    ctx = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, tree.parent, tree.tokens, tree.leaf_node,
+                           num_layers=2)
+    ctx.tree_build(tree.parent, tree.tokens, tree.leaf_node)
+    ref = ReferenceFlattener(16, ctx.cfg.pages_per_layer).build(tree.parent, tree.tokens, tree.leaf_node)
+    got = ctx.tree_export()
+    for key, val in ref.items():
+        assert np.array_equal(got[key], val), key
+    for layer in (0, 1):
+        ks, vs = node_values(tree, g, wl.value_seed, layer)
+        # two-stage fill: first 5 tokens of every node, then the rest (ragged page boundaries)
+        first = [min(5, int(t)) for t in tree.tokens]
+        fill_layer(ctx, layer, [k[:f] for k, f in zip(ks, first)], [v[:f] for v, f in zip(vs, first)])
+        fill_layer(ctx, layer, [k[f:] for k, f in zip(ks, first)], [v[f:] for v, f in zip(vs, first)])
+        assert np.array_equal(ctx.get_node_len(layer), tree.tokens)
+        for node in (0, 1, tree.n_nodes // 2, tree.n_nodes - 1):
+            kb, vb = _read_node(ctx, layer, node, int(tree.tokens[node]), g)
+            assert np.array_equal(kb, ks[node]) and np.array_equal(vb, vs[node])
+    ctx.poll_status()
+    st = ctx.get_stats()
+    assert st["unique_tokens"] == int(tree.tokens.sum())
+    # appending beyond the capacity is refused and changes nothing
+    k1 = bits_to_dev(ks[0][:1])
+    with pytest.raises(ets.EtsError) as e:
+        ctx.kv_append(0, [0], [1], k1, k1)
+    assert e.value.code == ets.ETS_ERR_POOL_EXHAUSTED
+    assert np.array_equal(ctx.get_node_len(0), tree.tokens)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2"])
+@pytest.mark.parametrize("host_api", [False, True])
+def test_small_configs_full_comparison(name, host_api):
+    wl = make_workload(name)
+    run_and_check(wl.tree, wl.geometry, wl.value_seed, host_api=host_api)
+
+
+@pytest.mark.parametrize("name", ["cfg3_diverse", "cfg3_ets", "cfg5a", "cfg5b", "cfg5c"])
+def test_wide_configs_sampled_leaves(name):
+    wl = make_workload(name)
+    L = wl.tree.n_leaves
+    rng = np.random.default_rng(5)
+    subset = sorted(set([0, L - 1] + [int(x) for x in rng.integers(0, L, size=6)]))
+    run_and_check(wl.tree, wl.geometry, wl.value_seed, leaves_subset=subset)
+
+
+@pytest.mark.parametrize("qscale", [4.0, 8.0])
+def test_peaked_softmax(qscale):
+    wl = make_workload("cfg2")
+    run_and_check(wl.tree, wl.geometry, wl.value_seed, qscale=qscale)
+
+
+@pytest.mark.parametrize("chunk_pages", [1, 3])
+def test_many_small_chunks(chunk_pages):
+    wl = make_workload("cfg1")
+    run_and_check(wl.tree, wl.geometry, wl.value_seed, chunk_pages=chunk_pages)
+
+
+def test_large_common_score_offset():
+    # every key shares a component aligned with q: scores near +60 before the max shift
+    g = Geometry(8, 2, 128)
+    tree = Tree(np.array([-1, 0, 0], np.int32), np.array([40, 33, 7], np.int32), np.array([1, 2], np.int32))
+    from workloads import f32_to_bf16_bits, bf16_bits_to_f32
+    from oracle.tree_attention import tree_decode_attention
+    from _harness import check_close
+    rng = np.random.default_rng(9)
+    u = rng.standard_normal(128).astype(np.float32)
+    u /= np.linalg.norm(u)
+    ks, vs = [], []
+    for n in range(3):
+        t = int(tree.tokens[n])
+        k = rng.standard_normal((t, 2, 128)).astype(np.float32) + 26.0 * u
+        ks.append(f32_to_bf16_bits(k))
+        vs.append(f32_to_bf16_bits(rng.standard_normal((t, 2, 128)).astype(np.float32)))
+    qb = f32_to_bf16_bits((rng.standard_normal((2, 8, 128)).astype(np.float32) + 26.0 * u))
+    ctx = context_for_tree(8, 2, 128, tree.parent, tree.tokens, tree.leaf_node)
+    ctx.tree_build(tree.parent, tree.tokens, tree.leaf_node)
+    fill_layer(ctx, 0, ks, vs)
+    q = bits_to_dev(qb)
+    out = torch.empty_like(q)
+    ctx.tree_attn_decode(0, q, out, None)
+    torch.cuda.synchronize()
+    ref, lse = tree_decode_attention(tree.parent, tree.tokens, tree.leaf_node, ks, vs, qb, 8, 2)
+    assert lse.min() > 40.0
+    check_close(dev_to_bits(out), ref)
+
+
+def test_random_small_trees_with_edge_cases():
+    """Forests, repeated leaves, leaves on internal nodes, zero-token nodes, ragged lengths
+    shorter than the reserved capacity, GQA 1 / 4 / 8, both head sizes."""
+    rng = np.random.default_rng(77)
+    done = 0
+    while done < 24:
+        tree = random_small_tree(rng, max_nodes=10, max_tokens=70, max_leaves=7)
+        # lengths below capacity
+        lengths = np.array([int(rng.integers(0, t + 1)) for t in tree.tokens], np.int32)
+        # every leaf needs at least one token on its path
+        ok = True
+        for leaf in tree.leaf_node:
+            s, v = 0, int(leaf)
+            while v >= 0:
+                s += int(lengths[v])
+                v = int(tree.parent[v])
+            ok &= s > 0
+        if not ok:
+            continue
+        hkv = int(rng.choice([1, 2]))
+        gqa = int(rng.choice([1, 4, 8]))
+        d = int(rng.choice([64, 128]))
+        geom = Geometry(hkv * gqa, hkv, d)
+        run_and_check(tree, geom, 1000 + done, cap=tree.tokens, lengths=lengths)
+        done += 1
+
+
+def test_single_token_tree_returns_v():
+    g = Geometry(4, 2, 64)
+    tree = Tree(np.array([-1], np.int32), np.array([1], np.int32), np.array([0], np.int32))
+    ctx = run_and_check(tree, g, 5)
+    k, v = node_kv_bits(5, 0, 1, 2, 64)
+    q = bits_to_dev(np.zeros((1, 4, 64), np.uint16))
+    out = torch.empty_like(q)
+    ctx.tree_attn_decode(0, q, out, None)
+    torch.cuda.synchronize()
+    ob = dev_to_bits(out)
+    for a in range(4):
+        assert np.array_equal(ob[0, a], v[0, a // 2])  # exactly V, also in bf16
+
+
+def test_empty_path_leaf_and_empty_tree():
+    g = Geometry(4, 1, 64)
+    # leaf 1 sits under an empty root with an empty node: zeros and lse = -inf, no NaN
+    tree = Tree(np.array([-1, 0, 0], np.int32), np.array([0, 9, 0], np.int32), np.array([1, 2], np.int32))
+    ctx = context_for_tree(4, 1, 64, tree.parent, [0, 9, 4], tree.leaf_node)
+    ctx.tree_build(tree.parent, [0, 9, 4], tree.leaf_node)
+    ks, vs = node_values(tree, g, 3, 0)
+    fill_layer(ctx, 0, ks, vs)
+    q = bits_to_dev(np.full((2, 4, 64), 0x3F80, np.uint16))
+    out = torch.full_like(q, 7.0)
+    lse = torch.zeros((2, 4), dtype=torch.float32, device="cuda")
+    ctx.tree_attn_decode(0, q, out, lse)
+    torch.cuda.synchronize()
+    assert torch.all(out[1] == 0) and torch.all(torch.isinf(lse[1])) and torch.all(lse[1] < 0)
+    assert torch.isfinite(out[0].float()).all() and torch.isfinite(lse[0]).all()
+    # empty tree: decode is a no-op
+    ctx.tree_build([], [], [])
+    ctx.tree_attn_decode(0, q, out, None)
+    ctx.poll_status()
+
+
+def test_rebuild_keeps_pages_and_contents():
+    """A search step: leaves grow children, one branch is pruned; kept nodes keep their KV."""
+    g = Geometry(8, 2, 128)
+    t0 = Tree(np.array([-1, 0, 0], np.int32), np.array([40, 20, 30], np.int32), np.array([1, 2], np.int32))
+    ctx = run_and_check(t0, g, 11)
+    # new tree: old 0 -> 0, old 2 -> 1 (old 1 pruned), two new children of node 1
+    t1 = Tree(np.array([-1, 0, 1, 1], np.int32), np.array([40, 30, 12, 25], np.int32), np.array([2, 3], np.int32))
+    ctx.tree_build(t1.parent, t1.tokens, t1.leaf_node, keep_pages_of=[0, 2, -1, -1])
+    assert ctx.get_node_len(0).tolist() == [40, 30, 0, 0]
+    ks0, vs0 = node_values(t0, g, 11, 0)
+    ks1, vs1 = node_values(t1, g, 12, 0)
+    ks = [ks0[0], ks0[2], ks1[2], ks1[3]]
+    vs = [vs0[0], vs0[2], vs1[2], vs1[3]]
+    fill_layer(ctx, 0, ks, vs, nodes=[2, 3])
+    from workloads import query_bits
+    from oracle.tree_attention import tree_decode_attention
+    from _harness import check_close
+    qb = query_bits(12, 0, 2, 8, 128)
+    q = bits_to_dev(qb)
+    out = torch.empty_like(q)
+    ctx.tree_attn_decode(0, q, out, None)
+    torch.cuda.synchronize()
+    ref, _ = tree_decode_attention(t1.parent, t1.tokens, t1.leaf_node, ks, vs, qb, 8, 2)
+    check_close(dev_to_bits(out), ref)
+    ctx.poll_status()
+
+
+def test_decode_loop_appends_one_token_per_leaf():
+    """Per-token decode: append the new token's K/V to each leaf node, then attend; lengths grow
+    without a rebuild."""
+    g = Geometry(8, 2, 128)
+    tree = make_workload("cfg1").tree
+    cap = tree.tokens.copy()
+    leaf_nodes = tree.leaf_node
+    cap[leaf_nodes] += 5
+    lengths = tree.tokens.copy()
+    ctx = context_for_tree(8, 2, 128, tree.parent, cap, tree.leaf_node)
+    ctx.tree_build(tree.parent, cap, tree.leaf_node)
+    full_k, full_v = [], []
+    for n in range(tree.n_nodes):
+        k, v = node_kv_bits(21, n, int(cap[n]), 2, 128)
+        full_k.append(k)
+        full_v.append(v)
+    fill_layer(ctx, 0, [k[:t] for k, t in zip(full_k, lengths)], [v[:t] for v, t in zip(full_v, lengths)])
+    from workloads import query_bits
+    from oracle.tree_attention import tree_decode_attention
+    from _harness import check_close
+    for step in range(5):
+        newk = np.stack([full_k[n][lengths[n]] for n in leaf_nodes])
+        newv = np.stack([full_v[n][lengths[n]] for n in leaf_nodes])
+        ctx.kv_append(0, leaf_nodes, [1] * len(leaf_nodes), bits_to_dev(newk), bits_to_dev(newv))
+        lengths[leaf_nodes] += 1
+        qb = query_bits(21, step, tree.n_leaves, 8, 128)
+        q = bits_to_dev(qb)
+        out = torch.empty_like(q)
+        ctx.tree_attn_decode(0, q, out, None)
+        torch.cuda.synchronize()
+        ref, _ = tree_decode_attention(tree.parent, lengths, tree.leaf_node, full_k, full_v, qb, 8, 2)
+        check_close(dev_to_bits(out), ref, f"step {step}")
+    ctx.poll_status()

@@ -1,0 +1,223 @@
+"""Host logic of the library, no GPU needed: the shared library loads and exports every symbol
+the header declares; its tables match the reference flattener bit for bit; its private work
+decomposition covers every (page, kv head, leaf) exactly once."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2502_13575_b200 as ets
+from oracle.flatten import ReferenceFlattener, BadTree, PoolExhausted
+from workloads import random_small_tree, make_workload, tree_stats, CONFIG_NAMES
+from _golden import read_golden
+
+TABLE_KEYS = ("node_page_off", "page_ids", "node_leaf_off", "node_leaves", "leaf_path_off",
+              "leaf_path", "leaf_path_pos", "node_depth", "node_len")
+
+
+def host_ctx(hq=4, hkv=1, d=64, page_size=16, pages=4096, max_nodes=4096, max_leaves=512,
+             max_path_tokens=8192, max_path_entries=8192, layers=1):
+    cfg = ets.make_config(hq, hkv, d, num_layers=layers, max_nodes=max_nodes, max_leaves=max_leaves,
+                          max_path_tokens=max_path_tokens, max_path_entries=max_path_entries,
+                          pages_per_layer=pages, page_size=page_size, device=-1)
+    return ets.EtsContext(cfg)
+
+
+def test_header_symbols_are_exported(repo_root):
+    text = open(os.path.join(repo_root, "include", "ets.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(ets_[a-z_]+)\s*\(", text))
+    assert {"ets_tree_build", "ets_kv_append", "ets_tree_attn_decode"} <= declared
+    for name in declared:
+        assert hasattr(ets.lib, name), f"{name} declared in ets.h but not exported"
+    assert ets.ets_version().startswith("ets-b200")
+
+
+def test_config_struct_layout_matches_header():
+    # a mis-declared ctypes struct would scramble these values on the C side
+    cfg = ets.make_config(32, 8, 128, max_nodes=10, max_leaves=4, max_path_tokens=64, max_path_entries=40,
+                          pages_per_layer=7, device=-1)
+    k, v, w = ets.ets_pool_bytes(cfg)
+    assert k == v == 7 * 8 * 16 * 128 * 2
+    bad = ets.make_config(32, 8, 96, max_nodes=10, max_leaves=4, max_path_tokens=64, max_path_entries=40,
+                          pages_per_layer=7, device=-1)
+    with pytest.raises(ets.EtsError) as e:
+        ets.ets_pool_bytes(bad)
+    assert e.value.code == ets.ETS_ERR_UNSUPPORTED
+
+
+def test_hand_worked_tree_matches():
+    g = read_golden("flatten_small_tree.txt")
+    ctx = host_ctx(page_size=g["page_size"][0], pages=g["pages_per_layer"][0])
+    ctx.tree_build(g["parent"], g["cap_tokens"], g["leaf_node"])
+    t = ctx.tree_export()
+    for key in TABLE_KEYS[:-1]:
+        assert t[key].tolist() == g[key], key
+
+
+def _assert_same_tables(ctx, ref_tables):
+    got = ctx.tree_export()
+    for key in TABLE_KEYS:
+        assert got[key].dtype == np.int32
+        assert np.array_equal(got[key], ref_tables[key]), key
+
+
+@pytest.mark.parametrize("name", CONFIG_NAMES)
+def test_tables_bit_exact_on_configs(name):
+    wl = make_workload(name)
+    g = wl.geometry
+    ctx = host_ctx(g.num_q_heads, g.num_kv_heads, g.head_dim, pages=1 << 15, max_path_entries=1 << 14)
+    ref = ReferenceFlattener(16, 1 << 15)
+    ctx.tree_build(wl.tree.parent, wl.tree.tokens, wl.tree.leaf_node)
+    _assert_same_tables(ctx, ref.build(wl.tree.parent, wl.tree.tokens, wl.tree.leaf_node))
+    st = ctx.get_stats()
+    assert st["n_nodes"] == wl.tree.n_nodes and st["n_leaves"] == wl.tree.n_leaves
+    assert st["unique_tokens"] == 0  # nothing appended yet
+
+
+def test_tables_bit_exact_on_random_trees_and_rebuilds():
+    rng = np.random.default_rng(31)
+    for trial in range(300):
+        page = int(rng.choice([1, 3, 4, 16]))
+        pages = int(rng.integers(8, 200))
+        ctx = host_ctx(page_size=page, pages=pages)
+        ref = ReferenceFlattener(page, pages)
+        prev_n = 0
+        for step in range(4):
+            tree = random_small_tree(rng)
+            keep = None
+            if prev_n and rng.random() < 0.8:
+                keep = np.full(tree.n_nodes, -1, np.int32)
+                olds = rng.permutation(prev_n)[: tree.n_nodes]
+                for i, o in enumerate(olds):
+                    if rng.random() < 0.6:
+                        keep[i] = o
+            try:
+                want = ref.build(tree.parent, tree.tokens, tree.leaf_node, keep)
+            except PoolExhausted:
+                with pytest.raises(ets.EtsError) as e:
+                    ctx.tree_build(tree.parent, tree.tokens, tree.leaf_node, keep)
+                assert e.value.code == ets.ETS_ERR_POOL_EXHAUSTED
+                continue
+            ctx.tree_build(tree.parent, tree.tokens, tree.leaf_node, keep)
+            _assert_same_tables(ctx, want)
+            prev_n = tree.n_nodes
+
+
+def test_errors_and_unchanged_state():
+    ctx = host_ctx(pages=4)
+    ctx.tree_build([-1, 0], [16, 16], [1])
+    before = ctx.tree_export()
+    cases = [
+        (([0, -1], [4, 4], [1]), ets.ETS_ERR_BAD_TREE),
+        (([-1, 0], [4, -1], [1]), ets.ETS_ERR_BAD_TREE),
+        (([-1, 0], [4, 4], [2]), ets.ETS_ERR_BAD_TREE),
+        (([-1, 0], [4, 4], [-1]), ets.ETS_ERR_BAD_TREE),
+        (([-1, 0], [48, 48], [1]), ets.ETS_ERR_POOL_EXHAUSTED),
+    ]
+    for args, code in cases:
+        with pytest.raises(ets.EtsError) as e:
+            ctx.tree_build(*args)
+        assert e.value.code == code
+    with pytest.raises(ets.EtsError) as e:
+        ctx.tree_build([-1, 0], [4, 4], [1], keep_pages_of=[0, 0])
+    assert e.value.code == ets.ETS_ERR_BAD_TREE
+    with pytest.raises(ets.EtsError) as e:
+        ctx.tree_build([-1, 0], [4, 4], [1], keep_pages_of=[5, -1])
+    assert e.value.code == ets.ETS_ERR_BAD_TREE
+    after = ctx.tree_export()
+    for k in TABLE_KEYS:
+        assert np.array_equal(before[k], after[k])
+    # device calls on a host-only context are refused, not attempted
+    with pytest.raises(ets.EtsError) as e:
+        ctx.tree_attn_decode(0, 0, 0)
+    assert e.value.code == ets.ETS_ERR_STATE
+    with pytest.raises(ets.EtsError) as e:
+        ctx.set_option(99, 1)
+    assert e.value.code == ets.ETS_ERR_INVALID_ARG
+
+
+def test_capacity_bounds():
+    ctx = host_ctx(max_nodes=3, max_leaves=2, max_path_entries=4)
+    for args in (([-1, 0, 0, 0], [1] * 4, [1]), ([-1, 0], [1, 1], [1, 1, 1]), ([-1, 0, 1], [1, 1, 1], [2, 2])):
+        with pytest.raises(ets.EtsError) as e:
+            ctx.tree_build(*args)
+        assert e.value.code == ets.ETS_ERR_POOL_EXHAUSTED
+
+
+def test_empty_tree():
+    ctx = host_ctx()
+    ctx.tree_build([], [], [])
+    t = ctx.tree_export()
+    assert t["node_page_off"].tolist() == [0] and t["leaf_path_off"].tolist() == [0]
+    w = ctx.work_export()
+    assert w["item"].shape[0] == 0
+
+
+def _check_work(ctx, tree, cap, hkv, gqa, page=16):
+    t = ctx.tree_export()
+    w = ctx.work_export()
+    unit, item = w["unit"], w["item"]
+    leaves_per_tile = max(1, 16 // gqa)
+    covered = {}   # (page, head, leaf) -> slot
+    for it in item:
+        ub, uc, head, lb, nl, slot0, chunk, _ = (int(x) for x in it)
+        assert 1 <= nl <= leaves_per_tile
+        leaves = t["node_leaves"][lb:lb + nl].tolist()
+        for u in range(ub, ub + uc):
+            pg, node, tok0, _z = (int(x) for x in unit[u])
+            # the unit really is that page of that node
+            j = tok0 // page
+            assert t["page_ids"][t["node_page_off"][node] + j] == pg
+            # every leaf of the tile descends from the node
+            grp = t["node_leaves"][t["node_leaf_off"][node]:t["node_leaf_off"][node + 1]].tolist()
+            for i, l in enumerate(leaves):
+                assert l in grp
+                key = (pg, head, l)
+                assert key not in covered
+                covered[key] = slot0 + i
+    # every page of every node on every leaf's path is covered for every head, and the slot
+    # that holds it is listed for that leaf
+    for l in range(tree.n_leaves):
+        slots = set(w["leaf_slots"][w["leaf_slot_off"][l]:w["leaf_slot_off"][l + 1]].tolist())
+        assert len(slots) == w["leaf_slot_off"][l + 1] - w["leaf_slot_off"][l]
+        used = set()
+        for v in t["leaf_path"][t["leaf_path_off"][l]:t["leaf_path_off"][l + 1]]:
+            for pg in t["page_ids"][t["node_page_off"][v]:t["node_page_off"][v + 1]]:
+                for h in range(hkv):
+                    assert (int(pg), h, l) in covered
+                    used.add(covered[(int(pg), h, l)])
+        assert used <= slots
+    n_cov = sum((t["node_page_off"][v + 1] - t["node_page_off"][v]) *
+                (t["node_leaf_off"][v + 1] - t["node_leaf_off"][v]) for v in range(tree.n_nodes)) * hkv
+    assert len(covered) == n_cov
+    # slots of different (chunk, leaf) never collide
+    assert w["n_partial_slots"] >= (max(covered.values()) + 1 if covered else 0)
+
+
+@pytest.mark.parametrize("chunk_pages", [0, 1, 2, 5])
+def test_work_decomposition_covers_everything_once(chunk_pages):
+    rng = np.random.default_rng(41)
+    for _ in range(60):
+        hkv = int(rng.choice([1, 2]))
+        gqa = int(rng.choice([1, 4, 8]))
+        ctx = host_ctx(hq=hkv * gqa, hkv=hkv, max_path_tokens=1 << 14)
+        ctx.set_option(ets.ETS_OPT_CHUNK_PAGES, chunk_pages)
+        tree = random_small_tree(rng, max_nodes=14, max_tokens=90, max_leaves=9)
+        ctx.tree_build(tree.parent, tree.tokens, tree.leaf_node)
+        _check_work(ctx, tree, tree.tokens, hkv, gqa)
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3_ets", "cfg5a", "cfg5c"])
+def test_work_decomposition_on_configs(name):
+    wl = make_workload(name)
+    g = wl.geometry
+    ctx = host_ctx(g.num_q_heads, g.num_kv_heads, g.head_dim, pages=1 << 15, max_path_entries=1 << 14)
+    ctx.tree_build(wl.tree.parent, wl.tree.tokens, wl.tree.leaf_node)
+    _check_work(ctx, wl.tree, wl.tree.tokens, g.num_kv_heads, g.gqa)
+    st = ctx.get_stats()
+    assert st["n_segments"] <= wl.tree.n_nodes
+    if name == "cfg5a":
+        # the five shared chain steps fuse with the root: 1 shared segment + 128 private ones
+        assert st["n_segments"] == 129
