@@ -176,9 +176,11 @@ def test_rebuild_keeps_pages_and_contents():
     """A search step: leaves grow children, one branch is pruned; kept nodes keep their KV."""
     g = Geometry(8, 2, 128)
     t0 = Tree(np.array([-1, 0, 0], np.int32), np.array([40, 20, 30], np.int32), np.array([1, 2], np.int32))
-    ctx = run_and_check(t0, g, 11)
     # new tree: old 0 -> 0, old 2 -> 1 (old 1 pruned), two new children of node 1
     t1 = Tree(np.array([-1, 0, 1, 1], np.int32), np.array([40, 30, 12, 25], np.int32), np.array([2, 3], np.int32))
+    ctx = context_for_tree(8, 2, 128, t1.parent, t1.tokens, t1.leaf_node, extra_pages=4)
+    ctx.tree_build(t0.parent, t0.tokens, t0.leaf_node)
+    run_and_check(t0, g, 11, ctx=ctx)
     ctx.tree_build(t1.parent, t1.tokens, t1.leaf_node, keep_pages_of=[0, 2, -1, -1])
     assert ctx.get_node_len(0).tolist() == [40, 30, 0, 0]
     ks0, vs0 = node_values(t0, g, 11, 0)
