@@ -130,12 +130,14 @@ int32_t ets_tree_export(const ets_ctx* ctx, ets_tables_host* out);
 /*
  * The private work decomposition, exported for invariant checks only (its content is an
  * implementation choice and may change): runs of chained nodes with one query group are
- * fused into segments; segments are cut into chunks of pages; a work item is one
- * (chunk, kv head, tile of the group's leaves).
+ * fused into segments; the line of all (segment, kv head, leaf tile) page-slot runs is cut into
+ * equal-cost pieces, one per resident warp of the attention kernel; a work item is one run or
+ * the part of a run inside one piece.
  *   unit[n_units*4]     per page slot: page id, node, first token index within the node, 0
  *   item[n_items*8]     unit_begin, unit_count, kv_head, leaf_list_begin (into node_leaves),
- *                       n_leaves_in_tile, partial_slot_of_first_leaf, chunk id, 0
- *   leaf_slot_off[n_leaves+1], leaf_slots[n_leaf_slots]  partial slots to merge per leaf
+ *                       n_leaves_in_tile, partial_slot_of_first_leaf, segment id, 0
+ *   leaf_slot_off[n_leaves*num_kv_heads+1], leaf_slots[n_leaf_slots]
+ *                       partial slots to merge per (leaf, kv head)
  */
 typedef struct ets_work_host {
     int64_t n_units, n_items, n_leaf_slots, n_partial_slots;
@@ -207,7 +209,7 @@ typedef struct ets_stats {
 int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
 
 /* Tuning and instrumentation knobs; unknown keys give ETS_ERR_INVALID_ARG. */
-#define ETS_OPT_CHUNK_PAGES   1  /* pages per chunk (0 = automatic); applies at the next build   */
+#define ETS_OPT_CHUNK_PAGES   1  /* longest page run per work item (0 = no limit); next build    */
 #define ETS_OPT_KERNEL        2  /* 0 automatic, 1 scalar-FMA kernel only                       */
 #define ETS_OPT_TIMING        3  /* 1: bracket the attention and merge kernels with events      */
 int32_t ets_set_option(ets_ctx* ctx, int32_t key, int64_t value);

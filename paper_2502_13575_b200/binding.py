@@ -234,10 +234,10 @@ class EtsContext:
     def work_export(self) -> Dict[str, np.ndarray]:
         w = ets_work_host()
         self._check(lib.ets_work_export(self._h, C.byref(w)))
-        n_leaves = self.get_stats()["n_leaves"]
+        n_lists = self.get_stats()["n_leaves"] * self.cfg.num_kv_heads
         out = {
             "unit": np.zeros(w.n_units * 4, np.int32), "item": np.zeros(w.n_items * 8, np.int32),
-            "leaf_slot_off": np.zeros(n_leaves + 1, np.int32), "leaf_slots": np.zeros(w.n_leaf_slots, np.int32),
+            "leaf_slot_off": np.zeros(n_lists + 1, np.int32), "leaf_slots": np.zeros(w.n_leaf_slots, np.int32),
         }
         for k, a in out.items():
             setattr(w, k, _p(a))

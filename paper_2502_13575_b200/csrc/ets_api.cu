@@ -21,6 +21,7 @@ namespace {
 constexpr int kStages = 3;        // pinned staging buffers for table uploads
 constexpr int kDescSlots = 8;     // pinned/device descriptor slots for appends
 constexpr int kTimingCap = 8192;  // decode calls that can be timed between two reads
+constexpr int kMaxWorkers = 2048; // warp-workers of the attention kernel the tables are sized for
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -65,8 +66,12 @@ Layout make_layout(const ets_config* c) {
     Layout L{};
     const int64_t path_pages = (int64_t)c->max_leaves * ((c->max_path_tokens + c->page_size - 1) / c->page_size) +
                                c->max_path_entries;
-    L.max_partial_slots = c->max_path_entries + (path_pages + 7) / 8;
-    L.max_items = L.max_partial_slots * c->num_kv_heads;
+    // a partial slot belongs to one (item, leaf); items are (segment piece, kv head, leaf tile), and
+    // each worker boundary can split one more item
+    const int gqa = c->num_q_heads / c->num_kv_heads;
+    L.max_partial_slots = (c->max_path_entries + (path_pages + 7) / 8) * c->num_kv_heads +
+                          (int64_t)kMaxWorkers * (16 / gqa > 0 ? 16 / gqa : 1);
+    L.max_items = L.max_partial_slots;
     L.max_units = c->pages_per_layer;
     L.max_append_tokens = c->max_append_tokens > 0 ? c->max_append_tokens : c->max_leaves;
     const size_t A = 1024;
@@ -76,7 +81,8 @@ Layout make_layout(const ets_config* c) {
     blob += align_up(((size_t)c->max_nodes + 1) * 4, 256);          // node_page_off
     blob += align_up((size_t)c->pages_per_layer * 4, 256);          // page_ids
     blob += align_up((size_t)c->max_path_entries * 4, 256);         // node_leaves
-    blob += align_up(((size_t)c->max_leaves + 1) * 4, 256);         // leaf_slot_off
+    blob += align_up(((size_t)c->max_leaves * c->num_kv_heads + 1) * 4, 256);  // leaf_slot_off
+    blob += align_up(((size_t)kMaxWorkers + 1) * 4, 256);           // worker_off
     blob += align_up((size_t)L.max_partial_slots * 4, 256);         // leaf_slots
     blob += align_up((size_t)c->num_layers * c->max_nodes * 4, 256);  // node_len
     L.blob_cap = align_up(blob, A);
@@ -84,7 +90,7 @@ Layout make_layout(const ets_config* c) {
     L.blob = off; off += L.blob_cap;
     L.desc_slot_bytes = align_up((size_t)c->max_nodes * 16, 256);
     L.desc = off; off += align_up(L.desc_slot_bytes * kDescSlots, A);
-    const size_t rows = (size_t)L.max_partial_slots * c->num_q_heads;
+    const size_t rows = (size_t)L.max_partial_slots * gqa;
     L.part_ml = off; off += align_up(rows * 8, A);
     L.part_o = off; off += align_up(rows * c->head_dim * 4, A);
     const size_t qbytes = (size_t)c->max_leaves * c->num_q_heads * c->head_dim * 2;
@@ -100,7 +106,7 @@ Layout make_layout(const ets_config* c) {
 }
 
 struct BlobOffsets {  // offsets of the packed tables of the current tree inside the device blob
-    size_t units, items, node_page_off, page_ids, node_leaves, leaf_slot_off, leaf_slots, node_len, total;
+    size_t units, items, node_page_off, page_ids, node_leaves, leaf_slot_off, leaf_slots, worker_off, node_len, total;
     int32_t len_stride;
 };
 
@@ -171,6 +177,7 @@ BlobOffsets pack_offsets(const ets_ctx* c, const ets::Tree& t) {
     b.node_leaves = take(t.node_leaves.size() * 4);
     b.leaf_slot_off = take(t.leaf_slot_off.size() * 4);
     b.leaf_slots = take(t.leaf_slots.size() * 4);
+    b.worker_off = take(t.worker_off.size() * 4);
     b.len_stride = t.n_nodes > 0 ? t.n_nodes : 1;
     b.node_len = take((size_t)c->cfg.num_layers * b.len_stride * 4);
     b.total = off;
@@ -186,6 +193,7 @@ void pack_blob(const ets_ctx* c, const ets::Tree& t, const BlobOffsets& b, char*
     put(b.node_leaves, t.node_leaves.data(), t.node_leaves.size() * 4);
     put(b.leaf_slot_off, t.leaf_slot_off.data(), t.leaf_slot_off.size() * 4);
     put(b.leaf_slots, t.leaf_slots.data(), t.leaf_slots.size() * 4);
+    put(b.worker_off, t.worker_off.data(), t.worker_off.size() * 4);
     for (int l = 0; l < c->cfg.num_layers; ++l)
         put(b.node_len + (size_t)l * b.len_stride * 4, t.len[l].data(), t.len[l].size() * 4);
 }
@@ -261,13 +269,14 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
             }
             if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->status_host, 64, cudaHostAllocDefault);
             if (e == cudaSuccess) e = cudaMemset(c->ws + c->lay.status, 0, 1024);
+            if (e == cudaSuccess) e = ets::narrow_prepare(cfg->head_dim);
         }
         if (e != cudaSuccess) {
             ets_destroy(c);
             return ETS_ERR_CUDA;
         }
     }
-    c->fp.n_workers = c->sm_count;
+    c->fp.n_workers = c->sm_count * ets::kNarrowWarps < kMaxWorkers ? c->sm_count * ets::kNarrowWarps : kMaxWorkers;
     ets::tree_init(c->tree, c->fp, cfg->pages_per_layer);
     *out = c;
     return ETS_OK;
@@ -522,6 +531,8 @@ static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, 
     a.G = c->cfg.num_q_heads / c->cfg.num_kv_heads;
     a.pages_per_layer = c->cfg.pages_per_layer;
     a.scale_log2 = c->scale_log2;
+    a.worker_off = blob_ptr<int32_t>(c, c->bo.worker_off);
+    a.n_workers = c->fp.n_workers;
 
     cudaEvent_t* ev = nullptr;
     if (c->opt_timing) {
@@ -538,7 +549,8 @@ static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, 
         ev = &c->tev[3 * c->timed_calls];
         ETS_CUDA(c, cudaEventRecord(ev[0], s));
     }
-    ets::launch_partial_fma(a, c->cfg.head_dim, s);
+    if (c->opt_kernel == 1) ets::launch_partial_fma(a, c->cfg.head_dim, s);
+    else ets::launch_partial_narrow(a, c->cfg.head_dim, (c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps, s);
     if (ev) ETS_CUDA(c, cudaEventRecord(ev[1], s));
     ets::launch_merge(a, c->cfg.head_dim, s);
     if (ev) {

@@ -16,6 +16,7 @@ namespace ets {
 //              + (e%8) * 2
 // i.e. rows of 128 bytes in 1024-byte atoms with the 128-byte swizzle pattern.
 constexpr int kPageTokens = 16;
+constexpr int kNarrowWarps = 8;   // independent warp-workers per CTA of the narrow attention kernel
 
 __host__ __device__ inline size_t tile_bytes(int D) { return (size_t)kPageTokens * D * 2; }
 
@@ -27,7 +28,7 @@ __host__ __device__ inline uint32_t tile_offset(int D, int t, int e) {
 
 struct DevItem {
     int32_t unit_begin, unit_count, kv_head, leaf_list_begin;
-    int32_t n_leaves_tile, slot_first, chunk, reserved;
+    int32_t n_leaves_tile, slot_first, segment, reserved;
 };
 
 // Everything a decode launch needs; passed by value.
@@ -36,15 +37,17 @@ struct DecodeArgs {
     const DevItem* items;
     const int32_t* node_leaves;
     const int32_t* node_len;       // this layer's lengths
-    const int32_t* leaf_slot_off;
+    const int32_t* leaf_slot_off;  // per (leaf, kv head)
     const int32_t* leaf_slots;
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
     float* lse;
     const char* k_pool;            // this layer's pools
     const char* v_pool;
-    float2* part_ml;               // [slot][Hq]  (m in log2 units, l)
-    float* part_o;                 // [slot][Hq][D]
+    float2* part_ml;               // [slot][G]  (m in log2 units, l); a slot belongs to one kv head
+    float* part_o;                 // [slot][G][D]
+    const int32_t* worker_off;     // items of warp-worker w: [worker_off[w], worker_off[w+1])
+    int32_t n_workers;
     int32_t* status;
     int32_t n_items, n_leaves, n_units;
     int32_t Hq, Hkv, G;
@@ -72,5 +75,8 @@ void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* page_
                     int Hkv, int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s);
 void launch_partial_fma(const DecodeArgs& a, int D, cudaStream_t s);
 void launch_merge(const DecodeArgs& a, int D, cudaStream_t s);
+size_t narrow_smem_bytes(int D);
+cudaError_t narrow_prepare(int D);
+void launch_partial_narrow(const DecodeArgs& a, int D, int n_ctas, cudaStream_t s);
 
 }  // namespace ets

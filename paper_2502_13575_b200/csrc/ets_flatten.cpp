@@ -2,6 +2,8 @@
 #include "ets_flatten.hpp"
 
 #include <algorithm>
+#include <climits>
+#include <cmath>
 #include <functional>
 #include <numeric>
 
@@ -16,6 +18,7 @@ void tree_init(Tree& t, const FlattenParams& p, int64_t pages_per_layer) {
     t.node_leaf_off.assign(1, 0);
     t.leaf_path_off.assign(1, 0);
     t.leaf_slot_off.assign(1, 0);
+    t.worker_off.assign((size_t)std::max(1, p.n_workers) + 1, 0);
 }
 
 static inline int32_t ceil_div(int32_t a, int32_t b) { return (a + b - 1) / b; }
@@ -170,69 +173,83 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             }
     }
 
-    // ---- chunking: enough (chunk, head) pairs to keep every worker busy several times over
-    int32_t cp = p.chunk_pages;
-    if (cp <= 0) {
-        int64_t want_items = (int64_t)p.n_workers * 8;
-        int64_t c = (n_units * p.num_kv_heads) / std::max<int64_t>(want_items, 1);
-        cp = (int32_t)std::min<int64_t>(std::max<int64_t>(c, 8), 64);
-    }
-    t.chunk_pages_used = cp;
+    // ---- work line: for every segment, kv head and leaf tile, the segment's page slots.  The line
+    // is cut into n_workers contiguous pieces of equal cost (a page slot costs 1, starting an item
+    // costs kItemCost), so a piece boundary may fall inside a run and split it into two items.
+    // Tiles of one (segment, head) are adjacent: the re-read of its K/V by the next tile is recent.
     const int32_t leaves_per_tile = std::max(1, p.rows_per_item / std::max(1, p.gqa));
-
-    struct Chunk { int32_t ub, uc, seg, slot_base; };
-    std::vector<Chunk> chunks;
-    std::vector<int32_t> seg_chunk_off((size_t)n_seg + 1, 0);
+    const int32_t n_workers = std::max(1, p.n_workers);
+    const int32_t max_run = p.chunk_pages > 0 ? p.chunk_pages : INT32_MAX;
+    constexpr double kItemCost = 2.0;
+    int64_t n_runs = 0, run_units = 0;
+    for (int32_t s = 0; s < n_seg; ++s) {
+        const int64_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
+        if (nu == 0) continue;
+        const int64_t tiles = ceil_div(g[seg_head[s]], leaves_per_tile);
+        n_runs += tiles * p.num_kv_heads;
+        run_units += nu * tiles * p.num_kv_heads;
+    }
+    const double target = ((double)run_units + kItemCost * (double)(n_runs + n_workers)) / n_workers;
+    t.chunk_pages_used = p.chunk_pages;
+    t.worker_off.assign((size_t)n_workers + 1, 0);
+    int32_t w = 0;
+    double load = 0.0;
     int64_t slots = 0;
     for (int32_t s = 0; s < n_seg; ++s) {
-        int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
-        int32_t nc = std::max(1, ceil_div(nu, cp));   // a segment without pages still gets one (empty) chunk
-        int32_t base = nu / nc, rem = nu % nc, ub = seg_unit_off[s];
-        for (int32_t c = 0; c < nc; ++c) {
-            int32_t uc = base + (c < rem ? 1 : 0);
-            chunks.push_back({ub, uc, s, (int32_t)slots});
-            slots += g[seg_head[s]];
-            ub += uc;
-        }
-        seg_chunk_off[s + 1] = (int32_t)chunks.size();
-    }
-    if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
-    t.n_chunks = (int64_t)chunks.size();
-    t.n_partial_slots = slots;
-
-    // ---- items: (chunk, kv head, leaf tile); tiles of one (chunk, head) are adjacent so that
-    // the re-reads of its K/V by later tiles hit in L2
-    for (size_t c = 0; c < chunks.size(); ++c) {
-        const Chunk& ch = chunks[c];
-        int32_t head = seg_head[ch.seg];
-        int32_t gn = g[head];
+        const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
+        if (nu == 0) continue;
+        const int32_t head_node = seg_head[s];
+        const int32_t gn = g[head_node];
         for (int32_t h = 0; h < p.num_kv_heads; ++h)
             for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile) {
-                Item it;
-                it.unit_begin = ch.ub;
-                it.unit_count = ch.uc;
-                it.kv_head = h;
-                it.leaf_list_begin = t.node_leaf_off[head] + l0;
-                it.n_leaves_tile = std::min(leaves_per_tile, gn - l0);
-                it.slot_first = ch.slot_base + l0;
-                it.chunk = (int32_t)c;
-                it.reserved = 0;
-                t.items.push_back(it);
+                int32_t done = 0;
+                while (done < nu) {
+                    if (w < n_workers - 1 && target - load < kItemCost + 1.0) {
+                        ++w;
+                        t.worker_off[w] = (int32_t)t.items.size();
+                        load = 0.0;
+                    }
+                    int32_t take = nu - done;
+                    if (w < n_workers - 1) {
+                        const double room = target - load - kItemCost;
+                        take = (int32_t)std::min<double>(take, std::max(1.0, std::floor(room)));
+                    }
+                    take = std::min(take, max_run);
+                    Item it;
+                    it.unit_begin = seg_unit_off[s] + done;
+                    it.unit_count = take;
+                    it.kv_head = h;
+                    it.leaf_list_begin = t.node_leaf_off[head_node] + l0;
+                    it.n_leaves_tile = std::min(leaves_per_tile, gn - l0);
+                    it.slot_first = (int32_t)slots;
+                    it.segment = s;
+                    it.reserved = 0;
+                    t.items.push_back(it);
+                    slots += it.n_leaves_tile;
+                    load += take + kItemCost;
+                    done += take;
+                    if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
+                }
             }
     }
+    for (int32_t k = w + 1; k <= n_workers; ++k) t.worker_off[k] = (int32_t)t.items.size();
+    t.n_chunks = (int64_t)t.items.size();
+    t.n_partial_slots = slots;
     if ((int64_t)t.items.size() > p.max_items) { err = "work items exceed the workspace bound"; return F_EXHAUSTED; }
 
-    // ---- per leaf: the partial slots to merge (one per chunk of every segment on its path)
-    t.leaf_slot_off.assign((size_t)n_leaves + 1, 0);
-    for (int32_t l = 0; l < n_leaves; ++l) {
-        for (int32_t e = t.leaf_path_off[l]; e < t.leaf_path_off[l + 1]; ++e) {
-            int32_t v = t.leaf_path[e];
-            int32_t s = seg_of[v];
-            if (seg_head[s] != v) continue;
-            for (int32_t c = seg_chunk_off[s]; c < seg_chunk_off[s + 1]; ++c)
-                t.leaf_slots.push_back(chunks[c].slot_base + t.leaf_path_pos[e]);
-        }
-        t.leaf_slot_off[l + 1] = (int32_t)t.leaf_slots.size();
+    // ---- per (leaf, kv head): the partial slots to merge
+    const int32_t H = p.num_kv_heads;
+    t.leaf_slot_off.assign((size_t)n_leaves * H + 1, 0);
+    for (const Item& it : t.items)
+        for (int32_t i = 0; i < it.n_leaves_tile; ++i)
+            ++t.leaf_slot_off[(size_t)t.node_leaves[it.leaf_list_begin + i] * H + it.kv_head + 1];
+    for (size_t k = 0; k < (size_t)n_leaves * H; ++k) t.leaf_slot_off[k + 1] += t.leaf_slot_off[k];
+    t.leaf_slots.assign((size_t)t.leaf_slot_off[(size_t)n_leaves * H], 0);
+    {
+        std::vector<int32_t> cur(t.leaf_slot_off.begin(), t.leaf_slot_off.end() - 1);
+        for (const Item& it : t.items)
+            for (int32_t i = 0; i < it.n_leaves_tile; ++i)
+                t.leaf_slots[(size_t)cur[(size_t)t.node_leaves[it.leaf_list_begin + i] * H + it.kv_head]++] = it.slot_first + i;
     }
     return F_OK;
 }

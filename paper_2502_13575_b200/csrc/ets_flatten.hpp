@@ -21,15 +21,15 @@ struct FlattenParams {
     int64_t max_path_entries = 0;
     int64_t max_partial_slots = 0;
     int64_t max_items = 0;
-    int32_t chunk_pages = 0;    // 0 = automatic
+    int32_t chunk_pages = 0;    // longest run of page slots in one item (0 = unlimited)
     int32_t rows_per_item = 16; // query rows (leaves * gqa) one work item covers
-    int32_t n_workers = 148;    // CTAs the attention kernel keeps resident (for chunk sizing)
+    int32_t n_workers = 148 * 8; // warps the attention kernel keeps resident; each gets one piece of the work
 };
 
 // One work item, as uploaded to the device (8 x int32).
 struct Item {
     int32_t unit_begin, unit_count, kv_head, leaf_list_begin;
-    int32_t n_leaves_tile, slot_first, chunk, reserved;
+    int32_t n_leaves_tile, slot_first, segment, reserved;
 };
 
 struct Tree {
@@ -43,7 +43,8 @@ struct Tree {
     // work decomposition
     std::vector<int32_t> unit;              // 4 per unit: page, node, tok0, 0
     std::vector<Item> items;
-    std::vector<int32_t> leaf_slot_off, leaf_slots;
+    std::vector<int32_t> leaf_slot_off, leaf_slots;   // per (leaf, kv head)
+    std::vector<int32_t> worker_off;                  // items of worker w: [worker_off[w], worker_off[w+1])
     int64_t n_segments = 0, n_chunks = 0, n_partial_slots = 0;
     int32_t chunk_pages_used = 0;
 };

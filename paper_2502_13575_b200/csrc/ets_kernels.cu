@@ -189,8 +189,7 @@ __global__ void __launch_bounds__(kFmaWarps * 32) attn_partial_fma_kernel(Decode
             acc += wgt * sm_o[w][r][e];
             ls += wgt * sm_l[w][r];
         }
-        const int slot = it.slot_first + r / G;
-        const size_t row = (size_t)slot * a.Hq + h * G + r % G;
+        const size_t row = (size_t)(it.slot_first + r / G) * G + r % G;
         a.part_o[row * D + e] = acc;
         if (e == 0) a.part_ml[row] = make_float2(ms, ls);
     }
@@ -215,11 +214,13 @@ __global__ void __launch_bounds__(128) lse_merge_kernel(DecodeArgs a) {
     const int64_t row = (int64_t)blockIdx.x * 4 + warp;
     if (row >= (int64_t)a.n_leaves * a.Hq) return;
     const int leaf = (int)(row / a.Hq), head = (int)(row % a.Hq);
-    const int s0 = a.leaf_slot_off[leaf], s1 = a.leaf_slot_off[leaf + 1];
+    const int G = a.G, sub = head % G;
+    const int list = leaf * a.Hkv + head / G;
+    const int s0 = a.leaf_slot_off[list], s1 = a.leaf_slot_off[list + 1];
 
     float ms = -INFINITY;
     for (int j = s0 + lane; j < s1; j += 32) {
-        const float2 ml = a.part_ml[(size_t)a.leaf_slots[j] * a.Hq + head];
+        const float2 ml = a.part_ml[(size_t)a.leaf_slots[j] * G + sub];
         if (ml.y > 0.f) ms = fmaxf(ms, ml.x);
     }
 #pragma unroll
@@ -230,7 +231,7 @@ __global__ void __launch_bounds__(128) lse_merge_kernel(DecodeArgs a) {
     for (int j = 0; j < EPL; ++j) acc[j] = 0.f;
     float ls = 0.f;
     for (int j = s0; j < s1; ++j) {
-        const size_t prow = (size_t)a.leaf_slots[j] * a.Hq + head;
+        const size_t prow = (size_t)a.leaf_slots[j] * G + sub;
         const float2 ml = a.part_ml[prow];
         if (!(ml.y > 0.f)) continue;
         const float w = exp2f(ml.x - ms);

@@ -162,8 +162,8 @@ def _check_work(ctx, tree, cap, hkv, gqa, page=16):
     leaves_per_tile = max(1, 16 // gqa)
     covered = {}   # (page, head, leaf) -> slot
     for it in item:
-        ub, uc, head, lb, nl, slot0, chunk, _ = (int(x) for x in it)
-        assert 1 <= nl <= leaves_per_tile
+        ub, uc, head, lb, nl, slot0, seg, _ = (int(x) for x in it)
+        assert 1 <= nl <= leaves_per_tile and uc >= 1
         leaves = t["node_leaves"][lb:lb + nl].tolist()
         for u in range(ub, ub + uc):
             pg, node, tok0, _z = (int(x) for x in unit[u])
@@ -180,15 +180,16 @@ def _check_work(ctx, tree, cap, hkv, gqa, page=16):
     # every page of every node on every leaf's path is covered for every head, and the slot
     # that holds it is listed for that leaf
     for l in range(tree.n_leaves):
-        slots = set(w["leaf_slots"][w["leaf_slot_off"][l]:w["leaf_slot_off"][l + 1]].tolist())
-        assert len(slots) == w["leaf_slot_off"][l + 1] - w["leaf_slot_off"][l]
-        used = set()
-        for v in t["leaf_path"][t["leaf_path_off"][l]:t["leaf_path_off"][l + 1]]:
-            for pg in t["page_ids"][t["node_page_off"][v]:t["node_page_off"][v + 1]]:
-                for h in range(hkv):
+        for h in range(hkv):
+            k = l * hkv + h
+            slots = w["leaf_slots"][w["leaf_slot_off"][k]:w["leaf_slot_off"][k + 1]].tolist()
+            assert len(set(slots)) == len(slots)
+            used = set()
+            for v in t["leaf_path"][t["leaf_path_off"][l]:t["leaf_path_off"][l + 1]]:
+                for pg in t["page_ids"][t["node_page_off"][v]:t["node_page_off"][v + 1]]:
                     assert (int(pg), h, l) in covered
                     used.add(covered[(int(pg), h, l)])
-        assert used <= slots
+            assert used == set(slots)
     n_cov = sum((t["node_page_off"][v + 1] - t["node_page_off"][v]) *
                 (t["node_leaf_off"][v + 1] - t["node_leaf_off"][v]) for v in range(tree.n_nodes)) * hkv
     assert len(covered) == n_cov
