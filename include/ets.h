@@ -189,6 +189,24 @@ int32_t ets_tree_attn_decode_host(ets_ctx* ctx, int32_t layer, const void* q, vo
                                   float* lse, void* cuda_stream);
 
 /*
+ * Tree-decode attention for callers that cannot allocate device memory (the paper has no
+ * counterpart: this is a packaging convenience, not a step of the method).  Same arguments,
+ * result and errors as ets_tree_attn_decode (DEVICE pointers), but the partial results between
+ * the attention and merge kernels live in an 8 MiB array built into the library instead of the
+ * caller's workspace.  Meant for embedders whose host application owns the memory budget or
+ * forbids allocation calls on its hot path (a cudaMalloc may synchronise the device).
+ *   - Limit: partial_slots * (Hq/Hkv) * (head_dim + 2) * 4 bytes (see ets_get_stats) must fit in
+ *     8 MiB; larger trees are refused with ETS_ERR_POOL_EXHAUSTED and a message.
+ *   - The first call on each device looks up the array's device address; make it before starting
+ *     any stream capture.  The call itself makes no allocation of any kind.
+ *   - One array per GPU, shared by every call and context: calls that overlap in time on the
+ *     same GPU corrupt each other.  The array keeps old contents between calls; none of it needs
+ *     clearing, because each call rewrites every slot it later reads.
+ */
+int32_t ets_tree_attn_decode_static(ets_ctx* ctx, int32_t layer, const void* q, void* out, float* lse,
+                                    void* cuda_stream);
+
+/*
  * Read one node's current K and V rows of one layer back in token order:
  * bf16 [node_len, num_kv_heads, head_dim] each, DEVICE pointers (either may be NULL).
  */

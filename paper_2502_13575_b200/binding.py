@@ -92,6 +92,7 @@ _SIGNATURES = {
     "ets_get_node_len": (C.c_int32, [C.c_void_p, C.c_int32, _I32P]),
     "ets_tree_attn_decode": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_tree_attn_decode_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ets_tree_attn_decode_static": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_kv_read_debug": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_get_stats": (C.c_int32, [C.c_void_p, C.POINTER(ets_stats)]),
     "ets_set_option": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int64]),
@@ -270,6 +271,12 @@ class EtsContext:
     def tree_attn_decode_host(self, layer: int, q, out, lse=None, stream=None):
         self._check(lib.ets_tree_attn_decode_host(self._h, layer, _dev_ptr(q), _dev_ptr(out), _dev_ptr(lse),
                                                   _stream_ptr(stream)))
+
+    def tree_attn_decode_static(self, layer: int, q, out, lse=None, stream=None):
+        """Decode using the library's built-in 8 MiB scratch: for callers that may not allocate
+        device memory.  Small trees only; calls on one GPU must not overlap."""
+        self._check(lib.ets_tree_attn_decode_static(self._h, layer, _dev_ptr(q), _dev_ptr(out), _dev_ptr(lse),
+                                                    _stream_ptr(stream)))
 
     def kv_read_debug(self, layer: int, node: int, k_out, v_out, stream=None):
         self._check(lib.ets_kv_read_debug(self._h, layer, node, _dev_ptr(k_out), _dev_ptr(v_out),

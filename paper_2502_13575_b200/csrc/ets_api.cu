@@ -595,6 +595,91 @@ int32_t ets_tree_attn_decode_host(ets_ctx* c, int32_t layer, const void* q, void
     return ETS_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Decode with built-in scratch, for callers that must not allocate.
+//
+// Some users of this library cannot create device allocations of their own: a plugin that runs
+// inside a host application's fixed memory budget, code that is called while another component
+// owns the allocator, or a real-time loop in which cudaMalloc (which may synchronise the whole
+// device) is not allowed.  Such callers still hand over q and out, but cannot provide room for
+// the partial results that the attention kernel writes and the merge kernel reads.  For them the
+// library carries a fixed 8 MiB array in device memory; it exists once per GPU that loads the
+// library and stays until the process ends.
+//
+// The array's name is only meaningful to device code.  Host code must translate it with
+// cudaGetSymbolAddress, per device and with that device current; that is done on the first call
+// for a device and cached.  That first call therefore performs a runtime query and should be made
+// before any stream capture begins.
+//
+// All calls share the one array and it keeps the previous call's contents.  Nothing in it needs to
+// start at zero: every partial slot that the merge kernel reads is written in full by the
+// attention kernel of the same call.  Two calls that overlap on the GPU (different streams, or
+// two contexts on one device) would overwrite each other's partials: run them one after another.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kStaticScratchBytes = (size_t)8 << 20;
+constexpr int kStaticMaxDevices = 64;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+unsigned char* g_static_scratch_addr[kStaticMaxDevices] = {};
+}  // namespace
+
+int32_t ets_tree_attn_decode_static(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse,
+                                    void* cuda_stream) {
+    if (int32_t rc = decode_check(c, layer, q, out)) return rc;
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, ETS_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
+    const int dev = c->cfg.device;
+    if (dev >= kStaticMaxDevices) return fail(c, ETS_ERR_UNSUPPORTED, "device ordinal beyond the built-in scratch table");
+    const ets::Tree& t = c->tree;
+    const int G = c->cfg.num_q_heads / c->cfg.num_kv_heads;
+    const int D = c->cfg.head_dim;
+    const size_t rows = (size_t)t.n_partial_slots * G;
+    const size_t ml_bytes = align_up(rows * sizeof(float2), 256);
+    const size_t need = ml_bytes + rows * D * sizeof(float);
+    if (need > kStaticScratchBytes)
+        return fail(c, ETS_ERR_POOL_EXHAUSTED,
+                    "tree needs " + std::to_string(need) + " bytes of partial results; the built-in scratch holds " +
+                        std::to_string(kStaticScratchBytes) + " (use ets_tree_attn_decode with a workspace)");
+    ETS_CUDA(c, cudaSetDevice(dev));
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        ETS_CUDA(c, cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_scratch_addr[dev] = static_cast<unsigned char*>(p);
+    }
+    if (t.n_leaves == 0) return ETS_OK;
+    unsigned char* scratch = g_static_scratch_addr[dev];
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    ets::DecodeArgs a{};
+    a.units = blob_ptr<int4>(c, c->bo.units);
+    a.items = blob_ptr<ets::DevItem>(c, c->bo.items);
+    a.node_leaves = blob_ptr<int32_t>(c, c->bo.node_leaves);
+    a.node_len = blob_ptr<int32_t>(c, c->bo.node_len) + (size_t)layer * c->bo.len_stride;
+    a.leaf_slot_off = blob_ptr<int32_t>(c, c->bo.leaf_slot_off);
+    a.leaf_slots = blob_ptr<int32_t>(c, c->bo.leaf_slots);
+    a.q = reinterpret_cast<const __nv_bfloat16*>(q);
+    a.out = reinterpret_cast<__nv_bfloat16*>(out);
+    a.lse = lse;
+    a.k_pool = c->k_pool + (size_t)layer * c->layer_pool_bytes;
+    a.v_pool = c->v_pool + (size_t)layer * c->layer_pool_bytes;
+    a.part_ml = reinterpret_cast<float2*>(scratch);
+    a.part_o = reinterpret_cast<float*>(scratch + ml_bytes);
+    a.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
+    a.n_items = (int32_t)t.items.size();
+    a.n_leaves = t.n_leaves;
+    a.n_units = (int32_t)(t.unit.size() / 4);
+    a.Hq = c->cfg.num_q_heads;
+    a.Hkv = c->cfg.num_kv_heads;
+    a.G = G;
+    a.pages_per_layer = c->cfg.pages_per_layer;
+    a.scale_log2 = c->scale_log2;
+    a.worker_off = blob_ptr<int32_t>(c, c->bo.worker_off);
+    a.n_workers = c->fp.n_workers;
+    if (c->opt_kernel == 1) ets::launch_partial_fma(a, D, s);
+    else ets::launch_partial_narrow(a, D, (c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps, s);
+    ets::launch_merge(a, D, s);
+    ETS_CUDA(c, cudaGetLastError());
+    return ETS_OK;
+}
+
 int32_t ets_kv_read_debug(ets_ctx* c, int32_t layer, int32_t node, void* k_out, void* v_out, void* cuda_stream) {
     if (!c) return ETS_ERR_INVALID_ARG;
     if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
