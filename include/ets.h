@@ -138,10 +138,11 @@ int32_t ets_tree_export(const ets_ctx* ctx, ets_tables_host* out);
  *                       n_leaves_in_tile, partial_slot_of_first_leaf, segment id, 0
  *   leaf_slot_off[n_leaves*num_kv_heads+1], leaf_slots[n_leaf_slots]
  *                       partial slots to merge per (leaf, kv head)
+ *   worker_off[n_workers+1]   items of resident warp w: [worker_off[w], worker_off[w+1])
  */
 typedef struct ets_work_host {
-    int64_t n_units, n_items, n_leaf_slots, n_partial_slots;
-    int32_t *unit, *item, *leaf_slot_off, *leaf_slots;
+    int64_t n_units, n_items, n_leaf_slots, n_partial_slots, n_workers;
+    int32_t *unit, *item, *leaf_slot_off, *leaf_slots, *worker_off;
 } ets_work_host;
 int32_t ets_work_export(const ets_ctx* ctx, ets_work_host* out);
 

@@ -67,8 +67,8 @@ class ets_tables_host(C.Structure):
 class ets_work_host(C.Structure):
     _fields_ = [
         ("n_units", C.c_int64), ("n_items", C.c_int64), ("n_leaf_slots", C.c_int64),
-        ("n_partial_slots", C.c_int64),
-        ("unit", _I32P), ("item", _I32P), ("leaf_slot_off", _I32P), ("leaf_slots", _I32P),
+        ("n_partial_slots", C.c_int64), ("n_workers", C.c_int64),
+        ("unit", _I32P), ("item", _I32P), ("leaf_slot_off", _I32P), ("leaf_slots", _I32P), ("worker_off", _I32P),
     ]
 
 
@@ -239,6 +239,7 @@ class EtsContext:
         out = {
             "unit": np.zeros(w.n_units * 4, np.int32), "item": np.zeros(w.n_items * 8, np.int32),
             "leaf_slot_off": np.zeros(n_lists + 1, np.int32), "leaf_slots": np.zeros(w.n_leaf_slots, np.int32),
+            "worker_off": np.zeros(w.n_workers + 1, np.int32),
         }
         for k, a in out.items():
             setattr(w, k, _p(a))

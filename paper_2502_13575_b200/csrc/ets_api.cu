@@ -382,6 +382,8 @@ int32_t ets_work_export(const ets_ctx* c, ets_work_host* o) {
     o->n_items = (int64_t)t.items.size();
     o->n_leaf_slots = (int64_t)t.leaf_slots.size();
     o->n_partial_slots = t.n_partial_slots;
+    o->n_workers = (int64_t)t.worker_off.size() - 1;
+    if (o->worker_off && !t.worker_off.empty()) std::memcpy(o->worker_off, t.worker_off.data(), t.worker_off.size() * 4);
     if (o->unit && !t.unit.empty()) std::memcpy(o->unit, t.unit.data(), t.unit.size() * 4);
     if (o->item && !t.items.empty()) std::memcpy(o->item, t.items.data(), t.items.size() * sizeof(ets::Item));
     if (o->leaf_slot_off) std::memcpy(o->leaf_slot_off, t.leaf_slot_off.data(), t.leaf_slot_off.size() * 4);

@@ -89,12 +89,50 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// A batch of up to 32 consecutive page slots of an item, one per lane: its page id and the number
+// of tokens it holds now (0 = skip: empty, or a page id outside the pool, which is also flagged).
+// Loading descriptors 32 at a time keeps the dependent global loads (slot -> node length) off the
+// per-tile critical path.
+struct UnitBatch {
+    int base = 0;       // index (within the item) of lane 0's slot
+    int page = 0;
+    int valid = 0;
+    uint32_t live = 0;  // bit i: lane i's slot has tokens
+
+    __device__ __forceinline__ void load(const DecodeArgs& a, int unit_begin, int unit_count, int from, int lane) {
+        base = from;
+        const int idx = from + lane;
+        page = 0;
+        valid = 0;
+        if (idx < unit_count) {
+            const int4 un = a.units[unit_begin + idx];
+            int v = a.node_len[un.y] - un.z;
+            v = v < 0 ? 0 : (v > 16 ? 16 : v);
+            if (v > 0 && (un.x < 0 || (int64_t)un.x >= a.pages_per_layer)) {  // never read outside the pool
+                atomicExch(a.status, -1);
+                v = 0;
+            }
+            page = un.x;
+            valid = v;
+        }
+        live = __ballot_sync(0xffffffffu, valid > 0);
+    }
+    // first live slot at or after item index u inside this batch, or -1
+    __device__ __forceinline__ int next_live(int u) const {
+        const int sh = u - base;
+        if (sh >= 32) return -1;
+        const uint32_t m = live >> sh;
+        return m ? u + __ffs(m) - 1 : -1;
+    }
+};
+
 // Issue side of a warp's ring: walks the worker's items and their page slots, skipping slots that
 // hold no token yet, and starts the two bulk copies of the next one.
 template <int D>
 struct Feeder {
     int it, it_end;       // next item index / end of this worker's items
     int u = 0, ub = 0, uc = 0, head = 0;
+    UnitBatch batch;
     uint32_t n_issued = 0;
     uint32_t ring, bars;  // shared-memory addresses of this warp's slots and barriers
 
@@ -106,21 +144,22 @@ struct Feeder {
                 const DevItem d = a.items[it];
                 ++it;
                 ub = d.unit_begin; uc = d.unit_count; head = d.kv_head; u = 0;
+                batch.load(a, ub, uc, 0, lane);
                 continue;
             }
-            const int4 un = a.units[ub + u];
-            ++u;
-            const int valid = a.node_len[un.y] - un.z;
-            if (valid <= 0) continue;
-            if (un.x < 0 || (int64_t)un.x >= a.pages_per_layer) {  // never read outside the pool
-                if (lane == 0) atomicExch(a.status, -1);
+            const int nxt = batch.next_live(u);
+            if (nxt < 0) {
+                u = batch.base + 32 < uc ? batch.base + 32 : uc;
+                if (u < uc) batch.load(a, ub, uc, u, lane);
                 continue;
             }
+            const int page = __shfl_sync(0xffffffffu, batch.page, nxt - batch.base);
+            u = nxt + 1;
             if (lane == 0) {
                 const uint32_t slot = n_issued % kDepth;
                 const uint32_t bar = bars + slot * 8;
                 const uint32_t dst = ring + slot * 2 * TB;
-                const size_t off = ((size_t)un.x * a.Hkv + head) * TB;
+                const size_t off = ((size_t)page * a.Hkv + head) * TB;
                 mbar_expect_tx(bar, 2 * TB);
                 bulk_g2s(dst, a.k_pool + off, TB, bar);
                 bulk_g2s(dst + TB, a.v_pool + off, TB, bar);
@@ -181,12 +220,17 @@ __device__ __forceinline__ void run_item(const DecodeArgs& a, const DevItem it, 
     const uint32_t k_row = (uint32_t)(k_tok >> 3) * (D / 64) * 1024u + (uint32_t)(k_tok & 7) * 128u;
     const uint32_t v_row = (uint32_t)(v_tok >> 3) * (D / 64) * 1024u + (uint32_t)(v_tok & 7) * 128u;
 
-    for (int u = 0; u < it.unit_count; ++u) {
-        const int4 un = a.units[it.unit_begin + u];
-        int valid = a.node_len[un.y] - un.z;
-        if (valid <= 0) continue;
-        if (un.x < 0 || (int64_t)un.x >= a.pages_per_layer) continue;   // the feeder skipped it too
-        valid = valid > 16 ? 16 : valid;
+    UnitBatch cb;
+    cb.load(a, it.unit_begin, it.unit_count, 0, lane);
+    for (int u = 0; u < it.unit_count;) {
+        const int nxt = cb.next_live(u);
+        if (nxt < 0) {
+            u = cb.base + 32 < it.unit_count ? cb.base + 32 : it.unit_count;
+            if (u < it.unit_count) cb.load(a, it.unit_begin, it.unit_count, u, lane);
+            continue;
+        }
+        const int valid = __shfl_sync(0xffffffffu, cb.valid, nxt - cb.base);
+        u = nxt + 1;
         const uint32_t slot = n_consumed % kDepth;
         const uint32_t parity = (n_consumed / kDepth) & 1u;
         const bool issued = n_consumed < feed.n_issued;

@@ -189,7 +189,13 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         n_runs += tiles * p.num_kv_heads;
         run_units += nu * tiles * p.num_kv_heads;
     }
-    const double target = ((double)run_units + kItemCost * (double)(n_runs + n_workers)) / n_workers;
+    // the target load is re-derived from what is left every time a worker is closed, so rounding
+    // never piles up on the last worker
+    int64_t left_units = run_units, left_runs = n_runs;
+    auto target_for = [&](int32_t workers_left) {
+        return ((double)left_units + kItemCost * (double)(left_runs + workers_left)) / workers_left;
+    };
+    double target = target_for(n_workers);
     t.chunk_pages_used = p.chunk_pages;
     t.worker_off.assign((size_t)n_workers + 1, 0);
     int32_t w = 0;
@@ -203,16 +209,18 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         for (int32_t h = 0; h < p.num_kv_heads; ++h)
             for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile) {
                 int32_t done = 0;
+                --left_runs;
                 while (done < nu) {
-                    if (w < n_workers - 1 && target - load < kItemCost + 1.0) {
+                    if (w < n_workers - 1 && target - load < kItemCost + 0.5) {
                         ++w;
                         t.worker_off[w] = (int32_t)t.items.size();
                         load = 0.0;
+                        target = target_for(n_workers - w);
                     }
                     int32_t take = nu - done;
                     if (w < n_workers - 1) {
                         const double room = target - load - kItemCost;
-                        take = (int32_t)std::min<double>(take, std::max(1.0, std::floor(room)));
+                        take = (int32_t)std::min<double>(take, std::max(1.0, std::floor(room + 0.5)));
                     }
                     take = std::min(take, max_run);
                     Item it;
@@ -228,6 +236,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
                     slots += it.n_leaves_tile;
                     load += take + kItemCost;
                     done += take;
+                    left_units -= take;
                     if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
                 }
             }

@@ -222,3 +222,18 @@ def test_work_decomposition_on_configs(name):
     if name == "cfg5a":
         # the five shared chain steps fuse with the root: 1 shared segment + 128 private ones
         assert st["n_segments"] == 129
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3_ets", "cfg3_diverse", "cfg4", "cfg5b"])
+def test_worker_pieces_are_balanced(name):
+    """The work line is cut into contiguous per-warp pieces of nearly equal cost."""
+    wl = make_workload(name)
+    g = wl.geometry
+    ctx = host_ctx(g.num_q_heads, g.num_kv_heads, g.head_dim, pages=1 << 15, max_path_entries=1 << 14)
+    ctx.tree_build(wl.tree.parent, wl.tree.tokens, wl.tree.leaf_node)
+    w = ctx.work_export()
+    off, item = w["worker_off"], w["item"]
+    assert off[0] == 0 and off[-1] == item.shape[0] and np.all(np.diff(off) >= 0)
+    units = np.array([item[off[i]:off[i + 1], 1].sum() for i in range(len(off) - 1)], dtype=np.float64)
+    cost = units + 2.0 * np.diff(off)
+    assert cost.max() <= cost.mean() * 1.15 + 4.0, (cost.max(), cost.mean())
