@@ -199,6 +199,49 @@ def measured_hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+# ----------------------------------------------------------------------------- ranks
+class RankComm:
+    """The only inter-rank traffic of the benchmark: a barrier and a max-reduce of a scalar.
+    Replicas are independent, so there is no data-path collective."""
+
+    def __init__(self, world: int, device: str):
+        self.world, self.device = world, device
+
+    def barrier(self):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    def max_over_ranks(self, x: float) -> float:
+        if self.world == 1:
+            return x
+        import torch
+        import torch.distributed as dist
+        t = torch.tensor([x], dtype=torch.float64, device=self.device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def all_values(self, x: float):
+        if self.world == 1:
+            return [x]
+        import torch
+        import torch.distributed as dist
+        t = torch.tensor([x], dtype=torch.float64, device=self.device)
+        out = [torch.zeros_like(t) for _ in range(self.world)]
+        dist.all_gather(out, t)
+        return [float(o.item()) for o in out]
+
+
+def replica_value_seed(base_seed: int, rank: int) -> int:
+    """Each replica draws its own K/V/Q values; the tree is the same on every rank."""
+    return base_seed + 7919 * rank
+
+
+def aggregate_value(leaves_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job leaf-queries/s: what all ranks processed in a step over the slowest rank's time."""
+    return world * leaves_per_rank / (ms_per_step / 1000.0)
+
+
 # ----------------------------------------------------------------------------- ours
 def run_ours(args):
     import torch
@@ -216,18 +259,13 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    comm = RankComm(world, device="cuda")
+    barrier, max_over_ranks = comm.barrier, comm.max_over_ranks
 
     wl = make_workload(args.workload)
+    if rank:
+        import dataclasses
+        wl = dataclasses.replace(wl, value_seed=replica_value_seed(wl.value_seed, rank))
     g, tree = wl.geometry, wl.tree
     layers = args.layers or g.num_layers
     K, W = args.steps, args.warmup
@@ -270,7 +308,7 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else {}
     ctx.poll_status()
     ms_step = ms_total / K
-    value = world * L / (ms_step / 1000.0)
+    value = aggregate_value(L, world, ms_step)
 
     # ---- same loop with the attention and merge kernels bracketed by events on their stream
     ctx.set_option(ets.ETS_OPT_TIMING, 1)

@@ -13,7 +13,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_NAME = "libets_b200.so"
-LIB_PATH = os.path.join(HERE, LIB_NAME)
+# ETS_B200_LIBRARY points the binding at another build of the same C ABI (e.g. a debug build)
+LIB_PATH = os.environ.get("ETS_B200_LIBRARY") or os.path.join(HERE, LIB_NAME)
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

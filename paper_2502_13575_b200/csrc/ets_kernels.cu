@@ -1,6 +1,7 @@
 // KV append / read-back, the scalar-FMA node-partial attention kernel and the
 // log-sum-exp merge kernel.
 #include "ets_device.cuh"
+#include "ets_merge.cuh"
 
 namespace ets {
 
@@ -202,57 +203,15 @@ void launch_partial_fma(const DecodeArgs& a, int D, cudaStream_t s) {
 }
 
 // ------------------------------------------------------------------------------------
-// Log-sum-exp merge along each leaf's path.  One warp per (leaf, query head); a lane owns
-// D/32 consecutive features.  With partials (m_j, l_j, o_j) in log2 units:
-//   m* = max_j m_j, l* = sum_j l_j 2^(m_j-m*), out = sum_j o_j 2^(m_j-m*) / l*,
-//   lse = (m* + log2 l*) ln 2.  Empty partials (l_j = 0) are skipped.
+// Log-sum-exp merge along each leaf's path: one warp per (leaf, query head); plenty of warps,
+// because each one is a short chain of dependent loads.
 // ------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(128) lse_merge_kernel(DecodeArgs a) {
-    constexpr int EPL = D / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * 4 + warp;
     if (row >= (int64_t)a.n_leaves * a.Hq) return;
-    const int leaf = (int)(row / a.Hq), head = (int)(row % a.Hq);
-    const int G = a.G, sub = head % G;
-    const int list = leaf * a.Hkv + head / G;
-    const int s0 = a.leaf_slot_off[list], s1 = a.leaf_slot_off[list + 1];
-
-    float ms = -INFINITY;
-    for (int j = s0 + lane; j < s1; j += 32) {
-        const float2 ml = a.part_ml[(size_t)a.leaf_slots[j] * G + sub];
-        if (ml.y > 0.f) ms = fmaxf(ms, ml.x);
-    }
-#pragma unroll
-    for (int x = 16; x > 0; x >>= 1) ms = fmaxf(ms, __shfl_xor_sync(0xffffffffu, ms, x));
-
-    float acc[EPL];
-#pragma unroll
-    for (int j = 0; j < EPL; ++j) acc[j] = 0.f;
-    float ls = 0.f;
-    for (int j = s0; j < s1; ++j) {
-        const size_t prow = (size_t)a.leaf_slots[j] * G + sub;
-        const float2 ml = a.part_ml[prow];
-        if (!(ml.y > 0.f)) continue;
-        const float w = exp2f(ml.x - ms);
-        ls += w * ml.y;
-        const float* po = a.part_o + prow * D + lane * EPL;
-        if constexpr (EPL == 4) {
-            const float4 v = *reinterpret_cast<const float4*>(po);
-            acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
-        } else {
-            const float2 v = *reinterpret_cast<const float2*>(po);
-            acc[0] += w * v.x; acc[1] += w * v.y;
-        }
-    }
-    const float inv = ls > 0.f ? 1.f / ls : 0.f;
-    __nv_bfloat16* op = a.out + (size_t)row * D + lane * EPL;
-#pragma unroll
-    for (int j = 0; j < EPL; j += 2) {
-        __nv_bfloat162 pk = __floats2bfloat162_rn(acc[j] * inv, acc[j + 1] * inv);
-        *reinterpret_cast<__nv_bfloat162*>(op + j) = pk;
-    }
-    if (a.lse && lane == 0) a.lse[row] = ls > 0.f ? (ms + log2f(ls)) * 0.6931471805599453f : -INFINITY;
+    merge_row<D>(a, (int)(row / a.Hq), (int)(row % a.Hq), lane);
 }
 
 void launch_merge(const DecodeArgs& a, int D, cudaStream_t s) {
