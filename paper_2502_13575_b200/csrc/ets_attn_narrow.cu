@@ -59,6 +59,29 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// same copy with an L2 eviction-priority hint
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void st_f32_hint(float* p, float v, uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(v), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void st_f32x2_hint(float2* p, float2 v, uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;" ::"l"(p), "f"(v.x), "f"(v.y), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -133,6 +156,8 @@ template <int D>
 struct Feeder {
     int it, it_end;       // next item index / end of this worker's items
     int u = 0, ub = 0, uc = 0, head = 0;
+    bool reread = false;  // the current item's pages are read again by the next leaf tile
+    uint64_t pol_stream;  // K/V read for the last time goes first when L2 needs room
     UnitBatch batch;
     uint32_t n_issued = 0;
     uint32_t ring, bars;  // shared-memory addresses of this warp's slots and barriers
@@ -145,6 +170,7 @@ struct Feeder {
                 const DevItem d = a.items[it];
                 ++it;
                 ub = d.unit_begin; uc = d.unit_count; head = d.kv_head; u = 0;
+                reread = (d.reserved & 1) != 0;
                 batch.load(a, ub, uc, 0, lane);
                 continue;
             }
@@ -162,8 +188,13 @@ struct Feeder {
                 const uint32_t dst = ring + slot * 2 * TB;
                 const size_t off = ((size_t)page * a.Hkv + head) * TB;
                 mbar_expect_tx(bar, 2 * TB);
-                bulk_g2s(dst, a.k_pool + off, TB, bar);
-                bulk_g2s(dst + TB, a.v_pool + off, TB, bar);
+                if (reread) {
+                    bulk_g2s(dst, a.k_pool + off, TB, bar);
+                    bulk_g2s(dst + TB, a.v_pool + off, TB, bar);
+                } else {
+                    bulk_g2s_hint(dst, a.k_pool + off, TB, bar, pol_stream);
+                    bulk_g2s_hint(dst + TB, a.v_pool + off, TB, bar, pol_stream);
+                }
             }
             ++n_issued;
             return true;
@@ -325,6 +356,7 @@ __device__ __forceinline__ void run_item(const DecodeArgs& a, const DevItem it, 
     }
 
     // partial (m, l, o) of this item, straight from registers
+    const uint64_t pol_keep = policy_evict_last();
 #pragma unroll
     for (int j = 0; j < NT; ++j)
 #pragma unroll
@@ -336,12 +368,13 @@ __device__ __forceinline__ void run_item(const DecodeArgs& a, const DevItem it, 
             const int n = 8 * j + 2 * quad + r;
             if (n < rows) {
                 const size_t prow = (size_t)(it.slot_first + n / G) * G + n % G;
-                if (grp == 0) a.part_ml[prow] = make_float2(m[j][r], ls);
+                // partials are read back by the merge kernel right after: ask L2 to hold on to them
+                if (grp == 0) st_f32x2_hint(a.part_ml + prow, make_float2(m[j][r], ls), pol_keep);
                 float* po = a.part_o + prow * D + grp;
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) {
-                    po[16 * mt] = o[mt][j][r];
-                    po[16 * mt + 8] = o[mt][j][r + 2];
+                    st_f32_hint(po + 16 * mt, o[mt][j][r], pol_keep);
+                    st_f32_hint(po + 16 * mt + 8, o[mt][j][r + 2], pol_keep);
                 }
             }
         }
@@ -362,6 +395,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_partial_narrow_kernel(Dec
     Feeder<D> feed;
     feed.it = i0;
     feed.it_end = i1;
+    feed.pol_stream = policy_evict_first();
     feed.ring = base + (uint32_t)warp * kDepth * 2 * TB;
     feed.bars = base + (uint32_t)kWarps * kDepth * 2 * TB + (uint32_t)warp * kDepth * 8;
     if (lane == 0) {

@@ -231,7 +231,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
                     it.n_leaves_tile = std::min(leaves_per_tile, gn - l0);
                     it.slot_first = (int32_t)slots;
                     it.segment = s;
-                    it.reserved = 0;
+                    it.reserved = (l0 + leaves_per_tile < gn) ? 1 : 0;   // bit 0: the next tile re-reads these pages
                     t.items.push_back(it);
                     slots += it.n_leaves_tile;
                     load += take + kItemCost;
