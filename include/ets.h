@@ -229,7 +229,10 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
 
 /* Tuning and instrumentation knobs; unknown keys give ETS_ERR_INVALID_ARG. */
 #define ETS_OPT_CHUNK_PAGES   1  /* longest page run per work item (0 = no limit); next build    */
-#define ETS_OPT_KERNEL        2  /* 0 tensor-core attention kernel (default), 1 scalar-FMA kernel */
+#define ETS_OPT_KERNEL        2  /* 0 tensor-core attention kernels (default), 1 scalar-FMA kernel;  */
+                                 /* rebuild the tree after changing it                             */
+#define ETS_OPT_WIDE          4  /* 1 (default): query groups above 16 rows use the tcgen05 kernel; */
+                                 /* 0: everything on the narrow kernel.  Applies at the next build. */
 #define ETS_OPT_TIMING        3  /* 1: bracket the attention and merge kernels with events      */
 int32_t ets_set_option(ets_ctx* ctx, int32_t key, int64_t value);
 

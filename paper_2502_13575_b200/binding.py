@@ -27,6 +27,7 @@ ETS_ERR_DEVICE_TIMEOUT = -7
 ETS_OPT_CHUNK_PAGES = 1
 ETS_OPT_KERNEL = 2
 ETS_OPT_TIMING = 3
+ETS_OPT_WIDE = 4
 
 _ERR_NAMES = {
     -1: "ETS_ERR_INVALID_ARG", -2: "ETS_ERR_BAD_TREE", -3: "ETS_ERR_POOL_EXHAUSTED",

@@ -140,6 +140,7 @@ struct ets_ctx {
     // options
     int32_t opt_chunk_pages = 0;
     int32_t opt_kernel = 0;
+    bool opt_wide = true;
     bool opt_timing = false;
     // timing
     std::vector<cudaEvent_t> tev;   // 3 per timed call
@@ -270,6 +271,7 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
             if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->status_host, 64, cudaHostAllocDefault);
             if (e == cudaSuccess) e = cudaMemset(c->ws + c->lay.status, 0, 1024);
             if (e == cudaSuccess) e = ets::narrow_prepare(cfg->head_dim);
+            if (e == cudaSuccess) e = ets::wide_prepare(cfg->head_dim);
         }
         if (e != cudaSuccess) {
             ets_destroy(c);
@@ -313,6 +315,9 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
             if (value < 0 || value > 1) return fail(c, ETS_ERR_INVALID_ARG, "unknown kernel selector");
             c->opt_kernel = (int32_t)value;
             return ETS_OK;
+        case ETS_OPT_WIDE:
+            c->opt_wide = value != 0;
+            return ETS_OK;
         case ETS_OPT_TIMING:
             if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
             c->opt_timing = value != 0;
@@ -328,6 +333,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
     if (!c) return ETS_ERR_INVALID_ARG;
     ets::FlattenParams fp = c->fp;
     fp.chunk_pages = c->opt_chunk_pages;
+    fp.wide_rows = (c->opt_wide && c->opt_kernel == 0) ? 128 : 0;
     ets::Tree next;
     std::string err;
     int32_t rc = ets::tree_build(c->tree, fp, n_nodes, parent, cap_tokens, keep_pages_of, n_leaves, leaf_node,
@@ -507,6 +513,23 @@ int32_t ets_kv_append_host(ets_ctx* c, int32_t layer, int32_t n_items, const int
     return append_impl(c, layer, n_items, node_id, n_new, k_new, v_new, true, (cudaStream_t)cuda_stream);
 }
 
+// The node-partial attention launches for the current tree: wide query groups on the tcgen05
+// kernel, everything else on the narrow kernel (or all of it on the scalar kernel when selected).
+static int32_t launch_attention(ets_ctx* c, const ets::DecodeArgs& a, cudaStream_t s) {
+    const int D = c->cfg.head_dim;
+    const int n_narrow = c->tree.n_narrow_items;
+    const int n_wide = (int)c->tree.items.size() - n_narrow;
+    if (c->opt_kernel == 1) {
+        if (n_wide > 0) return fail(c, ETS_ERR_STATE, "rebuild the tree after changing ETS_OPT_KERNEL");
+        ets::launch_partial_fma(a, D, s);
+        return ETS_OK;
+    }
+    ets::launch_partial_wide(a, D, n_narrow, n_wide, s);
+    if (n_narrow > 0)
+        ets::launch_partial_narrow(a, D, (c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps, s);
+    return ETS_OK;
+}
+
 static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse, cudaStream_t s) {
     const ets::Tree& t = c->tree;
     if (t.n_leaves == 0) return ETS_OK;
@@ -551,8 +574,7 @@ static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, 
         ev = &c->tev[3 * c->timed_calls];
         ETS_CUDA(c, cudaEventRecord(ev[0], s));
     }
-    if (c->opt_kernel == 1) ets::launch_partial_fma(a, c->cfg.head_dim, s);
-    else ets::launch_partial_narrow(a, c->cfg.head_dim, (c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps, s);
+    if (int32_t rc = launch_attention(c, a, s)) return rc;
     if (ev) ETS_CUDA(c, cudaEventRecord(ev[1], s));
     ets::launch_merge(a, c->cfg.head_dim, s);
     if (ev) {
@@ -675,8 +697,7 @@ int32_t ets_tree_attn_decode_static(ets_ctx* c, int32_t layer, const void* q, vo
     a.scale_log2 = c->scale_log2;
     a.worker_off = blob_ptr<int32_t>(c, c->bo.worker_off);
     a.n_workers = c->fp.n_workers;
-    if (c->opt_kernel == 1) ets::launch_partial_fma(a, D, s);
-    else ets::launch_partial_narrow(a, D, (c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps, s);
+    if (int32_t rc = launch_attention(c, a, s)) return rc;
     ets::launch_merge(a, D, s);
     ETS_CUDA(c, cudaGetLastError());
     return ETS_OK;

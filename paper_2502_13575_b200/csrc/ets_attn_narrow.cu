@@ -323,8 +323,10 @@ __device__ __forceinline__ void run_item(const DecodeArgs& a, const DevItem it, 
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
                 const float mn = fmaxf(m[j][r], mx);     // finite: token 0 of the tile is valid
                 const float corr = exp2f(m[j][r] - mn);
-                p[r] = exp2f(sv[r] - mn);
-                p[r + 2] = exp2f(sv[r + 2] - mn);
+                // weights are rounded to bf16 here, so that the row sum and the product use the same
+                // values and the rounding cancels in sum(p v) / sum(p)
+                p[r] = __bfloat162float(__float2bfloat16_rn(exp2f(sv[r] - mn)));
+                p[r + 2] = __bfloat162float(__float2bfloat16_rn(exp2f(sv[r + 2] - mn)));
                 l[j][r] = l[j][r] * corr + p[r] + p[r + 2];
                 m[j][r] = mn;
 #pragma unroll

@@ -1,0 +1,463 @@
+// Node-partial attention for wide query groups (17 .. 128 query rows per work item) on the
+// 5th-generation tensor cores: tcgen05.mma with accumulators in tensor memory.
+//
+// A wide group is where the path really is a dense contraction: one K/V tile serves up to 128
+// query rows, so both products are issued as UMMA instructions with M = 128 (query rows, one per
+// TMEM lane) instead of being re-read once per 16 rows by the narrow kernel.
+//
+// One CTA per work item, six warps:
+//   warp 0      producer: walks the item's page slots, skips empty ones, and brings up to eight
+//               K tiles and eight V tiles (128 tokens) per stage into shared memory with linear
+//               bulk copies; the page image in global memory already is the SWIZZLE_128B operand
+//               layout, so no tensor map is needed.  Also owns the TMEM allocation.
+//   warp 1      MMA issuer: S = Q . K^T   (A = Q from shared memory, K-major; B = K stage, K-major)
+//               then       O += P . V     (A = P from tensor memory;  B = V stage, MN-major).
+//   warps 2-5   softmax: one query row per thread (its TMEM lane); scores in log2 units, online
+//               maximum; when a row's maximum grows, O is rescaled in tensor memory.  (Raising the
+//               reference lazily, only after it is outgrown by 2^8, saves most rescales but leaves
+//               the dominant weight off a power of two, and its bf16 rounding then shows in peaked
+//               rows whose output nearly cancels; the exact policy keeps that weight at 1.)
+// Stages are processed one after another (QK -> softmax -> PV); the ring only lets the copies of
+// the next stage overlap the arithmetic of the current one.
+// Every wait is bounded.  A wait that runs out sets an abort flag that all roles poll, the status
+// word is raised, copies in flight are waited for (again boundedly), TMEM is released, and the CTA
+// returns.
+#include "ets_device.cuh"
+
+namespace ets {
+
+namespace {
+
+constexpr int kWideThreads = 192;
+constexpr int kStageUnits = 8;                 // page slots (16 tokens each) per stage
+constexpr int kStages = 2;
+constexpr uint32_t kSpin = 1u << 22;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
+constexpr float kRescaleThreshold = 0.0f;      // log2 units; see the softmax role
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: SWIZZLE_128B, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128, N given, B either K- or MN-major.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)acc)
+        : "memory");
+}
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)acc)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+        "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+        "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+        "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+        "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+        "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+        "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(v[0]),
+                 "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+struct StageInfo {
+    int32_t n_units;                 // page slots in the stage (0 = end of item)
+    int32_t valid[kStageUnits];      // tokens held by each
+};
+
+struct Shared {
+    uint64_t full[kStages];          // copies of a stage have landed (producer -> MMA warp)
+    uint64_t empty[kStages];         // stage may be overwritten (PV product done -> producer)
+    uint64_t s_ready;                // S = Q K^T is in tensor memory (MMA -> softmax)
+    uint64_t p_ready;                // P is in tensor memory (softmax -> MMA), 4 arrivals
+    uint64_t o_ready;                // O += P V done (MMA -> softmax)
+    uint32_t tmem_base;
+    volatile int32_t abort;
+    StageInfo info[kStages];
+};
+
+// Called by all 32 lanes of a warp together; the answer is the same in every lane, so that the
+// warp-collective tcgen05 instructions that follow are never reached by only part of a warp.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, Shared* sh) {
+    bool ok = false;
+    for (uint32_t i = 0; i < kSpin; ++i) {
+        if (mbar_try_wait(bar, parity)) { ok = true; break; }
+        if ((i & 255u) == 255u && sh->abort) break;
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) sh->abort = 1;
+    return ok;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kWideThreads, 1) attn_partial_wide_kernel(DecodeArgs a, int first_item) {
+    constexpr uint32_t TB = 16 * D * 2;                  // one tile
+    constexpr uint32_t STAGE_HALF = kStageUnits * TB;    // K (or V) part of a stage
+    constexpr int KS = D / 16;                           // k-steps of the QK product
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t q_smem = base;                                     // 128 rows x D bf16
+    const uint32_t ring = base + 128u * D * 2u;                       // kStages x (K half, V half)
+    Shared* sh = reinterpret_cast<Shared*>(base_ptr + 128u * D * 2u + kStages * 2u * STAGE_HALF);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const DevItem it = a.items[first_item + blockIdx.x];
+    const int G = a.G, h = it.kv_head;
+    const int rows = it.n_leaves_tile * G;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
+        mbar_init(smem_u32(&sh->s_ready), 1);
+        mbar_init(smem_u32(&sh->p_ready), 4);
+        mbar_init(smem_u32(&sh->o_ready), 1);
+        sh->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // Q tile: query row r = (leaf r / G of the tile, head h*G + r % G), K-major with the 128-byte swizzle
+    for (int i = threadIdx.x; i < 128 * (D / 8); i += kWideThreads) {
+        const int r = i / (D / 8), c = i % (D / 8);
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (r < rows) {
+            const int leaf = a.node_leaves[it.leaf_list_begin + r / G];
+            v = *reinterpret_cast<const uint4*>(a.q + ((size_t)leaf * a.Hq + h * G + r % G) * D + c * 8);
+        }
+        *reinterpret_cast<uint4*>(base_ptr + tile_offset(D, r, c * 8)) = v;
+    }
+    fence_proxy_async();      // the Q tile was written by ordinary stores and is read by the MMA unit
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+    uint32_t prod_stages = 0;   // producer only: stages whose copies were started
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        int u = 0;
+        for (uint32_t st = 0;; ++st) {
+            const uint32_t s = st % kStages;
+            if (st >= kStages && !wait_or_abort(smem_u32(&sh->empty[s]), ((st / kStages) - 1) & 1u, sh)) break;
+            // gather up to 8 page slots that hold tokens (lane-parallel look-ahead over 32 slots)
+            int n = 0;
+            const uint32_t kdst = ring + s * 2 * STAGE_HALF, vdst = kdst + STAGE_HALF;
+            while (n < kStageUnits && u < it.unit_count) {
+                const int idx = u + lane;
+                int page = 0, valid = 0;
+                if (idx < it.unit_count) {
+                    const int4 un = a.units[it.unit_begin + idx];
+                    valid = a.node_len[un.y] - un.z;
+                    valid = valid < 0 ? 0 : (valid > 16 ? 16 : valid);
+                    if (valid > 0 && (un.x < 0 || (int64_t)un.x >= a.pages_per_layer)) { atomicExch(a.status, -1); valid = 0; }
+                    page = un.x;
+                }
+                uint32_t live = __ballot_sync(0xffffffffu, valid > 0);
+                int consumed = 32;
+                while (live) {
+                    const int src = __ffs(live) - 1;
+                    if (n == kStageUnits) { consumed = src; break; }
+                    live &= live - 1;
+                    const int pg = __shfl_sync(0xffffffffu, page, src);
+                    const int vl = __shfl_sync(0xffffffffu, valid, src);
+                    if (lane == 0) {
+                        sh->info[s].valid[n] = vl;
+                        const size_t off = ((size_t)pg * a.Hkv + h) * TB;
+                        // raise the byte count first; the producer's single arrival comes after the
+                        // last copy of the stage has been started, so the phase cannot end early
+                        asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"(2 * TB) : "memory");
+                        bulk_g2s(kdst + n * TB, a.k_pool + off, TB, smem_u32(&sh->full[s]));
+                        bulk_g2s(vdst + n * TB, a.v_pool + off, TB, smem_u32(&sh->full[s]));
+                    }
+                    ++n;
+                }
+                u += consumed;
+                if (u > it.unit_count) u = it.unit_count;
+            }
+            if (lane == 0) {
+                sh->info[s].n_units = n;                 // n == 0: end marker
+                mbar_arrive(smem_u32(&sh->full[s]));      // publishes the stage info with release semantics
+            }
+            __syncwarp();
+            if (n == 0) break;
+            ++prod_stages;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        const uint32_t idesc_pv = instr_desc(D, true);
+        bool first = true;
+        for (uint32_t st = 0;; ++st) {
+            const uint32_t s = st % kStages;
+            if (!wait_or_abort(smem_u32(&sh->full[s]), (st / kStages) & 1u, sh)) break;
+            const int n = sh->info[s].n_units;
+            if (n == 0) {   // end of item: wake the softmax warps, which then see the same marker
+                if (lane == 0) mbar_arrive(smem_u32(&sh->s_ready));
+                break;
+            }
+            const uint32_t kst = ring + s * 2 * STAGE_HALF, vst = kst + STAGE_HALF;
+            // rows past a page's length hold stale bytes; zero them in V (0 * garbage could be NaN)
+            bool wrote = false;
+            for (int k = 0; k < n; ++k) {
+                const int valid = sh->info[s].valid[k];
+                if (valid < 16) {
+                    for (int i = lane; i < (16 - valid) * (D / 8); i += 32) {
+                        const int t = valid + i / (D / 8), c = i % (D / 8);
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vst + k * TB + tile_offset(D, t, c * 8)), "r"(0u) : "memory");
+                    }
+                    wrote = true;
+                }
+            }
+            if (wrote) fence_proxy_async();
+            __syncwarp();
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t idesc_qk = instr_desc(16u * n, false);
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const uint32_t koff = (uint32_t)(ks >> 2) * 1024u + (uint32_t)(ks & 3) * 32u;
+                    umma_ss(tmem + kColS, smem_desc(q_smem + koff, 16, 1024u * (D / 64)), smem_desc(kst + koff, 16, 1024u * (D / 64)),
+                            idesc_qk, ks > 0);
+                }
+                umma_commit(smem_u32(&sh->s_ready));
+            }
+            __syncwarp();
+            if (!wait_or_abort(smem_u32(&sh->p_ready), st & 1u, sh)) break;
+            tc_fence_after();
+            if (lane == 0) {
+                for (int k = 0; k < n; ++k)
+                    umma_ts(tmem + kColO, tmem + kColP + 8u * k, smem_desc(vst + k * TB, 1024, 1024u * (D / 64)), idesc_pv,
+                            !(first && k == 0));
+                umma_commit(smem_u32(&sh->empty[s]));
+                umma_commit(smem_u32(&sh->o_ready));
+            }
+            first = false;
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax, one row per thread
+        const int row = 32 * (warp & 3) + lane;
+        const uint32_t tlane = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+        float m_ref = -INFINITY, l = 0.f;
+        uint32_t n_stages = 0;
+        bool ok = true;
+        for (uint32_t st = 0;; ++st) {
+            const uint32_t s = st % kStages;
+            if (!wait_or_abort(smem_u32(&sh->s_ready), st & 1u, sh)) { ok = false; break; }
+            // s_ready can only complete after the MMA warp saw full[s]: the stage info is visible
+            const int n = sh->info[s].n_units;
+            if (n == 0) break;   // end marker passed on by the MMA warp
+            tc_fence_after();
+            // pass 1: row maximum over the stage's tokens
+            float mx = -INFINITY;
+            for (int c = 0; c < n; ++c) {
+                float v[16];
+                tmem_ld16(tlane + kColS + 16u * c, v);
+                const int vc = sh->info[s].valid[c];
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (i < vc) mx = fmaxf(mx, v[i]);
+            }
+            mx *= a.scale_log2;
+            // raise the reference (and rescale O, l) when the maximum outgrew it by the threshold
+            const bool need = mx > m_ref + kRescaleThreshold;
+            const bool any_need = __any_sync(0xffffffffu, need);
+            if (any_need) {
+                const float m_new = need ? mx : m_ref;
+                const float f = (m_ref == -INFINITY) ? 0.f : exp2f(m_ref - m_new);
+                if (st > 0) {
+                    // O of the previous stages is final in tensor memory (o_ready was waited for below)
+#pragma unroll 1
+                    for (int c = 0; c < D; c += 32) {
+                        float v[32];
+                        tmem_ld32(tlane + kColO + c, v);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] *= f;
+                        tmem_st32(tlane + kColO + c, v);
+                    }
+                    tmem_wait_st();
+                }
+                l *= f;
+                m_ref = m_new;
+            }
+            // pass 2: P = 2^(s - m_ref), packed bf16 into the A operand of the second product
+            for (int c = 0; c < n; ++c) {
+                float v[16];
+                tmem_ld16(tlane + kColS + 16u * c, v);
+                const int vc = sh->info[s].valid[c];
+                uint32_t pk[8];
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    const float p0 = i < vc ? exp2f(v[i] * a.scale_log2 - m_ref) : 0.f;
+                    const float p1 = i + 1 < vc ? exp2f(v[i + 1] * a.scale_log2 - m_ref) : 0.f;
+                    // the row sum uses the bf16-rounded weights, the same ones the product uses, so the
+                    // rounding cancels in sum(p v) / sum(p)
+                    const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
+                    l += __low2float(pr) + __high2float(pr);
+                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+                }
+                tmem_st8(tlane + kColP + 8u * c, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready));
+            ++n_stages;
+            if (!wait_or_abort(smem_u32(&sh->o_ready), st & 1u, sh)) { ok = false; break; }
+            tc_fence_after();
+        }
+        // epilogue: partial (m_ref, l, O) of this row
+        if (ok && row < rows) {
+            const size_t prow = (size_t)(it.slot_first + row / G) * G + row % G;
+            a.part_ml[prow] = make_float2(m_ref, l);
+        }
+        if (ok) {
+            float* po = a.part_o + ((size_t)(it.slot_first + row / G) * G + row % G) * D;
+#pragma unroll 1
+            for (int c = 0; c < D; c += 32) {
+                float v[32];
+                if (n_stages > 0) tmem_ld32(tlane + kColO + c, v);
+                else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0.f;
+                }
+                if (row < rows) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4*>(po + c + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (sh->abort) {
+        if (threadIdx.x == 0) atomicExch(a.status, -7);
+        // copies that were started still target this CTA's shared memory: give them time to land
+        if (warp == 0) {
+            const uint32_t lo = prod_stages > (uint32_t)kStages ? prod_stages - kStages : 0u;
+            for (uint32_t st = lo; st < prod_stages; ++st) {
+                const uint32_t bar = smem_u32(&sh->full[st % kStages]), par = (st / kStages) & 1u;
+                for (uint32_t i = 0; i < kSpin && !mbar_try_wait(bar, par); ++i) {}
+            }
+        }
+        __syncthreads();
+    }
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+size_t wide_smem_bytes_impl(int D) {
+    return 1024 + 128u * D * 2u + kStages * 2u * kStageUnits * 16u * D * 2u + sizeof(Shared) + 64;
+}
+
+}  // namespace
+
+size_t wide_smem_bytes(int D) { return wide_smem_bytes_impl(D); }
+
+cudaError_t wide_prepare(int D) {
+    if (D == 128)
+        return cudaFuncSetAttribute(attn_partial_wide_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)wide_smem_bytes_impl(128));
+    return cudaFuncSetAttribute(attn_partial_wide_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)wide_smem_bytes_impl(64));
+}
+
+void launch_partial_wide(const DecodeArgs& a, int D, int first_item, int n_wide, cudaStream_t s) {
+    if (n_wide <= 0) return;
+    if (D == 128) attn_partial_wide_kernel<128><<<n_wide, kWideThreads, wide_smem_bytes_impl(128), s>>>(a, first_item);
+    else attn_partial_wide_kernel<64><<<n_wide, kWideThreads, wide_smem_bytes_impl(64), s>>>(a, first_item);
+}
+
+}  // namespace ets

@@ -78,5 +78,8 @@ void launch_merge(const DecodeArgs& a, int D, cudaStream_t s);
 size_t narrow_smem_bytes(int D);
 cudaError_t narrow_prepare(int D);
 void launch_partial_narrow(const DecodeArgs& a, int D, int n_ctas, cudaStream_t s);
+size_t wide_smem_bytes(int D);
+cudaError_t wide_prepare(int D);
+void launch_partial_wide(const DecodeArgs& a, int D, int first_item, int n_wide, cudaStream_t s);
 
 }  // namespace ets

@@ -182,9 +182,10 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     const int32_t max_run = p.chunk_pages > 0 ? p.chunk_pages : INT32_MAX;
     constexpr double kItemCost = 2.0;
     int64_t n_runs = 0, run_units = 0;
+    auto is_wide = [&](int32_t s) { return p.wide_rows > 0 && g[seg_head[s]] * p.gqa > p.rows_per_item; };
     for (int32_t s = 0; s < n_seg; ++s) {
         const int64_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
-        if (nu == 0) continue;
+        if (nu == 0 || is_wide(s)) continue;
         const int64_t tiles = ceil_div(g[seg_head[s]], leaves_per_tile);
         n_runs += tiles * p.num_kv_heads;
         run_units += nu * tiles * p.num_kv_heads;
@@ -203,7 +204,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     int64_t slots = 0;
     for (int32_t s = 0; s < n_seg; ++s) {
         const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
-        if (nu == 0) continue;
+        if (nu == 0 || is_wide(s)) continue;
         const int32_t head_node = seg_head[s];
         const int32_t gn = g[head_node];
         for (int32_t h = 0; h < p.num_kv_heads; ++h)
@@ -242,6 +243,39 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             }
     }
     for (int32_t k = w + 1; k <= n_workers; ++k) t.worker_off[k] = (int32_t)t.items.size();
+    t.n_narrow_items = (int32_t)t.items.size();
+
+    // ---- wide items: segments whose query group exceeds one narrow tile go to the tcgen05 kernel,
+    // one CTA per (piece of the segment, kv head, tile of up to wide_rows query rows)
+    if (p.wide_rows > 0) {
+        const int32_t wide_leaves = std::max(1, p.wide_rows / std::max(1, p.gqa));
+        const int32_t piece = std::max(1, std::min(p.wide_max_units, max_run));
+        for (int32_t s = 0; s < n_seg; ++s) {
+            const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
+            if (nu == 0 || !is_wide(s)) continue;
+            const int32_t head_node = seg_head[s];
+            const int32_t gn = g[head_node];
+            const int32_t n_pieces = ceil_div(nu, piece);
+            for (int32_t pc = 0; pc < n_pieces; ++pc) {
+                const int32_t ub = (int32_t)((int64_t)nu * pc / n_pieces), ue = (int32_t)((int64_t)nu * (pc + 1) / n_pieces);
+                for (int32_t h = 0; h < p.num_kv_heads; ++h)
+                    for (int32_t l0 = 0; l0 < gn; l0 += wide_leaves) {
+                        Item it;
+                        it.unit_begin = seg_unit_off[s] + ub;
+                        it.unit_count = ue - ub;
+                        it.kv_head = h;
+                        it.leaf_list_begin = t.node_leaf_off[head_node] + l0;
+                        it.n_leaves_tile = std::min(wide_leaves, gn - l0);
+                        it.slot_first = (int32_t)slots;
+                        it.segment = s;
+                        it.reserved = (l0 + wide_leaves < gn) ? 1 : 0;
+                        t.items.push_back(it);
+                        slots += it.n_leaves_tile;
+                        if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
+                    }
+            }
+        }
+    }
     t.n_chunks = (int64_t)t.items.size();
     t.n_partial_slots = slots;
     if ((int64_t)t.items.size() > p.max_items) { err = "work items exceed the workspace bound"; return F_EXHAUSTED; }

@@ -23,6 +23,8 @@ struct FlattenParams {
     int64_t max_items = 0;
     int32_t chunk_pages = 0;    // longest run of page slots in one item (0 = unlimited)
     int32_t rows_per_item = 16; // query rows (leaves * gqa) one work item covers
+    int32_t wide_rows = 0;      // query rows one wide (tcgen05) item covers; 0 = no wide items
+    int32_t wide_max_units = 32; // longest page run of a wide item
     int32_t n_workers = 148 * 8; // warps the attention kernel keeps resident; each gets one piece of the work
 };
 
@@ -42,7 +44,8 @@ struct Tree {
     std::vector<int32_t> free_heap;         // min-heap of free page ids (std::greater)
     // work decomposition
     std::vector<int32_t> unit;              // 4 per unit: page, node, tok0, 0
-    std::vector<Item> items;
+    std::vector<Item> items;                // narrow items in worker order, then wide items
+    int32_t n_narrow_items = 0;
     std::vector<int32_t> leaf_slot_off, leaf_slots;   // per (leaf, kv head)
     std::vector<int32_t> worker_off;                  // items of worker w: [worker_off[w], worker_off[w+1])
     int64_t n_segments = 0, n_chunks = 0, n_partial_slots = 0;

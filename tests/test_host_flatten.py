@@ -163,7 +163,7 @@ def _check_work(ctx, tree, cap, hkv, gqa, page=16):
     covered = {}   # (page, head, leaf) -> slot
     for it in item:
         ub, uc, head, lb, nl, slot0, seg, _ = (int(x) for x in it)
-        assert 1 <= nl <= leaves_per_tile and uc >= 1
+        assert 1 <= nl <= max(1, 128 // gqa) and uc >= 1
         leaves = t["node_leaves"][lb:lb + nl].tolist()
         for u in range(ub, ub + uc):
             pg, node, tok0, _z = (int(x) for x in unit[u])
@@ -233,7 +233,9 @@ def test_worker_pieces_are_balanced(name):
     ctx.tree_build(wl.tree.parent, wl.tree.tokens, wl.tree.leaf_node)
     w = ctx.work_export()
     off, item = w["worker_off"], w["item"]
-    assert off[0] == 0 and off[-1] == item.shape[0] and np.all(np.diff(off) >= 0)
+    assert off[0] == 0 and off[-1] <= item.shape[0] and np.all(np.diff(off) >= 0)
+    # items after the last worker piece are the wide ones (tiles of groups with more than 16 query rows)
+    assert np.all(item[:off[-1], 4] * g.gqa <= 16)
     units = np.array([item[off[i]:off[i + 1], 1].sum() for i in range(len(off) - 1)], dtype=np.float64)
     cost = units + 2.0 * np.diff(off)
     assert cost.max() <= cost.mean() * 1.15 + 4.0, (cost.max(), cost.mean())
