@@ -40,6 +40,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (0 = its own)")
     ap.add_argument("--chunk-pages", type=int, default=None)
     ap.add_argument("--kernel", type=int, default=None)
+    ap.add_argument("--wide", type=int, default=None, help="0: no tcgen05 wide-group items")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time budget of the oracle sample")
@@ -271,7 +272,7 @@ def run_ours(args):
     K, W = args.steps, args.warmup
     headroom = K + W + 2
     job = DecodeJob(wl, headroom=headroom, device=local, layers=layers, chunk_pages=args.chunk_pages,
-                    kernel=args.kernel, host_buffers=not args.no_e2e)
+                    kernel=args.kernel, wide=args.wide, host_buffers=not args.no_e2e)
     ctx = job.ctx
     stats = ctx.get_stats()
     L = tree.n_leaves

@@ -231,8 +231,8 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
 #define ETS_OPT_CHUNK_PAGES   1  /* longest page run per work item (0 = no limit); next build    */
 #define ETS_OPT_KERNEL        2  /* 0 tensor-core attention kernels (default), 1 scalar-FMA kernel;  */
                                  /* rebuild the tree after changing it                             */
-#define ETS_OPT_WIDE          4  /* 1 (default): query groups above 16 rows use the tcgen05 kernel; */
-                                 /* 0: everything on the narrow kernel.  Applies at the next build. */
+#define ETS_OPT_WIDE          4  /* smallest query group, in rows (leaves * Hq/Hkv, at least 17), that */
+                                 /* goes to the tcgen05 kernel (default 65); 0: none.  Next build.      */
 #define ETS_OPT_TIMING        3  /* 1: bracket the attention and merge kernels with events      */
 int32_t ets_set_option(ets_ctx* ctx, int32_t key, int64_t value);
 

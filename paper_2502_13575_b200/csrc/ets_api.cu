@@ -137,10 +137,16 @@ struct ets_ctx {
     bool desc_used[kDescSlots] = {};
     int desc_next = 0;
     int32_t* status_host = nullptr;  // pinned, target of the status read-back
+    // second stream on which the wide-group kernel runs beside the narrow kernel
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // options
     int32_t opt_chunk_pages = 0;
     int32_t opt_kernel = 0;
-    bool opt_wide = true;
+    // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256
+    // tree: 65 beats both 17 and "never" (below ~64 rows the per-item latency of the wide kernel
+    // costs more than the re-reads it saves).
+    int32_t opt_wide = 65;
     bool opt_timing = false;
     // timing
     std::vector<cudaEvent_t> tev;   // 3 per timed call
@@ -269,6 +275,9 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
                 if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->desc_ev[i], cudaEventDisableTiming);
             }
             if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->status_host, 64, cudaHostAllocDefault);
+            if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
             if (e == cudaSuccess) e = cudaMemset(c->ws + c->lay.status, 0, 1024);
             if (e == cudaSuccess) e = ets::narrow_prepare(cfg->head_dim);
             if (e == cudaSuccess) e = ets::wide_prepare(cfg->head_dim);
@@ -298,6 +307,9 @@ int32_t ets_destroy(ets_ctx* c) {
             if (c->desc_ev[i]) cudaEventDestroy(c->desc_ev[i]);
         }
         if (c->status_host) cudaFreeHost(c->status_host);
+        if (c->side) cudaStreamDestroy(c->side);
+        if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+        if (c->ev_join) cudaEventDestroy(c->ev_join);
         for (cudaEvent_t e : c->tev) cudaEventDestroy(e);
     }
     delete c;
@@ -316,7 +328,8 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
             c->opt_kernel = (int32_t)value;
             return ETS_OK;
         case ETS_OPT_WIDE:
-            c->opt_wide = value != 0;
+            if (value < 0 || value > 1 << 20) return fail(c, ETS_ERR_INVALID_ARG, "wide threshold out of range");
+            c->opt_wide = (int32_t)value;
             return ETS_OK;
         case ETS_OPT_TIMING:
             if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
@@ -333,7 +346,8 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
     if (!c) return ETS_ERR_INVALID_ARG;
     ets::FlattenParams fp = c->fp;
     fp.chunk_pages = c->opt_chunk_pages;
-    fp.wide_rows = (c->opt_wide && c->opt_kernel == 0) ? 128 : 0;
+    fp.wide_rows = (c->opt_wide > 0 && c->opt_kernel == 0) ? 128 : 0;
+    fp.wide_min_rows = c->opt_wide;
     ets::Tree next;
     std::string err;
     int32_t rc = ets::tree_build(c->tree, fp, n_nodes, parent, cap_tokens, keep_pages_of, n_leaves, leaf_node,
@@ -524,9 +538,21 @@ static int32_t launch_attention(ets_ctx* c, const ets::DecodeArgs& a, cudaStream
         ets::launch_partial_fma(a, D, s);
         return ETS_OK;
     }
-    ets::launch_partial_wide(a, D, n_narrow, n_wide, s);
-    if (n_narrow > 0)
-        ets::launch_partial_narrow(a, D, (c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps, s);
+    const int n_ctas = (c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps;
+    if (n_wide > 0 && n_narrow > 0) {
+        // the two kernels write disjoint partial slots and are sized to share an SM: the wide one
+        // runs on a second stream, forked from and joined back into the caller's stream
+        ETS_CUDA(c, cudaEventRecord(c->ev_fork, s));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+        ets::launch_partial_narrow(a, D, n_ctas, s);
+        ets::launch_partial_wide(a, D, n_narrow, n_wide, c->side);
+        ETS_CUDA(c, cudaEventRecord(c->ev_join, c->side));
+        ETS_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));
+    } else if (n_wide > 0) {
+        ets::launch_partial_wide(a, D, n_narrow, n_wide, s);
+    } else if (n_narrow > 0) {
+        ets::launch_partial_narrow(a, D, n_ctas, s);
+    }
     return ETS_OK;
 }
 

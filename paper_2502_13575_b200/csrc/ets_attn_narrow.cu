@@ -5,7 +5,7 @@
 // bytes in flight, not around arithmetic:
 //   * persistent grid, one CTA per SM, kNarrowWarps independent warps per CTA; a warp is a worker
 //     with its own contiguous, cost-balanced piece of the work line, so no warp waits for another;
-//   * every warp owns a ring of kDepth shared-memory slots; a slot receives one K tile and one V
+//   * every warp owns a ring of kDepth (2) shared-memory slots; a slot receives one K tile and one V
 //     tile (16 tokens x D bf16 each) by two bulk asynchronous copies (TMA engine, linear form) that
 //     complete on the slot's mbarrier; the ring runs ahead across item boundaries;
 //   * a tile is stored in global memory as its shared-memory image (128-byte swizzle), so it lands
@@ -26,7 +26,7 @@ namespace ets {
 namespace {
 
 constexpr int kWarps = kNarrowWarps;
-constexpr int kDepth = 3;
+constexpr int kDepth = 2;   // measured as fast as 3; 2 leaves shared memory for a wide-kernel CTA on the same SM
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -383,11 +383,16 @@ __device__ __forceinline__ void run_item(const DecodeArgs& a, const DevItem it, 
 }
 
 template <int D>
-__global__ void __launch_bounds__(kWarps * 32, 1) attn_partial_narrow_kernel(DecodeArgs a) {
+// 168 registers x 256 threads leave room in the register file for a wide-kernel CTA (96 x 192)
+__global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
     constexpr uint32_t TB = 16 * D * 2;
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (base & 127u) {   // the swizzled tile rows must start on 128-byte boundaries
+        if (threadIdx.x == 0) atomicExch(a.status, -1);
+        return;
+    }
 
     const int worker = blockIdx.x * kWarps + warp;
     if (worker >= a.n_workers) return;
@@ -421,14 +426,22 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_partial_narrow_kernel(Dec
 
 }  // namespace
 
-size_t narrow_smem_bytes(int D) { return (size_t)kWarps * kDepth * 2 * 16 * D * 2 + kWarps * kDepth * 8 + 1024; }
+size_t narrow_smem_bytes(int D) { return (size_t)kWarps * kDepth * 2 * 16 * D * 2 + kWarps * kDepth * 8; }
 
 cudaError_t narrow_prepare(int D) {
-    if (D == 128)
-        return cudaFuncSetAttribute(attn_partial_narrow_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)narrow_smem_bytes(128));
-    return cudaFuncSetAttribute(attn_partial_narrow_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)narrow_smem_bytes(64));
+    // the largest shared-memory carve-out, so that a CTA of the other attention kernel can be
+    // resident on the same SM
+    cudaError_t e;
+    if (D == 128) {
+        e = cudaFuncSetAttribute(attn_partial_narrow_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)narrow_smem_bytes(128));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_partial_narrow_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    } else {
+        e = cudaFuncSetAttribute(attn_partial_narrow_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)narrow_smem_bytes(64));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_partial_narrow_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    }
+    return e;
 }
 
 void launch_partial_narrow(const DecodeArgs& a, int D, int n_ctas, cudaStream_t s) {

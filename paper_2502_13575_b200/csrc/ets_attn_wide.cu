@@ -17,8 +17,9 @@
 //               reference lazily, only after it is outgrown by 2^8, saves most rescales but leaves
 //               the dominant weight off a power of two, and its bf16 rounding then shows in peaked
 //               rows whose output nearly cancels; the exact policy keeps that weight at 1.)
-// Stages are processed one after another (QK -> softmax -> PV); the ring only lets the copies of
-// the next stage overlap the arithmetic of the current one.
+// Stages are processed one after another (QK -> softmax -> PV) and a CTA holds a single stage, so a
+// CTA alone does not saturate anything; it is sized (97 KB of shared memory, 256 TMEM columns) to sit
+// on an SM next to a CTA of the narrow kernel, launched on a second stream, and the two overlap.
 // Every wait is bounded.  A wait that runs out sets an abort flag that all roles poll, the status
 // word is raised, copies in flight are waited for (again boundedly), TMEM is released, and the CTA
 // returns.
@@ -30,10 +31,12 @@ namespace {
 
 constexpr int kWideThreads = 192;
 constexpr int kStageUnits = 8;                 // page slots (16 tokens each) per stage
-constexpr int kStages = 2;
+constexpr int kStages = 1;                     // one 128-token stage: leaves room for a narrow-kernel CTA on the same SM
 constexpr uint32_t kSpin = 1u << 22;
-constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
+constexpr uint32_t kTmemCols = 256;
+// P (bf16, 8 columns per 16 tokens) is written over the S columns it was computed from: chunk c of P
+// covers columns that only hold S chunks <= c/2, which the thread has consumed by then.
+constexpr uint32_t kColS = 0, kColP = 0, kColO = 128;
 constexpr float kRescaleThreshold = 0.0f;      // log2 units; see the softmax role
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -174,18 +177,22 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, Sha
 }
 
 template <int D>
-__global__ void __launch_bounds__(kWideThreads, 1) attn_partial_wide_kernel(DecodeArgs a, int first_item) {
+__global__ void __maxnreg__(96) attn_partial_wide_kernel(DecodeArgs a, int first_item) {
     constexpr uint32_t TB = 16 * D * 2;                  // one tile
     constexpr uint32_t STAGE_HALF = kStageUnits * TB;    // K (or V) part of a stage
     constexpr int KS = D / 16;                           // k-steps of the QK product
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    uint8_t* base_ptr = smem_raw;
     const uint32_t q_smem = base;                                     // 128 rows x D bf16
     const uint32_t ring = base + 128u * D * 2u;                       // kStages x (K half, V half)
     Shared* sh = reinterpret_cast<Shared*>(base_ptr + 128u * D * 2u + kStages * 2u * STAGE_HALF);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (base & 1023u) {   // the swizzled operand layout needs 1024-byte aligned tiles
+        if (threadIdx.x == 0) atomicExch(a.status, -1);
+        return;
+    }
     const DevItem it = a.items[first_item + blockIdx.x];
     const int G = a.G, h = it.kv_head;
     const int rows = it.n_leaves_tile * G;
@@ -204,20 +211,47 @@ __global__ void __launch_bounds__(kWideThreads, 1) attn_partial_wide_kernel(Deco
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // Q tile: query row r = (leaf r / G of the tile, head h*G + r % G), K-major with the 128-byte swizzle
-    for (int i = threadIdx.x; i < 128 * (D / 8); i += kWideThreads) {
-        const int r = i / (D / 8), c = i % (D / 8);
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (r < rows) {
-            const int leaf = a.node_leaves[it.leaf_list_begin + r / G];
-            v = *reinterpret_cast<const uint4*>(a.q + ((size_t)leaf * a.Hq + h * G + r % G) * D + c * 8);
-        }
-        *reinterpret_cast<uint4*>(base_ptr + tile_offset(D, r, c * 8)) = v;
-    }
-    fence_proxy_async();      // the Q tile was written by ordinary stores and is read by the MMA unit
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (warp != 0) {
+        // Q tile: query row r = (leaf r / G of the tile, head h*G + r % G), K-major with the 128-byte
+        // swizzle.  The producer warp is already fetching K/V meanwhile.  Leaf ids are fetched once
+        // per warp and all of a thread's 16-byte loads are issued before the first store, so the
+        // gather costs two memory round trips instead of two per chunk.
+        constexpr int kGatherThreads = kWideThreads - 32;
+        constexpr int kPer = (128 * (D / 8) + kGatherThreads - 1) / kGatherThreads;
+        const int my_leaf = lane < it.n_leaves_tile ? a.node_leaves[it.leaf_list_begin + lane] : 0;
+        const int leaf_hi = (lane + 32 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 32] : 0;
+        const int leaf_h2 = (lane + 64 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 64] : 0;
+        const int leaf_h3 = (lane + 96 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 96] : 0;
+        constexpr int kBatch = 4;   // loads in flight per thread; bounded to keep registers low
+#pragma unroll 1
+        for (int k0 = 0; k0 < kPer; k0 += kBatch) {
+            uint4 v[kBatch];
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                const int i = (int)threadIdx.x - 32 + (k0 + k) * kGatherThreads;
+                const int r = i / (D / 8), c = i % (D / 8);
+                const int lr = r / G;                       // leaf of the tile (up to 128 when G = 1)
+                const int l0 = __shfl_sync(0xffffffffu, my_leaf, lr & 31);
+                const int l1 = __shfl_sync(0xffffffffu, leaf_hi, lr & 31);
+                const int l2 = __shfl_sync(0xffffffffu, leaf_h2, lr & 31);
+                const int l3 = __shfl_sync(0xffffffffu, leaf_h3, lr & 31);
+                const int leaf = lr < 32 ? l0 : (lr < 64 ? l1 : (lr < 96 ? l2 : l3));
+                v[k] = make_uint4(0u, 0u, 0u, 0u);
+                if (i < 128 * (D / 8) && r < rows)
+                    v[k] = __ldg(reinterpret_cast<const uint4*>(a.q + ((size_t)leaf * a.Hq + h * G + r % G) * D + c * 8));
+            }
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                const int i = (int)threadIdx.x - 32 + (k0 + k) * kGatherThreads;
+                if (i < 128 * (D / 8)) *reinterpret_cast<uint4*>(base_ptr + tile_offset(D, i / (D / 8), (i % (D / 8)) * 8)) = v[k];
+            }
+        }
+        fence_proxy_async();      // the Q tile was written by ordinary stores and is read by the MMA unit
+        asm volatile("bar.sync 1, %0;" ::"r"(kWideThreads - 32) : "memory");
+    }
     const uint32_t tmem = sh->tmem_base;
     uint32_t prod_stages = 0;   // producer only: stages whose copies were started
 
@@ -439,7 +473,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) attn_partial_wide_kernel(Deco
 }
 
 size_t wide_smem_bytes_impl(int D) {
-    return 1024 + 128u * D * 2u + kStages * 2u * kStageUnits * 16u * D * 2u + sizeof(Shared) + 64;
+    return 128u * D * 2u + kStages * 2u * kStageUnits * 16u * D * 2u + sizeof(Shared) + 64;
 }
 
 }  // namespace
@@ -447,11 +481,19 @@ size_t wide_smem_bytes_impl(int D) {
 size_t wide_smem_bytes(int D) { return wide_smem_bytes_impl(D); }
 
 cudaError_t wide_prepare(int D) {
-    if (D == 128)
-        return cudaFuncSetAttribute(attn_partial_wide_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)wide_smem_bytes_impl(128));
-    return cudaFuncSetAttribute(attn_partial_wide_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)wide_smem_bytes_impl(64));
+    // the largest shared-memory carve-out, so that a CTA of the other attention kernel can be
+    // resident on the same SM
+    cudaError_t e;
+    if (D == 128) {
+        e = cudaFuncSetAttribute(attn_partial_wide_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wide_smem_bytes_impl(128));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_partial_wide_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    } else {
+        e = cudaFuncSetAttribute(attn_partial_wide_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wide_smem_bytes_impl(64));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_partial_wide_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    }
+    return e;
 }
 
 void launch_partial_wide(const DecodeArgs& a, int D, int first_item, int n_wide, cudaStream_t s) {

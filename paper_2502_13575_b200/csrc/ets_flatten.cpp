@@ -182,7 +182,10 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     const int32_t max_run = p.chunk_pages > 0 ? p.chunk_pages : INT32_MAX;
     constexpr double kItemCost = 2.0;
     int64_t n_runs = 0, run_units = 0;
-    auto is_wide = [&](int32_t s) { return p.wide_rows > 0 && g[seg_head[s]] * p.gqa > p.rows_per_item; };
+    auto is_wide = [&](int32_t s) {
+        const int32_t r = g[seg_head[s]] * p.gqa;
+        return p.wide_rows > 0 && r > p.rows_per_item && r >= p.wide_min_rows;
+    };
     for (int32_t s = 0; s < n_seg; ++s) {
         const int64_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
         if (nu == 0 || is_wide(s)) continue;

@@ -24,6 +24,7 @@ struct FlattenParams {
     int32_t chunk_pages = 0;    // longest run of page slots in one item (0 = unlimited)
     int32_t rows_per_item = 16; // query rows (leaves * gqa) one work item covers
     int32_t wide_rows = 0;      // query rows one wide (tcgen05) item covers; 0 = no wide items
+    int32_t wide_min_rows = 17; // smallest query group (in rows) that is treated as wide
     int32_t wide_max_units = 32; // longest page run of a wide item
     int32_t n_workers = 148 * 8; // warps the attention kernel keeps resident; each gets one piece of the work
 };

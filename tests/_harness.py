@@ -48,7 +48,7 @@ def check_close(gpu_bits, oracle, what=""):
     return float(err.max())
 
 
-def run_and_check(tree, geom, value_seed, *, layers=(0,), qscale=1.0, chunk_pages=None, kernel=None,
+def run_and_check(tree, geom, value_seed, *, layers=(0,), qscale=1.0, chunk_pages=None, kernel=None, wide=None,
                   cap=None, lengths=None, leaves_subset=None, host_api=False, sm_scale=0.0, ctx=None):
     """Build, fill, decode every requested layer, compare with the oracle.  Returns the context."""
     cap = tree.tokens if cap is None else cap
@@ -60,6 +60,8 @@ def run_and_check(tree, geom, value_seed, *, layers=(0,), qscale=1.0, chunk_page
                                sm_scale=sm_scale)
         if kernel is not None:
             ctx.set_option(ets.ETS_OPT_KERNEL, kernel)
+        if wide is not None:
+            ctx.set_option(ets.ETS_OPT_WIDE, wide)
         ctx.tree_build(tree.parent, cap, tree.leaf_node)
     L = tree.n_leaves
     for layer in layers:

@@ -60,19 +60,28 @@ def test_small_configs_full_comparison(name, host_api):
     run_and_check(wl.tree, wl.geometry, wl.value_seed, host_api=host_api)
 
 
+@pytest.mark.parametrize("kernel,wide", [(0, 0), (0, 17), (0, 65), (1, 0)])
+def test_every_kernel_choice_agrees_with_the_oracle(kernel, wide):
+    """Narrow tensor-core kernel only, tcgen05 kernel from 17 rows, from 65 rows, and the scalar kernel."""
+    wl = make_workload("cfg2")
+    run_and_check(wl.tree, wl.geometry, wl.value_seed, kernel=kernel, wide=wide)
+
+
 @pytest.mark.parametrize("name", ["cfg3_diverse", "cfg3_ets", "cfg5a", "cfg5b", "cfg5c"])
-def test_wide_configs_sampled_leaves(name):
+@pytest.mark.parametrize("wide", [17, 65])
+def test_wide_configs_sampled_leaves(name, wide):
     wl = make_workload(name)
     L = wl.tree.n_leaves
     rng = np.random.default_rng(5)
     subset = sorted(set([0, L - 1] + [int(x) for x in rng.integers(0, L, size=6)]))
-    run_and_check(wl.tree, wl.geometry, wl.value_seed, leaves_subset=subset)
+    run_and_check(wl.tree, wl.geometry, wl.value_seed, leaves_subset=subset, wide=wide)
 
 
 @pytest.mark.parametrize("qscale", [4.0, 8.0])
-def test_peaked_softmax(qscale):
+@pytest.mark.parametrize("wide", [17, 65])
+def test_peaked_softmax(qscale, wide):
     wl = make_workload("cfg2")
-    run_and_check(wl.tree, wl.geometry, wl.value_seed, qscale=qscale)
+    run_and_check(wl.tree, wl.geometry, wl.value_seed, qscale=qscale, wide=wide)
 
 
 @pytest.mark.parametrize("chunk_pages", [1, 3])
@@ -133,7 +142,7 @@ def test_random_small_trees_with_edge_cases():
         gqa = int(rng.choice([1, 4, 8]))
         d = int(rng.choice([64, 128]))
         geom = Geometry(hkv * gqa, hkv, d)
-        run_and_check(tree, geom, 1000 + done, cap=tree.tokens, lengths=lengths)
+        run_and_check(tree, geom, 1000 + done, cap=tree.tokens, lengths=lengths, wide=(17 if done % 2 else None))
         done += 1
 
 

@@ -53,7 +53,8 @@ class DecodeJob:
     append of one new token per leaf followed by tree-decode attention."""
 
     def __init__(self, wl: Workload, *, headroom: int, device: int = 0, layers: Optional[int] = None,
-                 chunk_pages: Optional[int] = None, kernel: Optional[int] = None, host_buffers: bool = True):
+                 chunk_pages: Optional[int] = None, kernel: Optional[int] = None, wide: Optional[int] = None,
+                 host_buffers: bool = True):
         import torch
         from paper_2502_13575_b200.runner import context_for_tree
         import paper_2502_13575_b200 as ets
@@ -71,6 +72,8 @@ class DecodeJob:
                                     chunk_pages=chunk_pages, extra_pages=8)
         if kernel is not None:
             self.ctx.set_option(ets.ETS_OPT_KERNEL, kernel)
+        if wide is not None:
+            self.ctx.set_option(ets.ETS_OPT_WIDE, wide)
         self.keep = np.arange(tree.n_nodes, dtype=np.int32)
         self.ctx.tree_build(tree.parent, self.cap, tree.leaf_node)
         # pools
