@@ -141,6 +141,13 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8])
                  "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
                  : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+        "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -177,7 +184,7 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, Sha
 }
 
 template <int D>
-__global__ void __maxnreg__(96) attn_partial_wide_kernel(DecodeArgs a, int first_item) {
+__global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first_item) {
     constexpr uint32_t TB = 16 * D * 2;                  // one tile
     constexpr uint32_t STAGE_HALF = kStageUnits * TB;    // K (or V) part of a stage
     constexpr int KS = D / 16;                           // k-steps of the QK product
@@ -197,24 +204,72 @@ __global__ void __maxnreg__(96) attn_partial_wide_kernel(DecodeArgs a, int first
     const int G = a.G, h = it.kv_head;
     const int rows = it.n_leaves_tile * G;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
-        mbar_init(smem_u32(&sh->s_ready), 1);
-        mbar_init(smem_u32(&sh->p_ready), 4);
-        mbar_init(smem_u32(&sh->o_ready), 1);
-        sh->abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
+    // Producer step: gather up to 8 page slots of the item that hold tokens (lane-parallel look-ahead
+    // over 32 slots), start their copies into stage st % kStages and publish the stage.  Returns the
+    // number of slots (0 = end marker).  Called by all lanes of warp 0.
+    int u = 0;
+    auto produce = [&](uint32_t st) -> int {
+        const uint32_t s = st % kStages;
+        int n = 0;
+        const uint32_t kdst = ring + s * 2 * STAGE_HALF, vdst = kdst + STAGE_HALF;
+        while (n < kStageUnits && u < it.unit_count) {
+            const int idx = u + lane;
+            int page = 0, valid = 0;
+            if (idx < it.unit_count) {
+                const int4 un = a.units[it.unit_begin + idx];
+                valid = a.node_len[un.y] - un.z;
+                valid = valid < 0 ? 0 : (valid > 16 ? 16 : valid);
+                if (valid > 0 && (un.x < 0 || (int64_t)un.x >= a.pages_per_layer)) { atomicExch(a.status, -1); valid = 0; }
+                page = un.x;
+            }
+            uint32_t live = __ballot_sync(0xffffffffu, valid > 0);
+            int consumed = 32;
+            while (live) {
+                const int src = __ffs(live) - 1;
+                if (n == kStageUnits) { consumed = src; break; }
+                live &= live - 1;
+                const int pg = __shfl_sync(0xffffffffu, page, src);
+                const int vl = __shfl_sync(0xffffffffu, valid, src);
+                if (lane == 0) {
+                    sh->info[s].valid[n] = vl;
+                    const size_t off = ((size_t)pg * a.Hkv + h) * TB;
+                    // raise the byte count first; the producer's single arrival comes after the
+                    // last copy of the stage has been started, so the phase cannot end early
+                    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"(2 * TB) : "memory");
+                    bulk_g2s(kdst + n * TB, a.k_pool + off, TB, smem_u32(&sh->full[s]));
+                    bulk_g2s(vdst + n * TB, a.v_pool + off, TB, smem_u32(&sh->full[s]));
+                }
+                ++n;
+            }
+            u += consumed;
+            if (u > it.unit_count) u = it.unit_count;
+        }
+        if (lane == 0) {
+            sh->info[s].n_units = n;                 // n == 0: end marker
+            mbar_arrive(smem_u32(&sh->full[s]));      // publishes the stage info with release semantics
+        }
+        __syncwarp();
+        return n;
+    };
+
+    int n_first = 0;
     if (warp == 0) {
+        if (lane == 0) {
+            for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
+            mbar_init(smem_u32(&sh->s_ready), 1);
+            mbar_init(smem_u32(&sh->p_ready), 4);
+            mbar_init(smem_u32(&sh->o_ready), 1);
+            sh->abort = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
                      "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    if (warp != 0) {
+        // the first stage's copies start before anybody else is ready for them
+        n_first = produce(0);
+    } else {
         // Q tile: query row r = (leaf r / G of the tile, head h*G + r % G), K-major with the 128-byte
         // swizzle.  The producer warp is already fetching K/V meanwhile.  Leaf ids are fetched once
         // per warp and all of a thread's 16-byte loads are issued before the first store, so the
@@ -225,7 +280,7 @@ __global__ void __maxnreg__(96) attn_partial_wide_kernel(DecodeArgs a, int first
         const int leaf_hi = (lane + 32 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 32] : 0;
         const int leaf_h2 = (lane + 64 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 64] : 0;
         const int leaf_h3 = (lane + 96 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 96] : 0;
-        constexpr int kBatch = 4;   // loads in flight per thread; bounded to keep registers low
+        constexpr int kBatch = 7;   // loads in flight per thread; bounded to keep registers low
 #pragma unroll 1
         for (int k0 = 0; k0 < kPer; k0 += kBatch) {
             uint4 v[kBatch];
@@ -250,59 +305,23 @@ __global__ void __maxnreg__(96) attn_partial_wide_kernel(DecodeArgs a, int first
             }
         }
         fence_proxy_async();      // the Q tile was written by ordinary stores and is read by the MMA unit
-        asm volatile("bar.sync 1, %0;" ::"r"(kWideThreads - 32) : "memory");
     }
+    tc_fence_before();
+    asm volatile("bar.sync 1, %0;" ::"r"(kWideThreads) : "memory");   // barriers, TMEM address, Q tile: visible to all
+    tc_fence_after();
     const uint32_t tmem = sh->tmem_base;
     uint32_t prod_stages = 0;   // producer only: stages whose copies were started
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
-        int u = 0;
-        for (uint32_t st = 0;; ++st) {
-            const uint32_t s = st % kStages;
-            if (st >= kStages && !wait_or_abort(smem_u32(&sh->empty[s]), ((st / kStages) - 1) & 1u, sh)) break;
-            // gather up to 8 page slots that hold tokens (lane-parallel look-ahead over 32 slots)
-            int n = 0;
-            const uint32_t kdst = ring + s * 2 * STAGE_HALF, vdst = kdst + STAGE_HALF;
-            while (n < kStageUnits && u < it.unit_count) {
-                const int idx = u + lane;
-                int page = 0, valid = 0;
-                if (idx < it.unit_count) {
-                    const int4 un = a.units[it.unit_begin + idx];
-                    valid = a.node_len[un.y] - un.z;
-                    valid = valid < 0 ? 0 : (valid > 16 ? 16 : valid);
-                    if (valid > 0 && (un.x < 0 || (int64_t)un.x >= a.pages_per_layer)) { atomicExch(a.status, -1); valid = 0; }
-                    page = un.x;
-                }
-                uint32_t live = __ballot_sync(0xffffffffu, valid > 0);
-                int consumed = 32;
-                while (live) {
-                    const int src = __ffs(live) - 1;
-                    if (n == kStageUnits) { consumed = src; break; }
-                    live &= live - 1;
-                    const int pg = __shfl_sync(0xffffffffu, page, src);
-                    const int vl = __shfl_sync(0xffffffffu, valid, src);
-                    if (lane == 0) {
-                        sh->info[s].valid[n] = vl;
-                        const size_t off = ((size_t)pg * a.Hkv + h) * TB;
-                        // raise the byte count first; the producer's single arrival comes after the
-                        // last copy of the stage has been started, so the phase cannot end early
-                        asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"(2 * TB) : "memory");
-                        bulk_g2s(kdst + n * TB, a.k_pool + off, TB, smem_u32(&sh->full[s]));
-                        bulk_g2s(vdst + n * TB, a.v_pool + off, TB, smem_u32(&sh->full[s]));
-                    }
-                    ++n;
-                }
-                u += consumed;
-                if (u > it.unit_count) u = it.unit_count;
+        if (n_first > 0) {
+            prod_stages = 1;
+            for (uint32_t st = 1;; ++st) {
+                const uint32_t s = st % kStages;
+                if (st >= (uint32_t)kStages && !wait_or_abort(smem_u32(&sh->empty[s]), ((st / kStages) - 1) & 1u, sh)) break;
+                if (produce(st) == 0) break;
+                ++prod_stages;
             }
-            if (lane == 0) {
-                sh->info[s].n_units = n;                 // n == 0: end marker
-                mbar_arrive(smem_u32(&sh->full[s]));      // publishes the stage info with release semantics
-            }
-            __syncwarp();
-            if (n == 0) break;
-            ++prod_stages;
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
@@ -369,15 +388,21 @@ __global__ void __maxnreg__(96) attn_partial_wide_kernel(DecodeArgs a, int first
             const int n = sh->info[s].n_units;
             if (n == 0) break;   // end marker passed on by the MMA warp
             tc_fence_after();
-            // pass 1: row maximum over the stage's tokens
+            // pass 1: row maximum over the stage's tokens, two page slots (32 columns) per load; for
+            // an odd count the last load also reads 16 stale S columns, which are masked
             float mx = -INFINITY;
-            for (int c = 0; c < n; ++c) {
-                float v[16];
-                tmem_ld16(tlane + kColS + 16u * c, v);
-                const int vc = sh->info[s].valid[c];
+            for (int c = 0; c < n; c += 2) {
+                float v[32];
+                tmem_ld32(tlane + kColS + 16u * c, v);
+                const int v0 = sh->info[s].valid[c];
+                const int v1 = c + 1 < n ? sh->info[s].valid[c + 1] : 0;
+                float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (i < vc) mx = fmaxf(mx, v[i]);
+                for (int i = 0; i < 16; ++i) {
+                    if (i < v0) m0 = fmaxf(m0, v[i]);
+                    if (i < v1) m1 = fmaxf(m1, v[16 + i]);
+                }
+                mx = fmaxf(mx, fmaxf(m0, m1));
             }
             mx *= a.scale_log2;
             // raise the reference (and rescale O, l) when the maximum outgrew it by the threshold
@@ -401,24 +426,33 @@ __global__ void __maxnreg__(96) attn_partial_wide_kernel(DecodeArgs a, int first
                 l *= f;
                 m_ref = m_new;
             }
-            // pass 2: P = 2^(s - m_ref), packed bf16 into the A operand of the second product
-            for (int c = 0; c < n; ++c) {
-                float v[16];
-                tmem_ld16(tlane + kColS + 16u * c, v);
-                const int vc = sh->info[s].valid[c];
-                uint32_t pk[8];
+            // pass 2: P = 2^(s - m_ref), packed bf16 into the A operand of the second product, two page
+            // slots per step with independent sums.  The row sum uses the bf16-rounded weights, the
+            // same ones the product uses, so the rounding cancels in sum(p v) / sum(p).
+            float l0 = 0.f, l1 = 0.f;
+            const float neg_ref = -m_ref;
+            for (int c = 0; c < n; c += 2) {
+                float v[32];
+                tmem_ld32(tlane + kColS + 16u * c, v);
+                const int v0 = sh->info[s].valid[c];
+                const int v1 = c + 1 < n ? sh->info[s].valid[c + 1] : 0;
+                uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
-                    const float p0 = i < vc ? exp2f(v[i] * a.scale_log2 - m_ref) : 0.f;
-                    const float p1 = i + 1 < vc ? exp2f(v[i + 1] * a.scale_log2 - m_ref) : 0.f;
-                    // the row sum uses the bf16-rounded weights, the same ones the product uses, so the
-                    // rounding cancels in sum(p v) / sum(p)
-                    const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
-                    l += __low2float(pr) + __high2float(pr);
-                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+                    const float a0 = i < v0 ? exp2f(fmaf(v[i], a.scale_log2, neg_ref)) : 0.f;
+                    const float a1 = i + 1 < v0 ? exp2f(fmaf(v[i + 1], a.scale_log2, neg_ref)) : 0.f;
+                    const float b0 = i < v1 ? exp2f(fmaf(v[16 + i], a.scale_log2, neg_ref)) : 0.f;
+                    const float b1 = i + 1 < v1 ? exp2f(fmaf(v[16 + i + 1], a.scale_log2, neg_ref)) : 0.f;
+                    const __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1);
+                    const __nv_bfloat162 pb = __floats2bfloat162_rn(b0, b1);
+                    l0 += __low2float(pa) + __high2float(pa);
+                    l1 += __low2float(pb) + __high2float(pb);
+                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pa);
+                    pk[8 + (i >> 1)] = *reinterpret_cast<const uint32_t*>(&pb);
                 }
-                tmem_st8(tlane + kColP + 8u * c, pk);
+                tmem_st16(tlane + kColP + 8u * c, pk);
             }
+            l += l0 + l1;
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
