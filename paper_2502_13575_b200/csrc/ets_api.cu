@@ -739,7 +739,7 @@ int32_t ets_kv_read_debug(ets_ctx* c, int32_t layer, int32_t node, void* k_out, 
     const int32_t* pages = blob_ptr<int32_t>(c, c->bo.page_ids) + c->tree.node_page_off[node];
     ets::launch_kv_read(c->k_pool + (size_t)layer * c->layer_pool_bytes,
                         c->v_pool + (size_t)layer * c->layer_pool_bytes, pages, c->tree.len[layer][node],
-                        c->cfg.num_kv_heads, c->cfg.head_dim, (__nv_bfloat16*)k_out, (__nv_bfloat16*)v_out,
+                        c->cfg.pages_per_layer, c->cfg.num_kv_heads, c->cfg.head_dim, (__nv_bfloat16*)k_out, (__nv_bfloat16*)v_out,
                         (cudaStream_t)cuda_stream);
     ETS_CUDA(c, cudaGetLastError());
     return ETS_OK;

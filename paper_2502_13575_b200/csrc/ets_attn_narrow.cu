@@ -186,7 +186,7 @@ struct Feeder {
                 const uint32_t slot = n_issued % kDepth;
                 const uint32_t bar = bars + slot * 8;
                 const uint32_t dst = ring + slot * 2 * TB;
-                const size_t off = ((size_t)page * a.Hkv + head) * TB;
+                const size_t off = pool_tile_offset(a.pages_per_layer, page, head, TB);
                 mbar_expect_tx(bar, 2 * TB);
                 if (reread) {
                     bulk_g2s(dst, a.k_pool + off, TB, bar);

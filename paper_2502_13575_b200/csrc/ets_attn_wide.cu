@@ -232,7 +232,7 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                 const int vl = __shfl_sync(0xffffffffu, valid, src);
                 if (lane == 0) {
                     sh->info[s].valid[n] = vl;
-                    const size_t off = ((size_t)pg * a.Hkv + h) * TB;
+                    const size_t off = pool_tile_offset(a.pages_per_layer, pg, h, TB);
                     // raise the byte count first; the producer's single arrival comes after the
                     // last copy of the stage has been started, so the phase cannot end early
                     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"(2 * TB) : "memory");

@@ -26,6 +26,12 @@ __host__ __device__ inline uint32_t tile_offset(int D, int t, int e) {
            ((((uint32_t)(e & 63) >> 3) ^ r) << 4) + (uint32_t)(e & 7) * 2u;
 }
 
+// Byte offset of the (page, kv head) tile inside one layer's pool: [kv head][page][tile].  Pages of a
+// node usually have consecutive ids, so a worker that streams one head of a node reads contiguous memory.
+__host__ __device__ inline size_t pool_tile_offset(int64_t pages_per_layer, int page, int head, size_t tb) {
+    return ((size_t)head * (size_t)pages_per_layer + (size_t)page) * tb;
+}
+
 struct DevItem {
     int32_t unit_begin, unit_count, kv_head, leaf_list_begin;
     int32_t n_leaves_tile, slot_first, segment, reserved;
@@ -72,7 +78,7 @@ struct AppendArgs {
 
 void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_t s);
 void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* page_ids_of_node, int n_tokens,
-                    int Hkv, int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s);
+                    int64_t pages_per_layer, int Hkv, int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s);
 void launch_partial_fma(const DecodeArgs& a, int D, cudaStream_t s);
 void launch_merge(const DecodeArgs& a, int D, cudaStream_t s);
 size_t narrow_smem_bytes(int D);

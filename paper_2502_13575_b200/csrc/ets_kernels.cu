@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
             continue;
         }
         const size_t src = ((size_t)(src_off + t) * a.Hkv + h) * a.D + (size_t)c * 8;
-        const size_t dst = ((size_t)page * a.Hkv + h) * tb + tile_offset(a.D, pos % kPageTokens, c * 8);
+        const size_t dst = pool_tile_offset(a.pages_per_layer, page, h, tb) + tile_offset(a.D, pos % kPageTokens, c * 8);
         *reinterpret_cast<uint4*>(a.k_pool + dst) = *reinterpret_cast<const uint4*>(a.k_new + src);
         *reinterpret_cast<uint4*>(a.v_pool + dst) = *reinterpret_cast<const uint4*>(a.v_new + src);
     }
@@ -60,8 +60,8 @@ void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_
 // Read one node's rows back in token order (debug / tests).
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) kv_read_kernel(const char* k_pool, const char* v_pool,
-                                                      const int32_t* pages, int n_tokens, int Hkv, int D,
-                                                      __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
+                                                      const int32_t* pages, int n_tokens, int64_t pages_per_layer, int Hkv,
+                                                      int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
     const int chunks_per_head = D / 8;
     const int chunks_per_tok = Hkv * chunks_per_head;
     const size_t tb = tile_bytes(D);
@@ -73,20 +73,20 @@ __global__ void __launch_bounds__(256) kv_read_kernel(const char* k_pool, const 
         const int h = ci / chunks_per_head;
         const int c = ci % chunks_per_head;
         const int page = pages[t / kPageTokens];
-        const size_t src = ((size_t)page * Hkv + h) * tb + tile_offset(D, t % kPageTokens, c * 8);
+        const size_t src = pool_tile_offset(pages_per_layer, page, h, tb) + tile_offset(D, t % kPageTokens, c * 8);
         const size_t dst = ((size_t)t * Hkv + h) * D + (size_t)c * 8;
         if (k_out) *reinterpret_cast<uint4*>(k_out + dst) = *reinterpret_cast<const uint4*>(k_pool + src);
         if (v_out) *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(v_pool + src);
     }
 }
 
-void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* pages, int n_tokens, int Hkv,
-                    int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s) {
+void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* pages, int n_tokens,
+                    int64_t pages_per_layer, int Hkv, int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s) {
     if (n_tokens <= 0) return;
     int64_t total = (int64_t)n_tokens * Hkv * (D / 8);
     int blocks = (int)((total + 255) / 256);
     if (blocks > 4096) blocks = 4096;
-    kv_read_kernel<<<blocks, 256, 0, s>>>(k_pool, v_pool, pages, n_tokens, Hkv, D, k_out, v_out);
+    kv_read_kernel<<<blocks, 256, 0, s>>>(k_pool, v_pool, pages, n_tokens, pages_per_layer, Hkv, D, k_out, v_out);
 }
 
 // ------------------------------------------------------------------------------------
@@ -138,8 +138,8 @@ __global__ void __launch_bounds__(kFmaWarps * 32) attn_partial_fma_kernel(Decode
         }
         int valid = a.node_len[un.y] - un.z;
         valid = valid < 0 ? 0 : (valid > kPageTokens ? kPageTokens : valid);
-        const char* kt = a.k_pool + ((size_t)un.x * a.Hkv + h) * tb;
-        const char* vt = a.v_pool + ((size_t)un.x * a.Hkv + h) * tb;
+        const char* kt = a.k_pool + pool_tile_offset(a.pages_per_layer, un.x, h, tb);
+        const char* vt = a.v_pool + pool_tile_offset(a.pages_per_layer, un.x, h, tb);
         for (int t = 0; t < valid; ++t) {
             const uint32_t off = tile_offset(D, t, e0);
             float kf[EPL], vf[EPL];
