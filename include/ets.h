@@ -180,8 +180,8 @@ int32_t ets_get_node_len(const ets_ctx* ctx, int32_t layer, int32_t* node_len);
  *   out  bf16 [n_leaves, num_q_heads, head_dim]   (fp32 result rounded to nearest even)
  *   lse  fp32 [n_leaves, num_q_heads], natural log; nullable
  * DEVICE pointers for ets_tree_attn_decode; HOST pointers for ets_tree_attn_decode_host, which
- * copies q in and out/lse back on the same stream (the results are valid once the stream has
- * passed the call).  A leaf whose path holds no token yields zeros and lse = -inf.
+ * copies q in and out/lse back on library streams ordered after cuda_stream's work so far (the
+ * results are valid once cuda_stream has passed the call; see ETS_OPT_HOST_PIPELINE for the relaxed form).  A leaf whose path holds no token yields zeros and lse = -inf.
  * Errors: ETS_ERR_STATE (no tree), ETS_ERR_INVALID_ARG, ETS_ERR_CUDA.
  */
 int32_t ets_tree_attn_decode(ets_ctx* ctx, int32_t layer, const void* q, void* out, float* lse,
@@ -233,8 +233,21 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
                                  /* rebuild the tree after changing it                             */
 #define ETS_OPT_WIDE          4  /* smallest query group, in rows (leaves * Hq/Hkv, at least 17), that */
                                  /* goes to the tcgen05 kernel (default 65); 0: none.  Next build.      */
+#define ETS_OPT_HOST_PIPELINE 6  /* 1: the *_host calls return without making cuda_stream wait for   */
+                                 /* them, so the copies of one call overlap the kernels of the next;   */
+                                 /* results are valid after ets_host_join + synchronising that stream;  */
+                                 /* the calls are ordered after cuda_stream's work only as of the first */
+                                 /* *_host call following a join                                        */
 #define ETS_OPT_TIMING        3  /* 1: bracket the attention and merge kernels with events      */
 int32_t ets_set_option(ets_ctx* ctx, int32_t key, int64_t value);
+
+/*
+ * With ETS_OPT_HOST_PIPELINE on: makes cuda_stream wait for every ets_kv_append_host /
+ * ets_tree_attn_decode_host call issued so far (their kernels and their copies back to the host).
+ * Any other device-side call on the context (tree build, device-pointer append/decode, status poll)
+ * joins implicitly first.  Without the option every *_host call joins by itself.
+ */
+int32_t ets_host_join(ets_ctx* ctx, void* cuda_stream);
 
 /* With ETS_OPT_TIMING on: waits for the recorded events, returns and clears the sums. */
 int32_t ets_timing_read(ets_ctx* ctx, double* attn_ms, double* merge_ms, int64_t* n_calls);

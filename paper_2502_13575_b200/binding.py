@@ -28,6 +28,7 @@ ETS_OPT_CHUNK_PAGES = 1
 ETS_OPT_KERNEL = 2
 ETS_OPT_TIMING = 3
 ETS_OPT_WIDE = 4
+ETS_OPT_HOST_PIPELINE = 6
 
 _ERR_NAMES = {
     -1: "ETS_ERR_INVALID_ARG", -2: "ETS_ERR_BAD_TREE", -3: "ETS_ERR_POOL_EXHAUSTED",
@@ -97,6 +98,7 @@ _SIGNATURES = {
     "ets_kv_read_debug": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_get_stats": (C.c_int32, [C.c_void_p, C.POINTER(ets_stats)]),
     "ets_set_option": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int64]),
+    "ets_host_join": (C.c_int32, [C.c_void_p, C.c_void_p]),
     "ets_timing_read": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "ets_poll_status": (C.c_int32, [C.c_void_p, C.c_void_p]),
     "ets_last_error": (C.c_char_p, [C.c_void_p]),
@@ -122,11 +124,14 @@ lib = _load()
 
 
 def _i32(a) -> np.ndarray:
+    if isinstance(a, np.ndarray) and a.dtype == np.int32 and a.flags["C_CONTIGUOUS"]:
+        return a
     return np.ascontiguousarray(a, dtype=np.int32)
 
 
 def _p(a: Optional[np.ndarray]):
-    return None if a is None else a.ctypes.data_as(_I32P)
+    # a raw address converts faster than numpy's ctypes view and is accepted for POINTER arguments
+    return None if a is None else C.cast(a.__array_interface__["data"][0], _I32P)
 
 
 def _dev_ptr(t) -> Optional[int]:
@@ -291,6 +296,9 @@ class EtsContext:
 
     def set_option(self, key: int, value: int):
         self._check(lib.ets_set_option(self._h, key, value))
+
+    def host_join(self, stream=None):
+        self._check(lib.ets_host_join(self._h, _stream_ptr(stream)))
 
     def timing_read(self):
         a, m, n = C.c_double(), C.c_double(), C.c_int64()

@@ -29,7 +29,8 @@ struct Layout {  // byte offsets inside the workspace
     size_t blob, blob_cap;
     size_t desc, desc_slot_bytes;
     size_t part_ml, part_o;
-    size_t q_stage, out_stage, lse_stage, k_stage, v_stage;
+    size_t q_stage, out_stage, lse_stage, k_stage, v_stage;   // two of each, *_stride bytes apart
+    size_t q_stride, lse_stride, kv_stride;
     size_t status;
     size_t total;
     int64_t max_partial_slots, max_items, max_units;
@@ -89,17 +90,20 @@ Layout make_layout(const ets_config* c) {
     size_t off = 0;
     L.blob = off; off += L.blob_cap;
     L.desc_slot_bytes = align_up((size_t)c->max_nodes * 16, 256);
-    L.desc = off; off += align_up(L.desc_slot_bytes * kDescSlots, A);
+    L.desc = off; off += align_up(L.desc_slot_bytes * (kDescSlots + 1), A);   // ring + the cached list
     const size_t rows = (size_t)L.max_partial_slots * gqa;
     L.part_ml = off; off += align_up(rows * 8, A);
     L.part_o = off; off += align_up(rows * c->head_dim * 4, A);
     const size_t qbytes = (size_t)c->max_leaves * c->num_q_heads * c->head_dim * 2;
-    L.q_stage = off; off += align_up(qbytes, A);
-    L.out_stage = off; off += align_up(qbytes, A);
-    L.lse_stage = off; off += align_up((size_t)c->max_leaves * c->num_q_heads * 4, A);
+    L.q_stride = align_up(qbytes, A);
+    L.lse_stride = align_up((size_t)c->max_leaves * c->num_q_heads * 4, A);
+    L.q_stage = off; off += 2 * L.q_stride;
+    L.out_stage = off; off += 2 * L.q_stride;
+    L.lse_stage = off; off += 2 * L.lse_stride;
     const size_t kvb = (size_t)L.max_append_tokens * c->num_kv_heads * c->head_dim * 2;
-    L.k_stage = off; off += align_up(kvb, A);
-    L.v_stage = off; off += align_up(kvb, A);
+    L.kv_stride = align_up(kvb, A);
+    L.k_stage = off; off += 2 * L.kv_stride;
+    L.v_stage = off; off += 2 * L.kv_stride;
     L.status = off; off += A;
     L.total = off;
     return L;
@@ -136,7 +140,24 @@ struct ets_ctx {
     cudaEvent_t desc_ev[kDescSlots] = {};
     bool desc_used[kDescSlots] = {};
     int desc_next = 0;
+    // descriptors of the last short append (at most 8 tokens per node) stay on the device: a decode loop
+    // repeats the same (node, count) list for every layer and step
+    std::vector<int32_t> cache_nodes, cache_nnew;
+    bool cache_valid = false;
+    cudaStream_t cache_stream = nullptr;
+    cudaEvent_t cache_ev = nullptr;
+    bool host_epoch_open = false;   // pipelined host calls: entry ordering already established
     int32_t* status_host = nullptr;  // pinned, target of the status read-back
+    // host-buffer entry points: copies in, kernels and copies out run on three library streams so that
+    // the transfers of one call overlap the kernels of its neighbours; staging areas alternate
+    cudaStream_t st_in = nullptr, st_comp = nullptr, st_out = nullptr;
+    cudaEvent_t ev_entry = nullptr, ev_q_in[2] = {}, ev_q_free[2] = {}, ev_comp[2] = {}, ev_out_free[2] = {};
+    cudaEvent_t ev_kv_in[2] = {}, ev_kv_free[2] = {};
+    bool q_used[2] = {false, false}, out_used[2] = {false, false}, kv_used[2] = {false, false};
+    uint64_t n_host_decode = 0, n_host_append = 0;
+    bool opt_host_pipeline = false;   // host-buffer calls do not make the caller's stream wait; ets_host_join does
+    bool host_pending = false;        // host-buffer work that the caller's stream has not been joined with yet
+    cudaEvent_t ev_join_comp = nullptr, ev_join_out = nullptr;
     // second stream on which the wide-group kernel runs beside the narrow kernel
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -212,6 +233,8 @@ const T* blob_ptr(const ets_ctx* c, size_t off) { return reinterpret_cast<const 
 
 extern "C" {
 
+static int32_t host_join(ets_ctx* c, cudaStream_t s);
+
 const char* ets_version(void) { return "ets-b200 0.1"; }
 
 const char* ets_last_error(const ets_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
@@ -276,6 +299,16 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
             }
             if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->status_host, 64, cudaHostAllocDefault);
             if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->st_in, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->st_comp, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->st_out, cudaStreamNonBlocking);
+            {
+                cudaEvent_t* evs[] = {&c->cache_ev, &c->ev_join_comp, &c->ev_join_out, &c->ev_entry, &c->ev_q_in[0], &c->ev_q_in[1], &c->ev_q_free[0], &c->ev_q_free[1],
+                                      &c->ev_comp[0], &c->ev_comp[1], &c->ev_out_free[0], &c->ev_out_free[1],
+                                      &c->ev_kv_in[0], &c->ev_kv_in[1], &c->ev_kv_free[0], &c->ev_kv_free[1]};
+                for (cudaEvent_t* ev : evs)
+                    if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+            }
             if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
             if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
             if (e == cudaSuccess) e = cudaMemset(c->ws + c->lay.status, 0, 1024);
@@ -308,6 +341,16 @@ int32_t ets_destroy(ets_ctx* c) {
         }
         if (c->status_host) cudaFreeHost(c->status_host);
         if (c->side) cudaStreamDestroy(c->side);
+        if (c->st_in) cudaStreamDestroy(c->st_in);
+        if (c->st_comp) cudaStreamDestroy(c->st_comp);
+        if (c->st_out) cudaStreamDestroy(c->st_out);
+        {
+            cudaEvent_t evs[] = {c->cache_ev, c->ev_join_comp, c->ev_join_out, c->ev_entry, c->ev_q_in[0], c->ev_q_in[1], c->ev_q_free[0], c->ev_q_free[1], c->ev_comp[0],
+                                 c->ev_comp[1], c->ev_out_free[0], c->ev_out_free[1], c->ev_kv_in[0], c->ev_kv_in[1],
+                                 c->ev_kv_free[0], c->ev_kv_free[1]};
+            for (cudaEvent_t ev : evs)
+                if (ev) cudaEventDestroy(ev);
+        }
         if (c->ev_fork) cudaEventDestroy(c->ev_fork);
         if (c->ev_join) cudaEventDestroy(c->ev_join);
         for (cudaEvent_t e : c->tev) cudaEventDestroy(e);
@@ -326,6 +369,10 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
         case ETS_OPT_KERNEL:
             if (value < 0 || value > 1) return fail(c, ETS_ERR_INVALID_ARG, "unknown kernel selector");
             c->opt_kernel = (int32_t)value;
+            return ETS_OK;
+        case ETS_OPT_HOST_PIPELINE:
+            if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+            c->opt_host_pipeline = value != 0;
             return ETS_OK;
         case ETS_OPT_WIDE:
             if (value < 0 || value > 1 << 20) return fail(c, ETS_ERR_INVALID_ARG, "wide threshold out of range");
@@ -360,6 +407,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
     if (!c->host_only) {
         cudaStream_t s = (cudaStream_t)cuda_stream;
         ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+        if (int32_t jrc = host_join(c, s)) return jrc;   // pipelined host-buffer calls still read the old tables
         const int i = c->stage_next;
         if (c->stage_used[i]) ETS_CUDA(c, cudaEventSynchronize(c->stage_ev[i]));
         pack_blob(c, next, bo, c->stage_host[i]);
@@ -443,6 +491,18 @@ int32_t ets_get_stats(const ets_ctx* c, ets_stats* o) {
     return ETS_OK;
 }
 
+// Make `s` wait for every host-buffer call issued so far (kernels and copies back).
+static int32_t host_join(ets_ctx* c, cudaStream_t s) {
+    if (!c->host_pending) return ETS_OK;
+    ETS_CUDA(c, cudaEventRecord(c->ev_join_comp, c->st_comp));
+    ETS_CUDA(c, cudaEventRecord(c->ev_join_out, c->st_out));
+    ETS_CUDA(c, cudaStreamWaitEvent(s, c->ev_join_comp, 0));
+    ETS_CUDA(c, cudaStreamWaitEvent(s, c->ev_join_out, 0));
+    c->host_pending = false;
+    c->host_epoch_open = false;
+    return ETS_OK;
+}
+
 static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int32_t* node_id,
                            const int32_t* n_new, const void* k_new, const void* v_new, bool host_src,
                            cudaStream_t s) {
@@ -474,27 +534,71 @@ static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int
     if (host_src && total > c->lay.max_append_tokens)
         return fail(c, ETS_ERR_POOL_EXHAUSTED, "more tokens than max_append_tokens in a host append");
     ETS_CUDA(c, cudaSetDevice(c->cfg.device));
-    const int slot = c->desc_next;
-    if (c->desc_used[slot]) ETS_CUDA(c, cudaEventSynchronize(c->desc_ev[slot]));
-    int4* d = c->desc_host[slot];
-    int32_t src = 0;
-    for (int32_t i = 0; i < n_items; ++i) {
-        d[i] = make_int4(node_id[i], len[node_id[i]], n_new[i], src);
-        src += n_new[i];
+    const cudaStream_t user = s;
+    const int hb = (int)(c->n_host_append & 1u);
+    if (!host_src) {
+        if (int32_t jrc = host_join(c, s)) return jrc;
     }
-    char* desc_dev = c->ws + c->lay.desc + (size_t)slot * c->lay.desc_slot_bytes;
-    ETS_CUDA(c, cudaMemcpyAsync(desc_dev, d, (size_t)n_items * 16, cudaMemcpyHostToDevice, s));
-    ETS_CUDA(c, cudaEventRecord(c->desc_ev[slot], s));
-    c->desc_used[slot] = true;
-    c->desc_next = (slot + 1) % kDescSlots;
+    if (host_src) {
+        // copy in on the library's input stream into the staging area that is free, run the kernel on
+        // the library's compute stream; the caller's stream only waits for the result at the end
+        const size_t bytes = (size_t)total * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
+        if (!c->host_epoch_open) {
+            ETS_CUDA(c, cudaEventRecord(c->ev_entry, user));
+            ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_entry, 0));
+            ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_entry, 0));
+            c->host_epoch_open = c->opt_host_pipeline;
+        }
+        if (c->kv_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_kv_free[hb], 0));
+        ETS_CUDA(c, cudaMemcpyAsync(c->ws + c->lay.k_stage + hb * c->lay.kv_stride, k_new, bytes, cudaMemcpyHostToDevice, c->st_in));
+        ETS_CUDA(c, cudaMemcpyAsync(c->ws + c->lay.v_stage + hb * c->lay.kv_stride, v_new, bytes, cudaMemcpyHostToDevice, c->st_in));
+        ETS_CUDA(c, cudaEventRecord(c->ev_kv_in[hb], c->st_in));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_kv_in[hb], 0));
+        s = c->st_comp;
+    }
+    char* desc_dev = nullptr;
+    const bool cacheable = max_new <= 8;   // one block per item: the kernel may read the start itself
+    const bool hit = cacheable && c->cache_valid && (int32_t)c->cache_nodes.size() == n_items &&
+                     std::memcmp(c->cache_nodes.data(), node_id, (size_t)n_items * 4) == 0 &&
+                     std::memcmp(c->cache_nnew.data(), n_new, (size_t)n_items * 4) == 0;
+    if (hit) {
+        desc_dev = c->ws + c->lay.desc + (size_t)kDescSlots * c->lay.desc_slot_bytes;
+        if (c->cache_stream != s) {   // the list was uploaded on another stream: order after it
+            ETS_CUDA(c, cudaStreamWaitEvent(s, c->cache_ev, 0));
+        }
+    } else {
+        const int slot = c->desc_next;
+        if (c->desc_used[slot]) ETS_CUDA(c, cudaEventSynchronize(c->desc_ev[slot]));
+        int4* d = c->desc_host[slot];
+        int32_t src = 0;
+        for (int32_t i = 0; i < n_items; ++i) {
+            d[i] = make_int4(node_id[i], cacheable ? -1 : len[node_id[i]], n_new[i], src);
+            src += n_new[i];
+        }
+        const int dev_slot = cacheable ? kDescSlots : slot;
+        desc_dev = c->ws + c->lay.desc + (size_t)dev_slot * c->lay.desc_slot_bytes;
+        if (cacheable && c->cache_valid && c->cache_stream != s) {
+            // a kernel on the other stream may still read the cached list we are about to replace
+            ETS_CUDA(c, cudaEventRecord(c->cache_ev, c->cache_stream));
+            ETS_CUDA(c, cudaStreamWaitEvent(s, c->cache_ev, 0));
+        }
+        ETS_CUDA(c, cudaMemcpyAsync(desc_dev, d, (size_t)n_items * 16, cudaMemcpyHostToDevice, s));
+        ETS_CUDA(c, cudaEventRecord(c->desc_ev[slot], s));
+        c->desc_used[slot] = true;
+        c->desc_next = (slot + 1) % kDescSlots;
+        if (cacheable) {
+            ETS_CUDA(c, cudaEventRecord(c->cache_ev, s));
+            c->cache_nodes.assign(node_id, node_id + n_items);
+            c->cache_nnew.assign(n_new, n_new + n_items);
+            c->cache_valid = true;
+            c->cache_stream = s;
+        }
+    }
     const void* ksrc = k_new;
     const void* vsrc = v_new;
     if (host_src) {
-        const size_t bytes = (size_t)total * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
-        ETS_CUDA(c, cudaMemcpyAsync(c->ws + c->lay.k_stage, k_new, bytes, cudaMemcpyHostToDevice, s));
-        ETS_CUDA(c, cudaMemcpyAsync(c->ws + c->lay.v_stage, v_new, bytes, cudaMemcpyHostToDevice, s));
-        ksrc = c->ws + c->lay.k_stage;
-        vsrc = c->ws + c->lay.v_stage;
+        ksrc = c->ws + c->lay.k_stage + hb * c->lay.kv_stride;
+        vsrc = c->ws + c->lay.v_stage + hb * c->lay.kv_stride;
     }
     ets::AppendArgs a{};
     a.desc = reinterpret_cast<const int4*>(desc_dev);
@@ -513,6 +617,13 @@ static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int
     a.D = c->cfg.head_dim;
     ets::launch_kv_append(a, n_items, max_new, s);
     ETS_CUDA(c, cudaGetLastError());
+    if (host_src) {
+        ETS_CUDA(c, cudaEventRecord(c->ev_kv_free[hb], c->st_comp));
+        if (c->opt_host_pipeline) c->host_pending = true;
+        else ETS_CUDA(c, cudaStreamWaitEvent(user, c->ev_kv_free[hb], 0));   // the caller's stream sees the append
+        c->kv_used[hb] = true;
+        ++c->n_host_append;
+    }
     for (int32_t i = 0; i < n_items; ++i) len[node_id[i]] += n_new[i];
     return ETS_OK;
 }
@@ -624,6 +735,7 @@ int32_t ets_tree_attn_decode(ets_ctx* c, int32_t layer, const void* q, void* out
     if (int32_t rc = decode_check(c, layer, q, out)) return rc;
     if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, ETS_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
     ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    if (int32_t jrc = host_join(c, (cudaStream_t)cuda_stream)) return jrc;
     return decode_impl(c, layer, q, out, lse, (cudaStream_t)cuda_stream);
 }
 
@@ -635,13 +747,35 @@ int32_t ets_tree_attn_decode_host(ets_ctx* c, int32_t layer, const void* q, void
     const size_t rows = (size_t)c->tree.n_leaves * c->cfg.num_q_heads;
     const size_t qbytes = rows * c->cfg.head_dim * 2;
     if (rows == 0) return ETS_OK;
-    char* qd = c->ws + c->lay.q_stage;
-    char* od = c->ws + c->lay.out_stage;
-    float* ld = reinterpret_cast<float*>(c->ws + c->lay.lse_stage);
-    ETS_CUDA(c, cudaMemcpyAsync(qd, q, qbytes, cudaMemcpyHostToDevice, s));
-    if (int32_t rc = decode_impl(c, layer, qd, od, lse ? ld : nullptr, s)) return rc;
-    ETS_CUDA(c, cudaMemcpyAsync(out, od, qbytes, cudaMemcpyDeviceToHost, s));
-    if (lse) ETS_CUDA(c, cudaMemcpyAsync(lse, ld, rows * 4, cudaMemcpyDeviceToHost, s));
+    // Three library streams: q goes in on one, the kernels run on the second, out/lse come back on the
+    // third; the staging areas alternate between calls, so the copies of one call overlap the kernels of
+    // the next.  The caller's stream waits for this call's copy-out, which keeps the contract that the
+    // results are valid once that stream has passed the call.
+    const int hb = (int)(c->n_host_decode & 1u);
+    char* qd = c->ws + c->lay.q_stage + hb * c->lay.q_stride;
+    char* od = c->ws + c->lay.out_stage + hb * c->lay.q_stride;
+    float* ld = reinterpret_cast<float*>(c->ws + c->lay.lse_stage + hb * c->lay.lse_stride);
+    if (!c->host_epoch_open) {
+        ETS_CUDA(c, cudaEventRecord(c->ev_entry, s));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_entry, 0));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_entry, 0));
+        c->host_epoch_open = c->opt_host_pipeline;
+    }
+    if (c->q_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_q_free[hb], 0));
+    ETS_CUDA(c, cudaMemcpyAsync(qd, q, qbytes, cudaMemcpyHostToDevice, c->st_in));
+    ETS_CUDA(c, cudaEventRecord(c->ev_q_in[hb], c->st_in));
+    ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_q_in[hb], 0));
+    if (c->out_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_out_free[hb], 0));
+    if (int32_t rc = decode_impl(c, layer, qd, od, lse ? ld : nullptr, c->st_comp)) return rc;
+    ETS_CUDA(c, cudaEventRecord(c->ev_q_free[hb], c->st_comp));   // kernels done: q staging reusable, out ready
+    ETS_CUDA(c, cudaStreamWaitEvent(c->st_out, c->ev_q_free[hb], 0));
+    ETS_CUDA(c, cudaMemcpyAsync(out, od, qbytes, cudaMemcpyDeviceToHost, c->st_out));
+    if (lse) ETS_CUDA(c, cudaMemcpyAsync(lse, ld, rows * 4, cudaMemcpyDeviceToHost, c->st_out));
+    ETS_CUDA(c, cudaEventRecord(c->ev_out_free[hb], c->st_out));
+    if (c->opt_host_pipeline) c->host_pending = true;
+    else ETS_CUDA(c, cudaStreamWaitEvent(s, c->ev_out_free[hb], 0));
+    c->q_used[hb] = c->out_used[hb] = true;
+    ++c->n_host_decode;
     return ETS_OK;
 }
 
@@ -745,6 +879,13 @@ int32_t ets_kv_read_debug(ets_ctx* c, int32_t layer, int32_t node, void* k_out, 
     return ETS_OK;
 }
 
+int32_t ets_host_join(ets_ctx* c, void* cuda_stream) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    return host_join(c, (cudaStream_t)cuda_stream);
+}
+
 int32_t ets_timing_read(ets_ctx* c, double* attn_ms, double* merge_ms, int64_t* n_calls) {
     if (!c || !attn_ms || !merge_ms || !n_calls) return ETS_ERR_INVALID_ARG;
     if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
@@ -770,6 +911,7 @@ int32_t ets_poll_status(ets_ctx* c, void* cuda_stream) {
     if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
     cudaStream_t s = (cudaStream_t)cuda_stream;
     ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    if (int32_t jrc = host_join(c, s)) return jrc;
     ETS_CUDA(c, cudaMemcpyAsync(c->status_host, c->ws + c->lay.status, 4, cudaMemcpyDeviceToHost, s));
     ETS_CUDA(c, cudaMemsetAsync(c->ws + c->lay.status, 0, 4, s));
     ETS_CUDA(c, cudaStreamSynchronize(s));

@@ -13,13 +13,18 @@ constexpr int kAppendTokPerBlock = 8;
 
 __global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
     const int4 d = a.desc[blockIdx.y];
-    const int node = d.x, start = d.y, n_new = d.z, src_off = d.w;
+    const int node = d.x, n_new = d.z, src_off = d.w;
     const int t0 = blockIdx.x * kAppendTokPerBlock;
     if (t0 >= n_new) return;
     if (node < 0 || node >= a.n_nodes) {
         if (threadIdx.x == 0) atomicExch(a.status, -1);
         return;
     }
+    // a negative start means "append at the node's current length" (used when one block covers the
+    // whole item, so nobody reads the length after it has been advanced); __syncthreads orders the
+    // read before thread 0's update at the end
+    const int start = d.y >= 0 ? d.y : a.node_len[node];
+    __syncthreads();
     const int chunks_per_head = a.D / 8;
     const int chunks_per_tok = a.Hkv * chunks_per_head;
     const int n_tok = min(kAppendTokPerBlock, n_new - t0);

@@ -99,6 +99,7 @@ class DecodeJob:
         self.leaf_nodes = tree.leaf_node.astype(np.int32)
         self.ones = np.ones(L, np.int32)
         if host_buffers:
+            self.ctx.set_option(ets.ETS_OPT_HOST_PIPELINE, 1)
             self.q_h = torch.from_numpy(qb.view(np.int16).copy()).pin_memory()
             self.newk_h = torch.from_numpy(nk.view(np.int16).copy()).pin_memory()
             self.newv_h = torch.from_numpy(nv.view(np.int16).copy()).pin_memory()
@@ -124,16 +125,33 @@ class DecodeJob:
         self.ctx.tree_build(t.parent, self.cap, t.leaf_node, keep_pages_of=self.keep)
         self.steps_done = 0
 
+    def _pointers(self):
+        """Raw addresses of the per-layer inputs and outputs, computed once: the step loop then costs
+        two C calls per layer and no tensor slicing."""
+        if getattr(self, "_ptrs", None) is None:
+            L = self.layers
+            p = {"q": [self.q[l].data_ptr() for l in range(L)], "out": [self.out[l].data_ptr() for l in range(L)],
+                 "nk": [self.newk[l].data_ptr() for l in range(L)], "nv": [self.newv[l].data_ptr() for l in range(L)]}
+            if hasattr(self, "q_h"):
+                p.update({"q_h": [self.q_h[l].data_ptr() for l in range(L)],
+                          "out_h": [self.out_h[l].data_ptr() for l in range(L)],
+                          "nk_h": [self.newk_h[l].data_ptr() for l in range(L)],
+                          "nv_h": [self.newv_h[l].data_ptr() for l in range(L)]})
+            self._ptrs = p
+        return self._ptrs
+
     def step(self):
         """Device-resident inputs: flatten + (append, attend) for every layer; all asynchronous."""
         if self.steps_done >= self.headroom:
             raise RuntimeError("step budget of this job exhausted; call reset_lengths()")
         t = self.wl.tree
         c = self.ctx
-        c.tree_build(t.parent, self.cap, t.leaf_node, keep_pages_of=self.keep)
+        p = self._pointers()
+        stream = self.torch.cuda.current_stream().cuda_stream
+        c.tree_build(t.parent, self.cap, t.leaf_node, keep_pages_of=self.keep, stream=stream)
         for layer in range(self.layers):
-            c.kv_append(layer, self.leaf_nodes, self.ones, self.newk[layer], self.newv[layer])
-            c.tree_attn_decode(layer, self.q[layer], self.out[layer], None)
+            c.kv_append(layer, self.leaf_nodes, self.ones, p["nk"][layer], p["nv"][layer], stream=stream)
+            c.tree_attn_decode(layer, p["q"][layer], p["out"][layer], None, stream=stream)
         self.steps_done += 1
 
     def step_host(self):
@@ -143,10 +161,13 @@ class DecodeJob:
             raise RuntimeError("step budget of this job exhausted; call reset_lengths()")
         t = self.wl.tree
         c = self.ctx
-        c.tree_build(t.parent, self.cap, t.leaf_node, keep_pages_of=self.keep)
+        p = self._pointers()
+        stream = self.torch.cuda.current_stream().cuda_stream
+        c.tree_build(t.parent, self.cap, t.leaf_node, keep_pages_of=self.keep, stream=stream)
         for layer in range(self.layers):
-            c.kv_append_host(layer, self.leaf_nodes, self.ones, self.newk_h[layer], self.newv_h[layer])
-            c.tree_attn_decode_host(layer, self.q_h[layer], self.out_h[layer], None)
+            c.kv_append_host(layer, self.leaf_nodes, self.ones, p["nk_h"][layer], p["nv_h"][layer], stream=stream)
+            c.tree_attn_decode_host(layer, p["q_h"][layer], p["out_h"][layer], None, stream=stream)
+        c.host_join(stream=stream)   # the step's results are complete once this stream has passed here
         self.steps_done += 1
 
     # ---- what the oracle needs for a sample of leaves
