@@ -4,6 +4,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -283,6 +284,10 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
     c->fp.max_partial_slots = c->lay.max_partial_slots;
     c->fp.max_items = c->lay.max_items;
     c->fp.rows_per_item = 16;
+    // the cost model's weights can be overridden for tuning runs
+    if (const char* e = std::getenv("ETS_COST_ITEM")) c->fp.cost_item = std::atof(e);
+    if (const char* e = std::getenv("ETS_COST_ROWS16")) c->fp.cost_rows16 = std::atof(e);
+    if (const char* e = std::getenv("ETS_COST_REREAD")) c->fp.cost_reread = std::atof(e);
     if (!host_only) {
         cudaError_t e = cudaSetDevice(cfg->device);
         cudaDeviceProp prop{};

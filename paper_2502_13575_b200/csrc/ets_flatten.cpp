@@ -180,24 +180,33 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     const int32_t leaves_per_tile = std::max(1, p.rows_per_item / std::max(1, p.gqa));
     const int32_t n_workers = std::max(1, p.n_workers);
     const int32_t max_run = p.chunk_pages > 0 ? p.chunk_pages : INT32_MAX;
-    constexpr double kItemCost = 2.0;
-    int64_t n_runs = 0, run_units = 0;
+    const double kItemCost = p.cost_item;
     auto is_wide = [&](int32_t s) {
         const int32_t r = g[seg_head[s]] * p.gqa;
         return p.wide_rows > 0 && r > p.rows_per_item && r >= p.wide_min_rows;
     };
+    // weight of one page slot of the tile starting at leaf l0 of a group of gn leaves
+    auto unit_weight = [&](int32_t gn, int32_t l0) {
+        const int32_t rows = std::min(leaves_per_tile, gn - l0) * p.gqa;
+        return (rows > 8 ? p.cost_rows16 : 1.0) * (l0 > 0 ? p.cost_reread : 1.0);
+    };
+    int64_t n_runs = 0;
+    double run_cost = 0.0;
     for (int32_t s = 0; s < n_seg; ++s) {
         const int64_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
         if (nu == 0 || is_wide(s)) continue;
-        const int64_t tiles = ceil_div(g[seg_head[s]], leaves_per_tile);
-        n_runs += tiles * p.num_kv_heads;
-        run_units += nu * tiles * p.num_kv_heads;
+        const int32_t gn = g[seg_head[s]];
+        for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile) {
+            n_runs += p.num_kv_heads;
+            run_cost += (double)nu * unit_weight(gn, l0) * p.num_kv_heads;
+        }
     }
     // the target load is re-derived from what is left every time a worker is closed, so rounding
     // never piles up on the last worker
-    int64_t left_units = run_units, left_runs = n_runs;
+    double left_cost = run_cost;
+    int64_t left_runs = n_runs;
     auto target_for = [&](int32_t workers_left) {
-        return ((double)left_units + kItemCost * (double)(left_runs + workers_left)) / workers_left;
+        return (std::max(left_cost, 0.0) + kItemCost * (double)(left_runs + workers_left)) / workers_left;
     };
     double target = target_for(n_workers);
     t.chunk_pages_used = p.chunk_pages;
@@ -212,10 +221,11 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         const int32_t gn = g[head_node];
         for (int32_t h = 0; h < p.num_kv_heads; ++h)
             for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile) {
+                const double uw = unit_weight(gn, l0);
                 int32_t done = 0;
                 --left_runs;
                 while (done < nu) {
-                    if (w < n_workers - 1 && target - load < kItemCost + 0.5) {
+                    if (w < n_workers - 1 && target - load < kItemCost + 0.5 * uw) {
                         ++w;
                         t.worker_off[w] = (int32_t)t.items.size();
                         load = 0.0;
@@ -223,7 +233,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
                     }
                     int32_t take = nu - done;
                     if (w < n_workers - 1) {
-                        const double room = target - load - kItemCost;
+                        const double room = (target - load - kItemCost) / uw;
                         take = (int32_t)std::min<double>(take, std::max(1.0, std::floor(room + 0.5)));
                     }
                     take = std::min(take, max_run);
@@ -238,9 +248,9 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
                     it.reserved = (l0 + leaves_per_tile < gn) ? 1 : 0;   // bit 0: the next tile re-reads these pages
                     t.items.push_back(it);
                     slots += it.n_leaves_tile;
-                    load += take + kItemCost;
+                    load += take * uw + kItemCost;
                     done += take;
-                    left_units -= take;
+                    left_cost -= take * uw;
                     if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
                 }
             }
@@ -252,7 +262,21 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     // one CTA per (piece of the segment, kv head, tile of up to wide_rows query rows)
     if (p.wide_rows > 0) {
         const int32_t wide_leaves = std::max(1, p.wide_rows / std::max(1, p.gqa));
-        const int32_t piece = std::max(1, std::min(p.wide_max_units, max_run));
+        // Piece length: long pieces amortise a CTA's fixed cost (TMEM allocation, Q tile, epilogue) over
+        // several stages, short ones spread a small amount of wide work over more SMs.  Start long and
+        // halve while the wide kernel would launch fewer CTAs than there are SMs.
+        const int32_t n_sm = std::max(1, n_workers / 8);
+        auto wide_ctas = [&](int32_t piece_len) {
+            int64_t n = 0;
+            for (int32_t s = 0; s < n_seg; ++s) {
+                const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
+                if (nu == 0 || !is_wide(s)) continue;
+                n += (int64_t)ceil_div(nu, piece_len) * p.num_kv_heads * ceil_div(g[seg_head[s]], wide_leaves);
+            }
+            return n;
+        };
+        int32_t piece = std::max(1, std::min(p.wide_max_units, max_run));
+        while (piece > 8 && wide_ctas(piece) < n_sm) piece = std::max(8, piece / 2);
         for (int32_t s = 0; s < n_seg; ++s) {
             const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
             if (nu == 0 || !is_wide(s)) continue;

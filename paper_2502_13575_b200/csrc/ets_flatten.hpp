@@ -23,6 +23,11 @@ struct FlattenParams {
     int64_t max_items = 0;
     int32_t chunk_pages = 0;    // longest run of page slots in one item (0 = unlimited)
     int32_t rows_per_item = 16; // query rows (leaves * gqa) one work item covers
+    // cost model of the narrow kernel's work line, in units of one first-read page slot of a tile of
+    // at most 8 query rows
+    double cost_item = 2.0;      // opening an item (Q fragments, partial stores)
+    double cost_rows16 = 1.2;    // factor for tiles of 9..16 query rows (two MMA column tiles); measured
+    double cost_reread = 1.0;    // factor for second and later leaf tiles (their pages come from L2)
     int32_t wide_rows = 0;      // query rows one wide (tcgen05) item covers; 0 = no wide items
     int32_t wide_min_rows = 17; // smallest query group (in rows) that is treated as wide
     int32_t wide_max_units = 32; // longest page run of a wide item
