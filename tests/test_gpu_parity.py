@@ -243,3 +243,88 @@ def test_decode_loop_appends_one_token_per_leaf():
         ref, _ = tree_decode_attention(tree.parent, lengths, tree.leaf_node, full_k, full_v, qb, 8, 2)
         check_close(dev_to_bits(out), ref, f"step {step}")
     ctx.poll_status()
+
+
+def test_append_descriptor_reuse_and_long_appends():
+    """Short appends (at most 8 tokens per node) keep their (node, count) list on the device and read the
+    start position from the device-side lengths; longer ones carry the start in the descriptor.  Mix
+    both, change the list in between, and read everything back."""
+    g = Geometry(8, 2, 128)
+    tree = Tree(np.array([-1, 0, 0, 1], np.int32), np.array([60, 50, 40, 30], np.int32), np.array([2, 3], np.int32))
+    ctx = context_for_tree(8, 2, 128, tree.parent, tree.tokens, tree.leaf_node)
+    ctx.tree_build(tree.parent, tree.tokens, tree.leaf_node)
+    full_k, full_v = [], []
+    for n in range(4):
+        k, v = node_kv_bits(31, n, int(tree.tokens[n]), 2, 128)
+        full_k.append(k)
+        full_v.append(v)
+    pos = [0, 0, 0, 0]
+
+    def push(nodes, counts):
+        k = np.concatenate([full_k[n][pos[n]:pos[n] + c] for n, c in zip(nodes, counts)])
+        v = np.concatenate([full_v[n][pos[n]:pos[n] + c] for n, c in zip(nodes, counts)])
+        ctx.kv_append(0, nodes, counts, bits_to_dev(k), bits_to_dev(v))
+        for n, c in zip(nodes, counts):
+            pos[n] += c
+
+    push([0, 1, 2, 3], [3, 1, 2, 8])      # short: uploaded and cached
+    push([0, 1, 2, 3], [3, 1, 2, 8])      # same list: reused
+    push([0, 1, 2, 3], [3, 1, 2, 8])
+    push([2, 0], [1, 5])                  # different list: replaced
+    push([2, 0], [1, 5])
+    push([0, 1, 2, 3], [20, 9, 11, 3])    # long: start positions travel with the descriptors
+    push([2, 0], [1, 5])                  # the cached list is still valid
+    push([1, 3], [7, 3])
+    torch.cuda.synchronize()
+    assert ctx.get_node_len(0).tolist() == pos
+    for n in range(4):
+        kb, vb = _read_node(ctx, 0, n, pos[n], g)
+        assert np.array_equal(kb, full_k[n][:pos[n]]) and np.array_equal(vb, full_v[n][:pos[n]])
+    ctx.poll_status()
+
+
+def test_pipelined_host_calls_match_device_calls():
+    """With ETS_OPT_HOST_PIPELINE the *_host calls return without joining; after ets_host_join and a
+    synchronisation the host buffers hold the same bytes the device-pointer calls produce."""
+    wl = make_workload("cfg2")
+    g, tree = wl.geometry, wl.tree
+    cap = tree.tokens.copy()
+    cap[tree.leaf_node] += 6
+    results = {}
+    for mode in ("device", "host"):
+        ctx = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, tree.parent, cap, tree.leaf_node,
+                               num_layers=3)
+        ctx.tree_build(tree.parent, cap, tree.leaf_node)
+        for layer in range(3):
+            ks, vs = node_values(tree, g, wl.value_seed, layer)
+            fill_layer(ctx, layer, ks, vs)
+        if mode == "host":
+            ctx.set_option(ets.ETS_OPT_HOST_PIPELINE, 1)
+        from workloads import query_bits
+        outs = []
+        L = tree.n_leaves
+        newk = node_kv_bits(wl.value_seed + 9, 0, 6 * L, g.num_kv_heads, g.head_dim)[0].reshape(6, L, g.num_kv_heads, g.head_dim)
+        for step in range(4):
+            for layer in range(3):
+                qb = query_bits(wl.value_seed + step, layer, L, g.num_q_heads, g.head_dim)
+                kn = np.ascontiguousarray(newk[step])
+                if mode == "device":
+                    ctx.kv_append(layer, tree.leaf_node, [1] * L, bits_to_dev(kn), bits_to_dev(kn))
+                    q = bits_to_dev(qb)
+                    out = torch.empty_like(q)
+                    ctx.tree_attn_decode(layer, q, out, None)
+                    outs.append(out)
+                else:
+                    k_h = torch.from_numpy(kn.view(np.int16)).pin_memory()
+                    q_h = torch.from_numpy(qb.view(np.int16)).pin_memory()
+                    out_h = torch.empty_like(q_h).pin_memory()
+                    ctx.kv_append_host(layer, tree.leaf_node, [1] * L, k_h, k_h)
+                    ctx.tree_attn_decode_host(layer, q_h, out_h, None)
+                    outs.append((out_h, k_h, q_h))
+        if mode == "host":
+            ctx.host_join()
+        torch.cuda.synchronize()
+        ctx.poll_status()
+        results[mode] = [dev_to_bits(o) if mode == "device" else o[0].numpy().view(np.uint16).copy() for o in outs]
+    for a, b in zip(results["device"], results["host"]):
+        assert np.array_equal(a, b)
