@@ -130,15 +130,18 @@ int32_t ets_tree_export(const ets_ctx* ctx, ets_tables_host* out);
 /*
  * The private work decomposition, exported for invariant checks only (its content is an
  * implementation choice and may change): runs of chained nodes with one query group are
- * fused into segments; the line of all (segment, kv head, leaf tile) page-slot runs is cut into
- * equal-cost pieces, one per resident warp of the attention kernel; a work item is one run or
- * the part of a run inside one piece.
+ * fused into segments; the page slots of a segment are cut into pieces, and a work item is one
+ * (piece, kv head, leaf tile).  Items of narrow query groups (at most 16 rows) come first and form a
+ * queue ordered longest piece first: resident warp w of the attention kernel takes item w and then
+ * claims the following items one at a time.  Items of wide groups follow, one CTA each.
  *   unit[n_units*4]     per page slot: page id, node, first token index within the node, 0
  *   item[n_items*8]     unit_begin, unit_count, kv_head, leaf_list_begin (into node_leaves),
- *                       n_leaves_in_tile, partial_slot_of_first_leaf, segment id, 0
+ *                       n_leaves_in_tile, partial_slot_of_first_leaf, segment id, flags
  *   leaf_slot_off[n_leaves*num_kv_heads+1], leaf_slots[n_leaf_slots]
  *                       partial slots to merge per (leaf, kv head)
- *   worker_off[n_workers+1]   items of resident warp w: [worker_off[w], worker_off[w+1])
+ *   worker_off[n_workers+1]   first item of resident warp w: [worker_off[w], worker_off[w+1]), one
+ *                       item or none; worker_off[n_workers] is also the number of narrow items
+ *                       when that is below n_workers
  */
 typedef struct ets_work_host {
     int64_t n_units, n_items, n_leaf_slots, n_partial_slots, n_workers;
@@ -224,6 +227,7 @@ typedef struct ets_stats {
     int64_t pages_used, pages_free;
     int64_t n_segments, n_chunks, n_items, n_units, n_partial_slots;
     int64_t attended_tokens;    /* current tokens of nodes that have a leaf below them       */
+    int64_t n_narrow_items;     /* items of narrow query groups (the first ones in the list) */
 } ets_stats;
 int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
 

@@ -78,7 +78,7 @@ class ets_stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_nodes", "n_leaves", "unique_tokens", "unique_kv_bytes", "path_tokens", "pages_used",
         "pages_free", "n_segments", "n_chunks", "n_items", "n_units", "n_partial_slots",
-        "attended_tokens")]
+        "attended_tokens", "n_narrow_items")]
 
 
 # every symbol include/ets.h declares, with its C signature

@@ -2,6 +2,7 @@
 // launches.  No torch types, no exceptions across the boundary.
 #include "../../include/ets.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -68,11 +69,11 @@ Layout make_layout(const ets_config* c) {
     Layout L{};
     const int64_t path_pages = (int64_t)c->max_leaves * ((c->max_path_tokens + c->page_size - 1) / c->page_size) +
                                c->max_path_entries;
-    // a partial slot belongs to one (item, leaf); items are (segment piece, kv head, leaf tile), and
-    // each worker boundary can split one more item
+    // a partial slot belongs to one (item, leaf); items are (piece of a segment, kv head, leaf tile).  The
+    // builder picks the piece length and falls back to longer pieces when a choice would not fit here.
     const int gqa = c->num_q_heads / c->num_kv_heads;
-    L.max_partial_slots = (c->max_path_entries + (path_pages + 7) / 8) * c->num_kv_heads +
-                          (int64_t)kMaxWorkers * (16 / gqa > 0 ? 16 / gqa : 1);
+    L.max_partial_slots = (c->max_path_entries + (path_pages + 3) / 4) * c->num_kv_heads +
+                          (int64_t)kMaxWorkers * 4 * (16 / gqa > 0 ? 16 / gqa : 1);
     L.max_items = L.max_partial_slots;
     L.max_units = c->pages_per_layer;
     L.max_append_tokens = c->max_append_tokens > 0 ? c->max_append_tokens : c->max_leaves;
@@ -84,7 +85,6 @@ Layout make_layout(const ets_config* c) {
     blob += align_up((size_t)c->pages_per_layer * 4, 256);          // page_ids
     blob += align_up((size_t)c->max_path_entries * 4, 256);         // node_leaves
     blob += align_up(((size_t)c->max_leaves * c->num_kv_heads + 1) * 4, 256);  // leaf_slot_off
-    blob += align_up(((size_t)kMaxWorkers + 1) * 4, 256);           // worker_off
     blob += align_up((size_t)L.max_partial_slots * 4, 256);         // leaf_slots
     blob += align_up((size_t)c->num_layers * c->max_nodes * 4, 256);  // node_len
     L.blob_cap = align_up(blob, A);
@@ -111,7 +111,7 @@ Layout make_layout(const ets_config* c) {
 }
 
 struct BlobOffsets {  // offsets of the packed tables of the current tree inside the device blob
-    size_t units, items, node_page_off, page_ids, node_leaves, leaf_slot_off, leaf_slots, worker_off, node_len, total;
+    size_t units, items, node_page_off, page_ids, node_leaves, leaf_slot_off, leaf_slots, node_len, total;
     int32_t len_stride;
 };
 
@@ -206,7 +206,6 @@ BlobOffsets pack_offsets(const ets_ctx* c, const ets::Tree& t) {
     b.node_leaves = take(t.node_leaves.size() * 4);
     b.leaf_slot_off = take(t.leaf_slot_off.size() * 4);
     b.leaf_slots = take(t.leaf_slots.size() * 4);
-    b.worker_off = take(t.worker_off.size() * 4);
     b.len_stride = t.n_nodes > 0 ? t.n_nodes : 1;
     b.node_len = take((size_t)c->cfg.num_layers * b.len_stride * 4);
     b.total = off;
@@ -222,7 +221,6 @@ void pack_blob(const ets_ctx* c, const ets::Tree& t, const BlobOffsets& b, char*
     put(b.node_leaves, t.node_leaves.data(), t.node_leaves.size() * 4);
     put(b.leaf_slot_off, t.leaf_slot_off.data(), t.leaf_slot_off.size() * 4);
     put(b.leaf_slots, t.leaf_slots.data(), t.leaf_slots.size() * 4);
-    put(b.worker_off, t.worker_off.data(), t.worker_off.size() * 4);
     for (int l = 0; l < c->cfg.num_layers; ++l)
         put(b.node_len + (size_t)l * b.len_stride * 4, t.len[l].data(), t.len[l].size() * 4);
 }
@@ -288,6 +286,7 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
     if (const char* e = std::getenv("ETS_COST_ITEM")) c->fp.cost_item = std::atof(e);
     if (const char* e = std::getenv("ETS_COST_ROWS16")) c->fp.cost_rows16 = std::atof(e);
     if (const char* e = std::getenv("ETS_COST_REREAD")) c->fp.cost_reread = std::atof(e);
+    if (const char* e = std::getenv("ETS_TAIL_PAGES")) c->fp.tail_pages = std::atoi(e);
     if (!host_only) {
         cudaError_t e = cudaSetDevice(cfg->device);
         cudaDeviceProp prop{};
@@ -493,6 +492,7 @@ int32_t ets_get_stats(const ets_ctx* c, ets_stats* o) {
     o->n_items = (int64_t)t.items.size();
     o->n_units = (int64_t)t.unit.size() / 4;
     o->n_partial_slots = t.n_partial_slots;
+    o->n_narrow_items = t.n_narrow_items;
     return ETS_OK;
 }
 
@@ -654,7 +654,9 @@ static int32_t launch_attention(ets_ctx* c, const ets::DecodeArgs& a, cudaStream
         ets::launch_partial_fma(a, D, s);
         return ETS_OK;
     }
-    const int n_ctas = (c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps;
+    // one CTA per SM; fewer when there are fewer narrow items than resident warps
+    const int n_ctas = std::min((c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps,
+                                (n_narrow + ets::kNarrowWarps - 1) / ets::kNarrowWarps);
     if (n_wide > 0 && n_narrow > 0) {
         // the two kernels write disjoint partial slots and are sized to share an SM: the wide one
         // runs on a second stream, forked from and joined back into the caller's stream
@@ -672,9 +674,10 @@ static int32_t launch_attention(ets_ctx* c, const ets::DecodeArgs& a, cudaStream
     return ETS_OK;
 }
 
-static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse, cudaStream_t s) {
+// Everything a decode launch reads, for the current tree and one layer.
+static ets::DecodeArgs decode_args(const ets_ctx* c, int32_t layer, const void* q, void* out, float* lse,
+                                   float2* part_ml, float* part_o) {
     const ets::Tree& t = c->tree;
-    if (t.n_leaves == 0) return ETS_OK;
     ets::DecodeArgs a{};
     a.units = blob_ptr<int4>(c, c->bo.units);
     a.items = blob_ptr<ets::DevItem>(c, c->bo.items);
@@ -687,10 +690,12 @@ static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, 
     a.lse = lse;
     a.k_pool = c->k_pool + (size_t)layer * c->layer_pool_bytes;
     a.v_pool = c->v_pool + (size_t)layer * c->layer_pool_bytes;
-    a.part_ml = reinterpret_cast<float2*>(c->ws + c->lay.part_ml);
-    a.part_o = reinterpret_cast<float*>(c->ws + c->lay.part_o);
+    a.part_ml = part_ml;
+    a.part_o = part_o;
     a.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
+    a.queue = a.status + 16;   // the status area is 1 KiB, zeroed at creation; the kernel rewinds the queue itself
     a.n_items = (int32_t)t.items.size();
+    a.n_narrow = t.n_narrow_items;
     a.n_leaves = t.n_leaves;
     a.n_units = (int32_t)(t.unit.size() / 4);
     a.Hq = c->cfg.num_q_heads;
@@ -698,8 +703,14 @@ static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, 
     a.G = c->cfg.num_q_heads / c->cfg.num_kv_heads;
     a.pages_per_layer = c->cfg.pages_per_layer;
     a.scale_log2 = c->scale_log2;
-    a.worker_off = blob_ptr<int32_t>(c, c->bo.worker_off);
-    a.n_workers = c->fp.n_workers;
+    return a;
+}
+
+static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse, cudaStream_t s) {
+    const ets::Tree& t = c->tree;
+    if (t.n_leaves == 0) return ETS_OK;
+    const ets::DecodeArgs a = decode_args(c, layer, q, out, lse, reinterpret_cast<float2*>(c->ws + c->lay.part_ml),
+                                          reinterpret_cast<float*>(c->ws + c->lay.part_o));
 
     cudaEvent_t* ev = nullptr;
     if (c->opt_timing) {
@@ -837,31 +848,8 @@ int32_t ets_tree_attn_decode_static(ets_ctx* c, int32_t layer, const void* q, vo
     if (t.n_leaves == 0) return ETS_OK;
     unsigned char* scratch = g_static_scratch_addr[dev];
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    ets::DecodeArgs a{};
-    a.units = blob_ptr<int4>(c, c->bo.units);
-    a.items = blob_ptr<ets::DevItem>(c, c->bo.items);
-    a.node_leaves = blob_ptr<int32_t>(c, c->bo.node_leaves);
-    a.node_len = blob_ptr<int32_t>(c, c->bo.node_len) + (size_t)layer * c->bo.len_stride;
-    a.leaf_slot_off = blob_ptr<int32_t>(c, c->bo.leaf_slot_off);
-    a.leaf_slots = blob_ptr<int32_t>(c, c->bo.leaf_slots);
-    a.q = reinterpret_cast<const __nv_bfloat16*>(q);
-    a.out = reinterpret_cast<__nv_bfloat16*>(out);
-    a.lse = lse;
-    a.k_pool = c->k_pool + (size_t)layer * c->layer_pool_bytes;
-    a.v_pool = c->v_pool + (size_t)layer * c->layer_pool_bytes;
-    a.part_ml = reinterpret_cast<float2*>(scratch);
-    a.part_o = reinterpret_cast<float*>(scratch + ml_bytes);
-    a.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
-    a.n_items = (int32_t)t.items.size();
-    a.n_leaves = t.n_leaves;
-    a.n_units = (int32_t)(t.unit.size() / 4);
-    a.Hq = c->cfg.num_q_heads;
-    a.Hkv = c->cfg.num_kv_heads;
-    a.G = G;
-    a.pages_per_layer = c->cfg.pages_per_layer;
-    a.scale_log2 = c->scale_log2;
-    a.worker_off = blob_ptr<int32_t>(c, c->bo.worker_off);
-    a.n_workers = c->fp.n_workers;
+    const ets::DecodeArgs a = decode_args(c, layer, q, out, lse, reinterpret_cast<float2*>(scratch),
+                                          reinterpret_cast<float*>(scratch + ml_bytes));
     if (int32_t rc = launch_attention(c, a, s)) return rc;
     ets::launch_merge(a, D, s);
     ETS_CUDA(c, cudaGetLastError());

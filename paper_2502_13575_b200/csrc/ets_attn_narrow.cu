@@ -4,7 +4,9 @@
 // 16 query rows, i.e. at most 16 flop per byte.  The kernel is therefore organised around keeping
 // bytes in flight, not around arithmetic:
 //   * persistent grid, one CTA per SM, kNarrowWarps independent warps per CTA; a warp is a worker
-//     with its own contiguous, cost-balanced piece of the work line, so no warp waits for another;
+//     that takes work items from a queue ordered longest first: item w for warp w, then whatever
+//     a shared counter hands out, so a warp that is early simply takes more; the next item
+//     (descriptor, page slots, lengths) is fetched in the background, one dependent load per tile;
 //   * every warp owns a ring of kDepth (2) shared-memory slots; a slot receives one K tile and one V
 //     tile (16 tokens x D bf16 each) by two bulk asynchronous copies (TMA engine, linear form) that
 //     complete on the slot's mbarrier; the ring runs ahead across item boundaries;
@@ -19,6 +21,8 @@
 //     the separate merge kernel: the merging warps stall their own streaming).
 // Every wait on an mbarrier is bounded; on expiry the warp raises the status word, starts no new
 // copy and only waits (again boundedly) for the few copies it had already started.
+#include <climits>
+
 #include "ets_device.cuh"
 
 namespace ets {
@@ -28,6 +32,10 @@ namespace {
 constexpr int kWarps = kNarrowWarps;
 constexpr int kDepth = 2;   // measured as fast as 3; 2 leaves shared memory for a wide-kernel CTA on the same SM
 constexpr uint32_t kSpinLimit = 1u << 22;
+#ifndef ETS_CLAIM_AHEAD
+#define ETS_CLAIM_AHEAD 6
+#endif
+constexpr int kClaimAhead = ETS_CLAIM_AHEAD;   // tiles left in the current item when the next one is claimed
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -113,314 +121,395 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// A batch of up to 32 consecutive page slots of an item, one per lane: its page id and the number
-// of tokens it holds now (0 = skip: empty, or a page id outside the pool, which is also flagged).
-// Loading descriptors 32 at a time keeps the dependent global loads (slot -> node length) off the
-// per-tile critical path.
-struct UnitBatch {
-    int base = 0;       // index (within the item) of lane 0's slot
+// The page slots of one narrow item, one per lane (an item has at most 32): page id and the number
+// of tokens the slot holds now (0 = skip: empty, or a page id outside the pool, which is also flagged).
+struct SlotView {
     int page = 0;
     int valid = 0;
     uint32_t live = 0;  // bit i: lane i's slot has tokens
-
-    __device__ __forceinline__ void load(const DecodeArgs& a, int unit_begin, int unit_count, int from, int lane) {
-        base = from;
-        const int idx = from + lane;
-        page = 0;
-        valid = 0;
-        if (idx < unit_count) {
-            const int4 un = a.units[unit_begin + idx];
-            int v = a.node_len[un.y] - un.z;
-            v = v < 0 ? 0 : (v > 16 ? 16 : v);
-            if (v > 0 && (un.x < 0 || (int64_t)un.x >= a.pages_per_layer)) {  // never read outside the pool
-                atomicExch(a.status, -1);
-                v = 0;
-            }
-            page = un.x;
-            valid = v;
-        }
-        live = __ballot_sync(0xffffffffu, valid > 0);
-    }
-    // first live slot at or after item index u inside this batch, or -1
-    __device__ __forceinline__ int next_live(int u) const {
-        const int sh = u - base;
-        if (sh >= 32) return -1;
-        const uint32_t m = live >> sh;
-        return m ? u + __ffs(m) - 1 : -1;
-    }
 };
 
-// Issue side of a warp's ring: walks the worker's items and their page slots, skipping slots that
-// hold no token yet, and starts the two bulk copies of the next one.
-template <int D>
-struct Feeder {
-    int it, it_end;       // next item index / end of this worker's items
-    int u = 0, ub = 0, uc = 0, head = 0;
-    bool reread = false;  // the current item's pages are read again by the next leaf tile
-    uint64_t pol_stream;  // K/V read for the last time goes first when L2 needs room
-    UnitBatch batch;
-    uint32_t n_issued = 0;
-    uint32_t ring, bars;  // shared-memory addresses of this warp's slots and barriers
-
-    __device__ bool issue_next(const DecodeArgs& a, int lane) {
-        constexpr uint32_t TB = 16 * D * 2;
-        while (true) {
-            if (u >= uc) {
-                if (it >= it_end) return false;
-                const DevItem d = a.items[it];
-                ++it;
-                ub = d.unit_begin; uc = d.unit_count; head = d.kv_head; u = 0;
-                reread = (d.reserved & 1) != 0;
-                batch.load(a, ub, uc, 0, lane);
-                continue;
-            }
-            const int nxt = batch.next_live(u);
-            if (nxt < 0) {
-                u = batch.base + 32 < uc ? batch.base + 32 : uc;
-                if (u < uc) batch.load(a, ub, uc, u, lane);
-                continue;
-            }
-            const int page = __shfl_sync(0xffffffffu, batch.page, nxt - batch.base);
-            u = nxt + 1;
-            if (lane == 0) {
-                const uint32_t slot = n_issued % kDepth;
-                const uint32_t bar = bars + slot * 8;
-                const uint32_t dst = ring + slot * 2 * TB;
-                const size_t off = pool_tile_offset(a.pages_per_layer, page, head, TB);
-                mbar_expect_tx(bar, 2 * TB);
-                if (reread) {
-                    bulk_g2s(dst, a.k_pool + off, TB, bar);
-                    bulk_g2s(dst + TB, a.v_pool + off, TB, bar);
-                } else {
-                    bulk_g2s_hint(dst, a.k_pool + off, TB, bar, pol_stream);
-                    bulk_g2s_hint(dst + TB, a.v_pool + off, TB, bar, pol_stream);
-                }
-            }
-            ++n_issued;
-            return true;
-        }
-    }
+// The next item of this warp, fetched in the background while the current one is processed.  The
+// chain claim -> descriptor -> page slots -> node lengths is four dependent memory round trips;
+// one link is started per consumed tile, so that none of them stalls the warp.
+struct NextItem {
+    int stage = 4;      // 0 nothing claimed, 1 claim in flight, 2 descriptor in flight, 3 slots in flight, 4 complete
+    int idx = INT_MAX;  // queue position; >= n_narrow: the queue is empty
+    int claim = 0;      // lane 0: value returned by the shared counter
+    DevItem it{};
+    int4 un = make_int4(0, 0, 0, 0);
+    int leaf[2] = {0, 0};   // leaf of query rows grp and 8 + grp
+    SlotView v;
 };
 
 template <int D, int NT>
-__device__ __forceinline__ void run_item(const DecodeArgs& a, const DevItem it, Feeder<D>& feed, uint32_t& n_consumed,
-                                         bool& dead, int lane) {
-    constexpr int KS = D / 16;
-    constexpr uint32_t TB = 16 * D * 2;
-    const int G = a.G;
-    const int rows = it.n_leaves_tile * G;
-    const int h = it.kv_head;
-    const int quad = lane & 3, grp = lane >> 2;
+struct Acc {
+    float o[D / 16][NT][4];
+    float m[NT][2], l[NT][2];
+};
 
-    // Q^T fragments (B operand): row n = 8j + grp, features 16ks + 2quad + {0,1} and + 8
-    uint32_t qf[NT][KS][2];
+// Q^T fragments (B operand) of an item: row n = 8j + grp, features 16ks + 2quad + {0,1} and + 8
+template <int D, int NT>
+__device__ __forceinline__ void load_q(const DecodeArgs& a, const DevItem& it, const int (&leaf)[2], int lane,
+                                       uint32_t (&qf)[NT][D / 16][2]) {
+    constexpr int KS = D / 16;
+    const int G = a.G, rows = it.n_leaves_tile * G, quad = lane & 3, grp = lane >> 2;
 #pragma unroll
     for (int j = 0; j < NT; ++j) {
         const int n = 8 * j + grp;
         if (n < rows) {
-            const int leaf = a.node_leaves[it.leaf_list_begin + n / G];
-            const uint32_t* qp = reinterpret_cast<const uint32_t*>(a.q + ((size_t)leaf * a.Hq + h * G + n % G) * D);
+            const uint32_t* qp = reinterpret_cast<const uint32_t*>(a.q + ((size_t)leaf[j] * a.Hq + it.kv_head * G + n % G) * D);
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
-                qf[j][ks][0] = qp[8 * ks + quad];
-                qf[j][ks][1] = qp[8 * ks + 4 + quad];
+                qf[j][ks][0] = __ldg(qp + 8 * ks + quad);
+                qf[j][ks][1] = __ldg(qp + 8 * ks + 4 + quad);
             }
         } else {
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) qf[j][ks][0] = qf[j][ks][1] = 0u;
         }
     }
+}
 
-    float o[KS][NT][4];
-    float m[NT][2], l[NT][2];
-#pragma unroll
-    for (int j = 0; j < NT; ++j) {
-        m[j][0] = m[j][1] = -INFINITY;
-        l[j][0] = l[j][1] = 0.f;
-#pragma unroll
-        for (int mt = 0; mt < KS; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) o[mt][j][i] = 0.f;
-    }
-
+// One K tile and one V tile (16 tokens) against the item's query rows: S^T = K . Q^T, online softmax
+// in log2 units, O^T += V^T . P^T.
+template <int D, int NT>
+__device__ __forceinline__ void tile_step(uint32_t kt, uint32_t vt, int valid, float scale_log2, int lane,
+                                          const uint32_t (&qf)[NT][D / 16][2], Acc<D, NT>& acc) {
+    constexpr int KS = D / 16;
+    const int grp = lane >> 2;
     // per-lane pieces of the ldmatrix row addresses inside a tile
     const int mat = lane >> 3, r8 = lane & 7;
     const int k_tok = r8 + (mat & 1) * 8;    // K: matrices 0/1 = tokens 0-7 / 8-15, 2/3 = next 8 features
-    const int k_cb = mat >> 1;
     const int v_tok = r8 + (mat >> 1) * 8;   // V^T: matrices 0/1 = features +0 / +8, 2/3 = tokens 8-15
-    const int v_cb = mat & 1;
-    const uint32_t k_row = (uint32_t)(k_tok >> 3) * (D / 64) * 1024u + (uint32_t)(k_tok & 7) * 128u;
-    const uint32_t v_row = (uint32_t)(v_tok >> 3) * (D / 64) * 1024u + (uint32_t)(v_tok & 7) * 128u;
+    // chunk index 2*ks + cb, XOR-swizzled by the row: (2ks | cb) ^ r8 = (2ks) ^ (cb ^ r8)
+    const uint32_t k_lane = kt + (uint32_t)(k_tok >> 3) * (D / 64) * 1024u + (uint32_t)r8 * 128u + (uint32_t)(((mat >> 1) ^ r8) << 4);
+    const uint32_t v_lane = vt + (uint32_t)(v_tok >> 3) * (D / 64) * 1024u + (uint32_t)r8 * 128u + (uint32_t)(((mat & 1) ^ r8) << 4);
 
-    UnitBatch cb;
-    cb.load(a, it.unit_begin, it.unit_count, 0, lane);
-    for (int u = 0; u < it.unit_count;) {
-        const int nxt = cb.next_live(u);
-        if (nxt < 0) {
-            u = cb.base + 32 < it.unit_count ? cb.base + 32 : it.unit_count;
-            if (u < it.unit_count) cb.load(a, it.unit_begin, it.unit_count, u, lane);
-            continue;
+    if (valid < 16) {
+        // rows past the node's length hold stale bytes: zero them in V so that 0 * garbage
+        // cannot produce NaN (their scores are masked below)
+        for (int i = lane; i < (16 - valid) * (D / 8); i += 32) {
+            const int t = valid + i / (D / 8), c = i % (D / 8);
+            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_offset(D, t, c * 8)), "r"(0u) : "memory");
         }
-        const int valid = __shfl_sync(0xffffffffu, cb.valid, nxt - cb.base);
-        u = nxt + 1;
-        const uint32_t slot = n_consumed % kDepth;
-        const uint32_t parity = (n_consumed / kDepth) & 1u;
-        const bool issued = n_consumed < feed.n_issued;
-        ++n_consumed;
-        if (dead) {
-            // gave up earlier: only wait (boundedly) for copies already started, so that none
-            // lands after the CTA has gone; nothing new is issued
-            if (issued) mbar_wait_bounded(feed.bars + slot * 8, parity);
-            continue;
-        }
-        if (!mbar_wait_bounded(feed.bars + slot * 8, parity)) {
-            if (lane == 0) atomicExch(a.status, -7);
-            dead = true;
-            continue;
-        }
-        const uint32_t kt = feed.ring + slot * 2 * TB;
-        const uint32_t vt = kt + TB;
+        __syncwarp();
+    }
 
-        if (valid < 16) {
-            // rows past the node's length hold stale bytes: zero them in V so that 0 * garbage
-            // cannot produce NaN (their scores are masked below)
-            for (int i = lane; i < (16 - valid) * (D / 8); i += 32) {
-                const int t = valid + i / (D / 8), c = i % (D / 8);
-                asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_offset(D, t, c * 8)), "r"(0u) : "memory");
-            }
-            __syncwarp();
-        }
-
-        // S^T = K_tile . Q^T
-        float s[NT][4];
+    // S^T = K_tile . Q^T; with a single column tile the k-steps alternate between two accumulators, so
+    // that the chain of dependent products is half as long
+    constexpr int NS = NT == 1 ? 2 : 1;
+    float s[NT][4], s2[NS][4];
 #pragma unroll
-        for (int j = 0; j < NT; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+    for (int j = 0; j < NT; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+    s2[0][0] = s2[0][1] = s2[0][2] = s2[0][3] = 0.f;
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            const int chunk = 2 * ks + k_cb;
-            uint32_t af[4];
-            ldsm_x4(kt + k_row + (uint32_t)(chunk >> 3) * 1024u + (uint32_t)(((chunk & 7) ^ (k_tok & 7)) << 4), af);
+    for (int ks = 0; ks < KS; ++ks) {
+        uint32_t af[4];
+        ldsm_x4((k_lane + (uint32_t)(ks >> 2) * 1024u) ^ (uint32_t)((ks & 3) << 5), af);
+        if (NT == 1 && (ks & 1)) {
+            mma_bf16(s2[0], af, qf[0][ks]);
+        } else {
 #pragma unroll
             for (int j = 0; j < NT; ++j) mma_bf16(s[j], af, qf[j][ks]);
         }
-
-        // online softmax (log2 units); this lane holds tokens grp and grp+8 of rows 2quad, 2quad+1
-        uint32_t pf[NT][2];
+    }
+    if (NT == 1) {
 #pragma unroll
-        for (int j = 0; j < NT; ++j) {
-            float sv[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int tok = grp + (i >> 1) * 8;
-                sv[i] = tok < valid ? s[j][i] * a.scale_log2 : -INFINITY;
-            }
-            float p[4];
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                float mx = fmaxf(sv[r], sv[r + 2]);
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-                const float mn = fmaxf(m[j][r], mx);     // finite: token 0 of the tile is valid
-                const float corr = exp2f(m[j][r] - mn);
-                // weights are rounded to bf16 here, so that the row sum and the product use the same
-                // values and the rounding cancels in sum(p v) / sum(p)
-                p[r] = __bfloat162float(__float2bfloat16_rn(exp2f(sv[r] - mn)));
-                p[r + 2] = __bfloat162float(__float2bfloat16_rn(exp2f(sv[r + 2] - mn)));
-                l[j][r] = l[j][r] * corr + p[r] + p[r + 2];
-                m[j][r] = mn;
-#pragma unroll
-                for (int mt = 0; mt < KS; ++mt) {
-                    o[mt][j][r] *= corr;
-                    o[mt][j][r + 2] *= corr;
-                }
-            }
-            // P^T as B operand: transpose the two 8x8 (token x row) blocks
-            pf[j][0] = movmatrix_trans(pack_bf16(p[0], p[1]));
-            pf[j][1] = movmatrix_trans(pack_bf16(p[2], p[3]));
-        }
-
-        // O^T += V_tile^T . P^T
-#pragma unroll
-        for (int mt = 0; mt < KS; ++mt) {
-            const int chunk = 2 * mt + v_cb;
-            uint32_t af[4];
-            ldsm_x4_trans(vt + v_row + (uint32_t)(chunk >> 3) * 1024u + (uint32_t)(((chunk & 7) ^ (v_tok & 7)) << 4), af);
-#pragma unroll
-            for (int j = 0; j < NT; ++j) mma_bf16(o[mt][j], af, pf[j]);
-        }
-
-        // the slot is free again: order our shared-memory reads (and the zero fill) before the
-        // next asynchronous write into it, then refill
-        __syncwarp();
-        fence_proxy_async();
-        feed.issue_next(a, lane);
+        for (int i = 0; i < 4; ++i) s[0][i] += s2[0][i];
     }
 
-    // partial (m, l, o) of this item, straight from registers
+    // online softmax (log2 units); this lane holds tokens grp and grp+8 of rows 2quad, 2quad+1
+    uint32_t pf[NT][2];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+        float sv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int tok = grp + (i >> 1) * 8;
+            sv[i] = tok < valid ? s[j][i] * scale_log2 : -INFINITY;
+        }
+        float p[4];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            float mx = fmaxf(sv[r], sv[r + 2]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float mn = fmaxf(acc.m[j][r], mx);     // finite: token 0 of the tile is valid
+            const float corr = exp2f(acc.m[j][r] - mn);
+            // weights are rounded to bf16 here, so that the row sum and the product use the same
+            // values and the rounding cancels in sum(p v) / sum(p)
+            p[r] = __bfloat162float(__float2bfloat16_rn(exp2f(sv[r] - mn)));
+            p[r + 2] = __bfloat162float(__float2bfloat16_rn(exp2f(sv[r + 2] - mn)));
+            acc.l[j][r] = acc.l[j][r] * corr + p[r] + p[r + 2];
+            acc.m[j][r] = mn;
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+                acc.o[mt][j][r] *= corr;
+                acc.o[mt][j][r + 2] *= corr;
+            }
+        }
+        // P^T as B operand: transpose the two 8x8 (token x row) blocks
+        pf[j][0] = movmatrix_trans(pack_bf16(p[0], p[1]));
+        pf[j][1] = movmatrix_trans(pack_bf16(p[2], p[3]));
+    }
+
+    // O^T += V_tile^T . P^T
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt) {
+        uint32_t af[4];
+        ldsm_x4_trans((v_lane + (uint32_t)(mt >> 2) * 1024u) ^ (uint32_t)((mt & 3) << 5), af);
+#pragma unroll
+        for (int j = 0; j < NT; ++j) mma_bf16(acc.o[mt][j], af, pf[j]);
+    }
+}
+
+// partial (m, l, o) of an item, straight from registers
+template <int D, int NT>
+__device__ __forceinline__ void store_partials(const DecodeArgs& a, const DevItem& it, int lane, Acc<D, NT>& acc) {
+    constexpr int KS = D / 16;
+    const int G = a.G, rows = it.n_leaves_tile * G, quad = lane & 3, grp = lane >> 2;
     const uint64_t pol_keep = policy_evict_last();
 #pragma unroll
     for (int j = 0; j < NT; ++j)
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-            float ls = l[j][r];
+            float ls = acc.l[j][r];
             ls += __shfl_xor_sync(0xffffffffu, ls, 4);
             ls += __shfl_xor_sync(0xffffffffu, ls, 8);
             ls += __shfl_xor_sync(0xffffffffu, ls, 16);
             const int n = 8 * j + 2 * quad + r;
             if (n < rows) {
-                const size_t prow = (size_t)(it.slot_first + n / G) * G + n % G;
+                // rows of an item are consecutive: (slot_first + n / G) * G + n % G = slot_first * G + n
+                const size_t prow = (size_t)it.slot_first * G + n;
                 // partials are read back by the merge kernel right after: ask L2 to hold on to them
-                if (grp == 0) st_f32x2_hint(a.part_ml + prow, make_float2(m[j][r], ls), pol_keep);
+                if (grp == 0) st_f32x2_hint(a.part_ml + prow, make_float2(acc.m[j][r], ls), pol_keep);
                 float* po = a.part_o + prow * D + grp;
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) {
-                    st_f32_hint(po + 16 * mt, o[mt][j][r], pol_keep);
-                    st_f32_hint(po + 16 * mt + 8, o[mt][j][r + 2], pol_keep);
+                    st_f32_hint(po + 16 * mt, acc.o[mt][j][r], pol_keep);
+                    st_f32_hint(po + 16 * mt + 8, acc.o[mt][j][r + 2], pol_keep);
                 }
             }
         }
 }
 
+template <int N>
+struct IntTag { static constexpr int value = N; };
+
 template <int D>
-// 168 registers x 256 threads leave room in the register file for a wide-kernel CTA (96 x 192)
+// 168 registers x 256 threads leave room in the register file for a wide-kernel CTA (80 x 192)
 __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
     constexpr uint32_t TB = 16 * D * 2;
+    constexpr uint32_t FULL = 0xffffffffu;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_warps = (int)gridDim.x * kWarps;
+    const int worker = blockIdx.x * kWarps + warp;
+    const int grp = lane >> 2;
+    const int G = a.G;
+
     if (base & 127u) {   // the swizzled tile rows must start on 128-byte boundaries
         if (threadIdx.x == 0) atomicExch(a.status, -1);
-        return;
-    }
-
-    const int worker = blockIdx.x * kWarps + warp;
-    if (worker >= a.n_workers) return;
-    const int i0 = a.worker_off[worker], i1 = a.worker_off[worker + 1];
-    if (i0 >= i1) return;
-
-    Feeder<D> feed;
-    feed.it = i0;
-    feed.it_end = i1;
-    feed.pol_stream = policy_evict_first();
-    feed.ring = base + (uint32_t)warp * kDepth * 2 * TB;
-    feed.bars = base + (uint32_t)kWarps * kDepth * 2 * TB + (uint32_t)warp * kDepth * 8;
-    if (lane == 0) {
+    } else if (worker < a.n_narrow) {
+        const uint32_t ring = base + (uint32_t)warp * kDepth * 2 * TB;
+        const uint32_t bars = base + (uint32_t)kWarps * kDepth * 2 * TB + (uint32_t)warp * kDepth * 8;
+        if (lane == 0) {
 #pragma unroll
-        for (int s = 0; s < kDepth; ++s) mbar_init(feed.bars + s * 8, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            for (int s = 0; s < kDepth; ++s) mbar_init(bars + s * 8, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+        const uint64_t pol_stream = policy_evict_first();   // K/V read for the last time goes first when L2 needs room
+
+        uint32_t n_issued = 0, n_consumed = 0;
+        DevItem cur{};
+        SlotView cv;
+        int cur_leaf[2] = {0, 0};
+        bool f_on_next = false;     // the issue side has moved on to the next item
+        uint32_t f_live = 0;        // slots of its item that it has not started yet
+        int f_page = 0, f_head = 0; // its item: page id per lane, kv head
+        bool f_reread = false;      // its item's pages are read again by the next leaf tile
+        NextItem nx;
+
+        // one link of the background fetch of the next item
+        auto fetch_step = [&]() {
+            switch (nx.stage) {
+                case 0:
+                    if (lane == 0) nx.claim = atomicAdd(a.queue, 1);
+                    nx.stage = 1;
+                    break;
+                case 1:
+                    nx.idx = n_warps + __shfl_sync(FULL, nx.claim, 0);
+                    if (nx.idx < a.n_narrow) {
+                        nx.it = a.items[nx.idx];
+                        nx.stage = 2;
+                    } else {
+                        nx.idx = INT_MAX;
+                        nx.stage = 4;
+                    }
+                    break;
+                case 2: {
+                    nx.un = lane < nx.it.unit_count ? a.units[nx.it.unit_begin + lane] : make_int4(0, 0, 0, 0);
+                    const int rows = nx.it.n_leaves_tile * G;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j)
+                        nx.leaf[j] = 8 * j + grp < rows ? a.node_leaves[nx.it.leaf_list_begin + (8 * j + grp) / G] : 0;
+                    nx.stage = 3;
+                    break;
+                }
+                case 3: {
+                    int v = 0;
+                    if (lane < nx.it.unit_count) {
+                        v = a.node_len[nx.un.y] - nx.un.z;
+                        v = v < 0 ? 0 : (v > 16 ? 16 : v);
+                        if (v > 0 && (nx.un.x < 0 || (int64_t)nx.un.x >= a.pages_per_layer)) {  // never read outside the pool
+                            atomicExch(a.status, -1);
+                            v = 0;
+                        }
+                    }
+                    nx.v.page = nx.un.x;
+                    nx.v.valid = v;
+                    nx.v.live = __ballot_sync(FULL, v > 0);
+                    nx.stage = 4;
+                    break;
+                }
+                default:
+                    break;
+            }
+        };
+        auto fetch_finish = [&]() {
+            while (nx.stage < 4) fetch_step();
+        };
+
+        // Issue side of the ring: starts the two bulk copies of the next page slot that holds tokens,
+        // in the current item or, once that is exhausted, in the next one.
+        auto issue_next = [&]() -> bool {
+            while (true) {
+                if (f_live) {
+                    const int b = __ffs(f_live) - 1;
+                    f_live &= f_live - 1;
+                    const int page = __shfl_sync(FULL, f_page, b);
+                    if (lane == 0) {
+                        const uint32_t slot = n_issued % kDepth;
+                        const uint32_t bar = bars + slot * 8;
+                        const uint32_t dst = ring + slot * 2 * TB;
+                        const size_t off = pool_tile_offset(a.pages_per_layer, page, f_head, TB);
+                        mbar_expect_tx(bar, 2 * TB);
+                        if (f_reread) {
+                            bulk_g2s(dst, a.k_pool + off, TB, bar);
+                            bulk_g2s(dst + TB, a.v_pool + off, TB, bar);
+                        } else {
+                            bulk_g2s_hint(dst, a.k_pool + off, TB, bar, pol_stream);
+                            bulk_g2s_hint(dst + TB, a.v_pool + off, TB, bar, pol_stream);
+                        }
+                    }
+                    ++n_issued;
+                    return true;
+                }
+                if (f_on_next) return false;   // nothing is known beyond the next item yet
+                fetch_finish();
+                if (nx.idx == INT_MAX) return false;   // the queue is empty
+                // the issue side keeps its own copy of what it needs of its item, so that it never
+                // touches the registers of a fetch that is still in flight
+                f_on_next = true;
+                f_live = nx.v.live;
+                f_page = nx.v.page;
+                f_head = nx.it.kv_head;
+                f_reread = (nx.it.reserved & 1) != 0;
+            }
+        };
+
+        // the first item of this warp is its own index in the queue
+        nx.idx = worker;
+        nx.it = a.items[worker];
+        nx.stage = 2;
+        fetch_finish();
+
+        bool dead = false;
+        while (nx.idx != INT_MAX && !dead) {
+            // make the fetched item the current one and start fetching its successor
+            cur = nx.it;
+            cv = nx.v;
+            cur_leaf[0] = nx.leaf[0];
+            cur_leaf[1] = nx.leaf[1];
+            if (f_on_next) {
+                f_on_next = false;
+            } else {
+                f_live = cv.live;
+                f_page = cv.page;
+                f_head = cur.kv_head;
+                f_reread = (cur.reserved & 1) != 0;
+            }
+            nx.stage = 0;
+            nx.idx = INT_MAX;
+            if (__popc(cv.live) <= kClaimAhead) fetch_step();
+            while (n_issued - n_consumed < (uint32_t)kDepth && issue_next()) {}
+
+            auto process = [&](auto tag) {
+                constexpr int NT = decltype(tag)::value;
+                constexpr int KS = D / 16;
+                uint32_t qf[NT][KS][2];
+                load_q<D, NT>(a, cur, cur_leaf, lane, qf);
+                Acc<D, NT> acc;
+#pragma unroll
+                for (int j = 0; j < NT; ++j) {
+                    acc.m[j][0] = acc.m[j][1] = -INFINITY;
+                    acc.l[j][0] = acc.l[j][1] = 0.f;
+#pragma unroll
+                    for (int mt = 0; mt < KS; ++mt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc.o[mt][j][i] = 0.f;
+                }
+                uint32_t todo = cv.live;
+                while (todo) {
+                    const int b = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const int valid = __shfl_sync(FULL, cv.valid, b);
+                    const uint32_t slot = n_consumed % kDepth;
+                    const uint32_t parity = (n_consumed / kDepth) & 1u;
+                    ++n_consumed;
+                    if (!__all_sync(FULL, mbar_wait_bounded(bars + slot * 8, parity))) {   // same answer in every lane
+                        if (lane == 0) atomicExch(a.status, -7);
+                        dead = true;
+                        return;
+                    }
+                    const uint32_t kt = ring + slot * 2 * TB;
+                    tile_step<D, NT>(kt, kt + TB, valid, a.scale_log2, lane, qf, acc);
+                    // The slot is free again once every lane has its fragments (their values have been
+                    // consumed by the products above).  Only the zero fill of a partial page is a write
+                    // through the generic proxy that the next asynchronous copy must be ordered after.
+                    __syncwarp();
+                    if (valid < 16) fence_proxy_async();
+                    issue_next();
+                    // the successor is claimed late (an early claim would tie work to this warp while
+                    // others run out of it), but early enough for its four loads to finish in time
+                    if (__popc(todo) < kClaimAhead) fetch_step();
+                }
+                store_partials<D, NT>(a, cur, lane, acc);
+            };
+            if (cur.n_leaves_tile * G <= 8) process(IntTag<1>{});
+            else process(IntTag<2>{});
+            if (!dead) fetch_finish();
+        }
+        if (dead) {
+            // gave up: nothing new is started; wait (boundedly) for the copies already started, so that
+            // none lands after the CTA has gone.  The slot whose wait ran out counts as consumed.
+            while (n_consumed < n_issued) {
+                mbar_wait_bounded(bars + (n_consumed % kDepth) * 8, (n_consumed / kDepth) & 1u);
+                ++n_consumed;
+            }
+        }
     }
+
+    // Every warp of the grid reports here; the last one rewinds the queue for the next launch.  A warp's
+    // claims have all returned before it gets here, so nobody touches the counter after the last report.
     __syncwarp();
-
-#pragma unroll
-    for (int s = 0; s < kDepth; ++s) feed.issue_next(a, lane);
-
-    uint32_t n_consumed = 0;
-    bool dead = false;
-    for (int i = i0; i < i1; ++i) {
-        const DevItem it = a.items[i];
-        if (it.n_leaves_tile * a.G <= 8) run_item<D, 1>(a, it, feed, n_consumed, dead, lane);
-        else run_item<D, 2>(a, it, feed, n_consumed, dead, lane);
+    if (lane == 0 && atomicAdd(a.queue + 1, 1) == n_warps - 1) {
+        a.queue[0] = 0;
+        a.queue[1] = 0;
     }
 }
 
@@ -445,7 +534,7 @@ cudaError_t narrow_prepare(int D) {
 }
 
 void launch_partial_narrow(const DecodeArgs& a, int D, int n_ctas, cudaStream_t s) {
-    if (a.n_items <= 0 || n_ctas <= 0) return;
+    if (a.n_narrow <= 0 || n_ctas <= 0) return;
     if (D == 128) attn_partial_narrow_kernel<128><<<n_ctas, kWarps * 32, narrow_smem_bytes(128), s>>>(a);
     else attn_partial_narrow_kernel<64><<<n_ctas, kWarps * 32, narrow_smem_bytes(64), s>>>(a);
 }

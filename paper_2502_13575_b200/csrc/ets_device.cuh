@@ -52,10 +52,9 @@ struct DecodeArgs {
     const char* v_pool;
     float2* part_ml;               // [slot][G]  (m in log2 units, l); a slot belongs to one kv head
     float* part_o;                 // [slot][G][D]
-    const int32_t* worker_off;     // items of warp-worker w: [worker_off[w], worker_off[w+1])
-    int32_t n_workers;
+    int32_t* queue;                // [0] narrow items handed out beyond the first per warp, [1] warps that have finished
     int32_t* status;
-    int32_t n_items, n_leaves, n_units;
+    int32_t n_items, n_narrow, n_leaves, n_units;   // narrow items come first in `items`
     int32_t Hq, Hkv, G;
     int64_t pages_per_layer;
     float scale_log2;              // sm_scale * log2(e)

@@ -173,90 +173,128 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             }
     }
 
-    // ---- work line: for every segment, kv head and leaf tile, the segment's page slots.  The line
-    // is cut into n_workers contiguous pieces of equal cost (a page slot costs 1, starting an item
-    // costs kItemCost), so a piece boundary may fall inside a run and split it into two items.
-    // Tiles of one (segment, head) are adjacent: the re-read of its K/V by the next tile is recent.
+    // ---- narrow work queue.  A run is the page slots of one segment for one (kv head, leaf tile).
+    // Runs are cut into pieces of at most `cap` page slots (at most 32: one lane per slot); a piece is
+    // one work item.  The resident warps of the attention kernel take item w first (w = warp index)
+    // and then claim the following items one by one from a shared counter, so the queue is ordered
+    // longest piece first and its last pieces are cut shorter: whichever warp is early takes more.
+    // The pieces of one (segment part) for all heads and leaf tiles stay adjacent in the queue: they
+    // are claimed at about the same time, so the re-read of K/V by the next leaf tile hits in L2.
     const int32_t leaves_per_tile = std::max(1, p.rows_per_item / std::max(1, p.gqa));
     const int32_t n_workers = std::max(1, p.n_workers);
-    const int32_t max_run = p.chunk_pages > 0 ? p.chunk_pages : INT32_MAX;
-    const double kItemCost = p.cost_item;
+    const int32_t max_run = std::min(32, p.chunk_pages > 0 ? p.chunk_pages : 32);
     auto is_wide = [&](int32_t s) {
         const int32_t r = g[seg_head[s]] * p.gqa;
         return p.wide_rows > 0 && r > p.rows_per_item && r >= p.wide_min_rows;
     };
-    // weight of one page slot of the tile starting at leaf l0 of a group of gn leaves
-    auto unit_weight = [&](int32_t gn, int32_t l0) {
-        const int32_t rows = std::min(leaves_per_tile, gn - l0) * p.gqa;
-        return (rows > 8 ? p.cost_rows16 : 1.0) * (l0 > 0 ? p.cost_reread : 1.0);
-    };
-    int64_t n_runs = 0;
-    double run_cost = 0.0;
-    for (int32_t s = 0; s < n_seg; ++s) {
-        const int64_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
-        if (nu == 0 || is_wide(s)) continue;
-        const int32_t gn = g[seg_head[s]];
-        for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile) {
-            n_runs += p.num_kv_heads;
-            run_cost += (double)nu * unit_weight(gn, l0) * p.num_kv_heads;
-        }
-    }
-    // the target load is re-derived from what is left every time a worker is closed, so rounding
-    // never piles up on the last worker
-    double left_cost = run_cost;
-    int64_t left_runs = n_runs;
-    auto target_for = [&](int32_t workers_left) {
-        return (std::max(left_cost, 0.0) + kItemCost * (double)(left_runs + workers_left)) / workers_left;
-    };
-    double target = target_for(n_workers);
-    t.chunk_pages_used = p.chunk_pages;
-    t.worker_off.assign((size_t)n_workers + 1, 0);
-    int32_t w = 0;
-    double load = 0.0;
-    int64_t slots = 0;
+    struct Part { int32_t seg, begin, len; };
+    // per narrow segment: page slots, pieces per part (heads x leaf tiles), mean weight of a page slot
+    // over its leaf tiles, leaves
+    struct SegInfo { int32_t seg, nu, mult, gn; double w; };
+    std::vector<SegInfo> narrow;
+    narrow.reserve((size_t)n_seg);
     for (int32_t s = 0; s < n_seg; ++s) {
         const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
         if (nu == 0 || is_wide(s)) continue;
-        const int32_t head_node = seg_head[s];
+        const int32_t gn = g[seg_head[s]];
+        const int32_t tiles = ceil_div(gn, leaves_per_tile);
+        double wsum = 0.0;
+        for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile)
+            wsum += (std::min(leaves_per_tile, gn - l0) * p.gqa > 8 ? p.cost_rows16 : 1.0) * (l0 > 0 ? p.cost_reread : 1.0);
+        narrow.push_back({s, nu, p.num_kv_heads * tiles, gn, wsum / tiles});
+    }
+    // Estimated time of the queue for a piece length, in page-slot units: the mean load of a warp plus
+    // half of a late piece, or the longest piece when that is more (fewer pieces than warps).
+    auto estimate = [&](int32_t cap, int32_t tail_cap, int64_t& slots_needed) {
+        double total = 0.0, longest = 0.0, shortest = 1e30;
+        slots_needed = 0;
+        int64_t pieces = 0;
+        for (const SegInfo& q : narrow) {
+            const int32_t np_ = ceil_div(q.nu, cap);
+            const double len = (double)q.nu / np_;
+            total += ((double)np_ * p.cost_item + q.nu * q.w) * q.mult;
+            longest = std::max(longest, p.cost_item + std::ceil(len) * q.w);
+            shortest = std::min(shortest, p.cost_item + std::min<double>(len, tail_cap) * q.w);
+            pieces += (int64_t)np_ * q.mult;
+            slots_needed += (int64_t)np_ * p.num_kv_heads * q.gn;
+        }
+        if (narrow.empty()) return 0.0;
+        // the cut of the last pieces adds about one item per warp
+        if (pieces > n_workers && tail_cap < cap) { total += p.cost_item * n_workers; slots_needed += (int64_t)n_workers * leaves_per_tile; }
+        return std::max(total / n_workers + 0.5 * shortest, longest);
+    };
+    int32_t cap = 0, tail_cap = 0;
+    {
+        static const int32_t kCaps[] = {32, 24, 16, 12, 8, 6, 4, 3, 2, 1};
+        double best = 0.0;
+        int32_t prev_c = 0;
+        for (int32_t cand : kCaps) {
+            const int32_t c = std::min(cand, max_run);
+            if (c == prev_c) continue;
+            prev_c = c;
+            const int32_t tc = p.tail_pages > 0 ? p.tail_pages : std::max(8, c / 3);
+            int64_t need_slots = 0;
+            const double est = estimate(c, tc, need_slots);
+            if (need_slots > p.max_partial_slots || need_slots > p.max_items) continue;
+            if (cap == 0 || est < best * 0.98) { best = est; cap = c; tail_cap = tc; }
+        }
+        if (cap == 0) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
+        t.chunk_pages_used = cap;
+    }
+    std::vector<Part> best_parts;
+    {
+        auto by_len = [](const Part& a, const Part& b) { return a.len > b.len; };
+        auto cut = [](std::vector<Part>& out, int32_t seg, int32_t begin, int32_t len, int32_t c) {
+            const int32_t np_ = (len + c - 1) / c;
+            for (int32_t k = 0; k < np_; ++k) {
+                const int32_t b = (int32_t)((int64_t)len * k / np_), e = (int32_t)((int64_t)len * (k + 1) / np_);
+                out.push_back({seg, begin + b, e - b});
+            }
+        };
+        std::vector<int32_t> mult_of((size_t)n_seg, 0);
+        int64_t total_pieces = 0;
+        for (const SegInfo& q : narrow) {
+            mult_of[q.seg] = q.mult;
+            cut(best_parts, q.seg, 0, q.nu, cap);
+        }
+        std::stable_sort(best_parts.begin(), best_parts.end(), by_len);
+        for (const Part& q : best_parts) total_pieces += mult_of[q.seg];
+        if (tail_cap < cap && total_pieces > n_workers) {
+            // the parts that hold the last n_workers pieces of the queue are cut down to tail_cap
+            size_t first = best_parts.size();
+            int64_t pieces = 0;
+            while (first > 0 && pieces < n_workers) { --first; pieces += mult_of[best_parts[first].seg]; }
+            std::vector<Part> tail;
+            for (size_t k = first; k < best_parts.size(); ++k) cut(tail, best_parts[k].seg, best_parts[k].begin, best_parts[k].len, tail_cap);
+            best_parts.resize(first);
+            best_parts.insert(best_parts.end(), tail.begin(), tail.end());
+            std::stable_sort(best_parts.begin(), best_parts.end(), by_len);
+        }
+    }
+    int64_t slots = 0;
+    for (const Part& q : best_parts) {
+        const int32_t head_node = seg_head[q.seg];
         const int32_t gn = g[head_node];
         for (int32_t h = 0; h < p.num_kv_heads; ++h)
             for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile) {
-                const double uw = unit_weight(gn, l0);
-                int32_t done = 0;
-                --left_runs;
-                while (done < nu) {
-                    if (w < n_workers - 1 && target - load < kItemCost + 0.5 * uw) {
-                        ++w;
-                        t.worker_off[w] = (int32_t)t.items.size();
-                        load = 0.0;
-                        target = target_for(n_workers - w);
-                    }
-                    int32_t take = nu - done;
-                    if (w < n_workers - 1) {
-                        const double room = (target - load - kItemCost) / uw;
-                        take = (int32_t)std::min<double>(take, std::max(1.0, std::floor(room + 0.5)));
-                    }
-                    take = std::min(take, max_run);
-                    Item it;
-                    it.unit_begin = seg_unit_off[s] + done;
-                    it.unit_count = take;
-                    it.kv_head = h;
-                    it.leaf_list_begin = t.node_leaf_off[head_node] + l0;
-                    it.n_leaves_tile = std::min(leaves_per_tile, gn - l0);
-                    it.slot_first = (int32_t)slots;
-                    it.segment = s;
-                    it.reserved = (l0 + leaves_per_tile < gn) ? 1 : 0;   // bit 0: the next tile re-reads these pages
-                    t.items.push_back(it);
-                    slots += it.n_leaves_tile;
-                    load += take * uw + kItemCost;
-                    done += take;
-                    left_cost -= take * uw;
-                    if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
-                }
+                Item it;
+                it.unit_begin = seg_unit_off[q.seg] + q.begin;
+                it.unit_count = q.len;
+                it.kv_head = h;
+                it.leaf_list_begin = t.node_leaf_off[head_node] + l0;
+                it.n_leaves_tile = std::min(leaves_per_tile, gn - l0);
+                it.slot_first = (int32_t)slots;
+                it.segment = q.seg;
+                it.reserved = (l0 + leaves_per_tile < gn) ? 1 : 0;   // bit 0: the next tile re-reads these pages
+                t.items.push_back(it);
+                slots += it.n_leaves_tile;
             }
     }
-    for (int32_t k = w + 1; k <= n_workers; ++k) t.worker_off[k] = (int32_t)t.items.size();
+    if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
     t.n_narrow_items = (int32_t)t.items.size();
+    // static first assignment: warp w starts with item w
+    t.worker_off.assign((size_t)n_workers + 1, 0);
+    for (int32_t k = 0; k <= n_workers; ++k) t.worker_off[k] = std::min(k, t.n_narrow_items);
 
     // ---- wide items: segments whose query group exceeds one narrow tile go to the tcgen05 kernel,
     // one CTA per (piece of the segment, kv head, tile of up to wide_rows query rows)
@@ -275,7 +313,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             }
             return n;
         };
-        int32_t piece = std::max(1, std::min(p.wide_max_units, max_run));
+        int32_t piece = std::max(1, std::min(p.wide_max_units, p.chunk_pages > 0 ? p.chunk_pages : INT32_MAX));
         while (piece > 8 && wide_ctas(piece) < n_sm) piece = std::max(8, piece / 2);
         for (int32_t s = 0; s < n_seg; ++s) {
             const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];

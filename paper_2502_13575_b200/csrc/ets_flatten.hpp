@@ -21,9 +21,10 @@ struct FlattenParams {
     int64_t max_path_entries = 0;
     int64_t max_partial_slots = 0;
     int64_t max_items = 0;
-    int32_t chunk_pages = 0;    // longest run of page slots in one item (0 = unlimited)
+    int32_t chunk_pages = 0;    // longest run of page slots in one item (0 = chosen by the builder; narrow items hold at most 32)
+    int32_t tail_pages = 0;     // longest run in the last pieces of the narrow queue (0 = a third of the chosen length, at least 8)
     int32_t rows_per_item = 16; // query rows (leaves * gqa) one work item covers
-    // cost model of the narrow kernel's work line, in units of one first-read page slot of a tile of
+    // cost model of the narrow kernel's queue, in units of one first-read page slot of a tile of
     // at most 8 query rows
     double cost_item = 2.0;      // opening an item (Q fragments, partial stores)
     double cost_rows16 = 1.2;    // factor for tiles of 9..16 query rows (two MMA column tiles); measured
@@ -31,7 +32,7 @@ struct FlattenParams {
     int32_t wide_rows = 0;      // query rows one wide (tcgen05) item covers; 0 = no wide items
     int32_t wide_min_rows = 17; // smallest query group (in rows) that is treated as wide
     int32_t wide_max_units = 32; // longest page run of a wide item
-    int32_t n_workers = 148 * 8; // warps the attention kernel keeps resident; each gets one piece of the work
+    int32_t n_workers = 148 * 8; // warps the attention kernel keeps resident; they share the queue of narrow items
 };
 
 // One work item, as uploaded to the device (8 x int32).
@@ -50,10 +51,10 @@ struct Tree {
     std::vector<int32_t> free_heap;         // min-heap of free page ids (std::greater)
     // work decomposition
     std::vector<int32_t> unit;              // 4 per unit: page, node, tok0, 0
-    std::vector<Item> items;                // narrow items in worker order, then wide items
+    std::vector<Item> items;                // narrow items in queue order, then wide items
     int32_t n_narrow_items = 0;
     std::vector<int32_t> leaf_slot_off, leaf_slots;   // per (leaf, kv head)
-    std::vector<int32_t> worker_off;                  // items of worker w: [worker_off[w], worker_off[w+1])
+    std::vector<int32_t> worker_off;                  // first item of warp w: [worker_off[w], worker_off[w+1]) (one or none)
     int64_t n_segments = 0, n_chunks = 0, n_partial_slots = 0;
     int32_t chunk_pages_used = 0;
 };

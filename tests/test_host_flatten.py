@@ -225,17 +225,33 @@ def test_work_decomposition_on_configs(name):
 
 
 @pytest.mark.parametrize("name", ["cfg2", "cfg3_ets", "cfg3_diverse", "cfg4", "cfg5b"])
-def test_worker_pieces_are_balanced(name):
-    """The work line is cut into contiguous per-warp pieces of nearly equal cost."""
+def test_narrow_queue_is_ordered_longest_first(name):
+    """Narrow items form a queue: warp w starts with item w and the rest are claimed in index order, so
+    the items are sorted by length (longest first), none is longer than 32 page slots (one lane each),
+    the late ones are short, and the static first assignment is one item per warp."""
     wl = make_workload(name)
     g = wl.geometry
     ctx = host_ctx(g.num_q_heads, g.num_kv_heads, g.head_dim, pages=1 << 15, max_path_entries=1 << 14)
     ctx.tree_build(wl.tree.parent, wl.tree.tokens, wl.tree.leaf_node)
     w = ctx.work_export()
     off, item = w["worker_off"], w["item"]
-    assert off[0] == 0 and off[-1] <= item.shape[0] and np.all(np.diff(off) >= 0)
-    # items after the last worker piece are the wide ones (tiles of groups with more than 16 query rows)
-    assert np.all(item[:off[-1], 4] * g.gqa <= 16)
-    units = np.array([item[off[i]:off[i + 1], 1].sum() for i in range(len(off) - 1)], dtype=np.float64)
-    cost = units + 2.0 * np.diff(off)
-    assert cost.max() <= cost.mean() * 1.15 + 4.0, (cost.max(), cost.mean())
+    n_workers = len(off) - 1
+    n_narrow = ctx.get_stats()["n_narrow_items"]
+    assert off.tolist() == [min(k, n_narrow) for k in range(n_workers + 1)]
+    narrow = item[:n_narrow]
+    # items after the narrow queue are the wide ones (tiles of groups with more than 16 query rows)
+    assert np.all(narrow[:, 4] * g.gqa <= 16)
+    lens = narrow[:, 1]
+    assert lens.max() <= 32 and lens.min() >= 1
+    assert np.all(np.diff(lens) <= 0)
+    if n_narrow > 2 * n_workers:
+        # the pieces claimed last are at most half as long as the longest
+        assert lens[-n_workers // 2:].max() * 2 <= max(lens.max(), 2) + 1
+    # pieces of one (segment part) for all heads and leaf tiles are adjacent in the queue
+    key = [(int(r[6]), int(r[0])) for r in narrow]
+    seen, prev = set(), None
+    for k in key:
+        if k != prev:
+            assert k not in seen
+            seen.add(k)
+            prev = k
