@@ -70,11 +70,12 @@ typedef struct ets_config {
 } ets_config;
 
 /*
- * Byte sizes of the three caller-provided DEVICE buffers for a configuration:
- * the K pool and the V pool (num_layers * pages_per_layer pages each; a page holds
- * page_size tokens of all KV heads, bf16, in a layout private to the library) and the
- * workspace (tables, partial results, staging).  All three must be 1024-byte aligned
- * (any cudaMalloc / torch allocation is).  Pool contents need no initialisation.
+ * Byte sizes of the three caller-provided DEVICE buffers for a configuration: the two pool
+ * buffers (called K pool and V pool for their sizes' sake; together they hold num_layers *
+ * pages_per_layer pages of page_size tokens for all KV heads, bf16, in a layout private to the
+ * library, which spreads the pages over both buffers and keeps a page's K and V next to each
+ * other) and the workspace (tables, partial results, staging).  All three must be 1024-byte
+ * aligned (any cudaMalloc / torch allocation is).  Pool contents need no initialisation.
  */
 int32_t ets_pool_bytes(const ets_config* cfg, size_t* k_bytes, size_t* v_bytes,
                        size_t* workspace_bytes);

@@ -242,7 +242,8 @@ int32_t ets_pool_bytes(const ets_config* cfg, size_t* k_bytes, size_t* v_bytes, 
     std::string why;
     if (!config_ok(cfg, why)) return ETS_ERR_INVALID_ARG;
     if (int32_t rc = config_supported(cfg, why)) return rc;
-    const size_t pool = (size_t)cfg->num_layers * (size_t)cfg->pages_per_layer * cfg->num_kv_heads *
+    // each buffer holds the K and V tiles of every other page (see kv_tile)
+    const size_t pool = (size_t)cfg->num_layers * ets::pool_pairs(cfg->pages_per_layer) * cfg->num_kv_heads * 2 *
                         ets::tile_bytes(cfg->head_dim);
     if (k_bytes) *k_bytes = pool;
     if (v_bytes) *v_bytes = pool;
@@ -269,7 +270,7 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
     c->k_pool = (char*)k_pool;
     c->v_pool = (char*)v_pool;
     c->ws = (char*)workspace;
-    c->layer_pool_bytes = (size_t)cfg->pages_per_layer * cfg->num_kv_heads * ets::tile_bytes(cfg->head_dim);
+    c->layer_pool_bytes = ets::pool_pairs(cfg->pages_per_layer) * cfg->num_kv_heads * 2 * ets::tile_bytes(cfg->head_dim);
     const float sm = cfg->sm_scale != 0.f ? cfg->sm_scale : 1.0f / std::sqrt((float)cfg->head_dim);
     c->scale_log2 = sm * 1.4426950408889634f;
     c->fp.num_kv_heads = cfg->num_kv_heads;

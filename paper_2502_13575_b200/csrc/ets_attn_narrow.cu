@@ -396,15 +396,10 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
                         const uint32_t slot = n_issued % kDepth;
                         const uint32_t bar = bars + slot * 8;
                         const uint32_t dst = ring + slot * 2 * TB;
-                        const size_t off = pool_tile_offset(a.pages_per_layer, page, f_head, TB);
+                        const char* src = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, page, f_head, TB);
                         mbar_expect_tx(bar, 2 * TB);
-                        if (f_reread) {
-                            bulk_g2s(dst, a.k_pool + off, TB, bar);
-                            bulk_g2s(dst + TB, a.v_pool + off, TB, bar);
-                        } else {
-                            bulk_g2s_hint(dst, a.k_pool + off, TB, bar, pol_stream);
-                            bulk_g2s_hint(dst + TB, a.v_pool + off, TB, bar, pol_stream);
-                        }
+                        if (f_reread) bulk_g2s(dst, src, 2 * TB, bar);   // K tile and V tile in one copy
+                        else bulk_g2s_hint(dst, src, 2 * TB, bar, pol_stream);
                     }
                     ++n_issued;
                     return true;

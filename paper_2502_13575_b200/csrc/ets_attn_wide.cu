@@ -232,12 +232,12 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                 const int vl = __shfl_sync(0xffffffffu, valid, src);
                 if (lane == 0) {
                     sh->info[s].valid[n] = vl;
-                    const size_t off = pool_tile_offset(a.pages_per_layer, pg, h, TB);
+                    const char* src = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, pg, h, TB);
                     // raise the byte count first; the producer's single arrival comes after the
                     // last copy of the stage has been started, so the phase cannot end early
                     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"(2 * TB) : "memory");
-                    bulk_g2s(kdst + n * TB, a.k_pool + off, TB, smem_u32(&sh->full[s]));
-                    bulk_g2s(vdst + n * TB, a.v_pool + off, TB, smem_u32(&sh->full[s]));
+                    bulk_g2s(kdst + n * TB, src, TB, smem_u32(&sh->full[s]));
+                    bulk_g2s(vdst + n * TB, src + TB, TB, smem_u32(&sh->full[s]));
                 }
                 ++n;
             }

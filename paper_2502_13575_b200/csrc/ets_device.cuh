@@ -26,10 +26,16 @@ __host__ __device__ inline uint32_t tile_offset(int D, int t, int e) {
            ((((uint32_t)(e & 63) >> 3) ^ r) << 4) + (uint32_t)(e & 7) * 2u;
 }
 
-// Byte offset of the (page, kv head) tile inside one layer's pool: [kv head][page][tile].  Pages of a
-// node usually have consecutive ids, so a worker that streams one head of a node reads contiguous memory.
-__host__ __device__ inline size_t pool_tile_offset(int64_t pages_per_layer, int page, int head, size_t tb) {
-    return ((size_t)head * (size_t)pages_per_layer + (size_t)page) * tb;
+// Where the K tile of a (page, kv head) lives; its V tile follows it directly, so one bulk copy of two
+// tiles brings both (half as many copy requests as one per tile).  Pages alternate between the two
+// pool buffers the caller provides: even page ids in the first, odd ones in the second, and inside a
+// buffer [kv head][page / 2][K tile | V tile].  Pages of a node usually have consecutive ids, so a
+// worker that streams one head of a node reads two contiguous runs.
+__host__ __device__ inline size_t pool_pairs(int64_t pages_per_layer) { return ((size_t)pages_per_layer + 1) / 2; }
+template <typename P>
+__host__ __device__ inline P* kv_tile(P* pool_even, P* pool_odd, int64_t pages_per_layer, int page, int head, size_t tb) {
+    P* pool = (page & 1) ? pool_odd : pool_even;
+    return pool + ((size_t)head * pool_pairs(pages_per_layer) + (size_t)(page >> 1)) * 2 * tb;
 }
 
 struct DevItem {
@@ -48,7 +54,7 @@ struct DecodeArgs {
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
     float* lse;
-    const char* k_pool;            // this layer's pools
+    const char* k_pool;            // this layer's pool buffers (see kv_tile: each holds K and V of half the pages)
     const char* v_pool;
     float2* part_ml;               // [slot][G]  (m in log2 units, l); a slot belongs to one kv head
     float* part_o;                 // [slot][G][D]

@@ -48,9 +48,9 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
             continue;
         }
         const size_t src = ((size_t)(src_off + t) * a.Hkv + h) * a.D + (size_t)c * 8;
-        const size_t dst = pool_tile_offset(a.pages_per_layer, page, h, tb) + tile_offset(a.D, pos % kPageTokens, c * 8);
-        *reinterpret_cast<uint4*>(a.k_pool + dst) = *reinterpret_cast<const uint4*>(a.k_new + src);
-        *reinterpret_cast<uint4*>(a.v_pool + dst) = *reinterpret_cast<const uint4*>(a.v_new + src);
+        char* dst = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, page, h, tb) + tile_offset(a.D, pos % kPageTokens, c * 8);
+        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(a.k_new + src);
+        *reinterpret_cast<uint4*>(dst + tb) = *reinterpret_cast<const uint4*>(a.v_new + src);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) a.node_len[node] = start + n_new;
 }
@@ -78,10 +78,10 @@ __global__ void __launch_bounds__(256) kv_read_kernel(const char* k_pool, const 
         const int h = ci / chunks_per_head;
         const int c = ci % chunks_per_head;
         const int page = pages[t / kPageTokens];
-        const size_t src = pool_tile_offset(pages_per_layer, page, h, tb) + tile_offset(D, t % kPageTokens, c * 8);
+        const char* src = kv_tile(k_pool, v_pool, pages_per_layer, page, h, tb) + tile_offset(D, t % kPageTokens, c * 8);
         const size_t dst = ((size_t)t * Hkv + h) * D + (size_t)c * 8;
-        if (k_out) *reinterpret_cast<uint4*>(k_out + dst) = *reinterpret_cast<const uint4*>(k_pool + src);
-        if (v_out) *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(v_pool + src);
+        if (k_out) *reinterpret_cast<uint4*>(k_out + dst) = *reinterpret_cast<const uint4*>(src);
+        if (v_out) *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(src + tb);
     }
 }
 
@@ -143,8 +143,8 @@ __global__ void __launch_bounds__(kFmaWarps * 32) attn_partial_fma_kernel(Decode
         }
         int valid = a.node_len[un.y] - un.z;
         valid = valid < 0 ? 0 : (valid > kPageTokens ? kPageTokens : valid);
-        const char* kt = a.k_pool + pool_tile_offset(a.pages_per_layer, un.x, h, tb);
-        const char* vt = a.v_pool + pool_tile_offset(a.pages_per_layer, un.x, h, tb);
+        const char* kt = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, un.x, h, tb);
+        const char* vt = kt + tb;
         for (int t = 0; t < valid; ++t) {
             const uint32_t off = tile_offset(D, t, e0);
             float kf[EPL], vf[EPL];

@@ -39,7 +39,8 @@ def test_config_struct_layout_matches_header():
     cfg = ets.make_config(32, 8, 128, max_nodes=10, max_leaves=4, max_path_tokens=64, max_path_entries=40,
                           pages_per_layer=7, device=-1)
     k, v, w = ets.ets_pool_bytes(cfg)
-    assert k == v == 7 * 8 * 16 * 128 * 2
+    # each of the two buffers holds K and V of every other page: ceil(7 / 2) page pairs x 8 heads x 2 tiles
+    assert k == v == 4 * 8 * 2 * 16 * 128 * 2
     bad = ets.make_config(32, 8, 96, max_nodes=10, max_leaves=4, max_path_tokens=64, max_path_entries=40,
                           pages_per_layer=7, device=-1)
     with pytest.raises(ets.EtsError) as e:
