@@ -288,6 +288,7 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
     if (const char* e = std::getenv("ETS_COST_ROWS16")) c->fp.cost_rows16 = std::atof(e);
     if (const char* e = std::getenv("ETS_COST_REREAD")) c->fp.cost_reread = std::atof(e);
     if (const char* e = std::getenv("ETS_TAIL_PAGES")) c->fp.tail_pages = std::atoi(e);
+    if (const char* e = std::getenv("ETS_WIDE_PIECE")) c->fp.wide_piece = std::atoi(e);
     if (!host_only) {
         cudaError_t e = cudaSetDevice(cfg->device);
         cudaDeviceProp prop{};

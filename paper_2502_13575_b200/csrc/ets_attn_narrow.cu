@@ -30,7 +30,10 @@ namespace ets {
 namespace {
 
 constexpr int kWarps = kNarrowWarps;
-constexpr int kDepth = 2;   // measured as fast as 3; 2 leaves shared memory for a wide-kernel CTA on the same SM
+#ifndef ETS_DEPTH
+#define ETS_DEPTH 2
+#endif
+constexpr int kDepth = ETS_DEPTH;   // measured as fast as 3; 2 leaves shared memory for a wide-kernel CTA on the same SM
 constexpr uint32_t kSpinLimit = 1u << 22;
 #ifndef ETS_CLAIM_AHEAD
 #define ETS_CLAIM_AHEAD 6

@@ -232,7 +232,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             const int32_t c = std::min(cand, max_run);
             if (c == prev_c) continue;
             prev_c = c;
-            const int32_t tc = p.tail_pages > 0 ? p.tail_pages : std::max(8, c / 3);
+            const int32_t tc = p.tail_pages > 0 ? p.tail_pages : std::max(8, c / 4);
             int64_t need_slots = 0;
             const double est = estimate(c, tc, need_slots);
             if (need_slots > p.max_partial_slots || need_slots > p.max_items) continue;
@@ -315,6 +315,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         };
         int32_t piece = std::max(1, std::min(p.wide_max_units, p.chunk_pages > 0 ? p.chunk_pages : INT32_MAX));
         while (piece > 8 && wide_ctas(piece) < n_sm) piece = std::max(8, piece / 2);
+        if (p.wide_piece > 0) piece = p.wide_piece;
         for (int32_t s = 0; s < n_seg; ++s) {
             const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
             if (nu == 0 || !is_wide(s)) continue;

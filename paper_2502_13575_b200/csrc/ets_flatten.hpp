@@ -22,7 +22,7 @@ struct FlattenParams {
     int64_t max_partial_slots = 0;
     int64_t max_items = 0;
     int32_t chunk_pages = 0;    // longest run of page slots in one item (0 = chosen by the builder; narrow items hold at most 32)
-    int32_t tail_pages = 0;     // longest run in the last pieces of the narrow queue (0 = a third of the chosen length, at least 8)
+    int32_t tail_pages = 0;     // longest run in the last pieces of the narrow queue (0 = a quarter of the chosen length, at least 8)
     int32_t rows_per_item = 16; // query rows (leaves * gqa) one work item covers
     // cost model of the narrow kernel's queue, in units of one first-read page slot of a tile of
     // at most 8 query rows
@@ -32,6 +32,7 @@ struct FlattenParams {
     int32_t wide_rows = 0;      // query rows one wide (tcgen05) item covers; 0 = no wide items
     int32_t wide_min_rows = 17; // smallest query group (in rows) that is treated as wide
     int32_t wide_max_units = 32; // longest page run of a wide item
+    int32_t wide_piece = 0;      // page run of a wide item (0 = chosen by the builder)
     int32_t n_workers = 148 * 8; // warps the attention kernel keeps resident; they share the queue of narrow items
 };
 
