@@ -41,6 +41,8 @@ def parse_args():
     ap.add_argument("--chunk-pages", type=int, default=None)
     ap.add_argument("--kernel", type=int, default=None)
     ap.add_argument("--wide", type=int, default=None, help="0: no tcgen05 wide-group items")
+    ap.add_argument("--loop-tokens", type=int, default=16,
+                    help="decode iterations of the search-step loop figure (0 = skip it)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time budget of the oracle sample")
@@ -284,7 +286,7 @@ def run_ours(args):
     g, tree = wl.geometry, wl.tree
     layers = args.layers or g.num_layers
     K, W = args.steps, args.warmup
-    headroom = K + W + 2
+    headroom = max(K + W + 2, args.loop_tokens + 4)
     job = DecodeJob(wl, headroom=headroom, device=local, layers=layers, chunk_pages=args.chunk_pages,
                     kernel=args.kernel, wide=args.wide, host_buffers=not args.no_e2e)
     ctx = job.ctx
@@ -377,6 +379,31 @@ def run_ours(args):
         "whole_step_gbs": (u_mean * kv_bytes_tok + qo_bytes) * layers / (ms_step * 1e-3) / 1e9,
     }
 
+    # ---- a search step's decode loop: one flatten, then T decode iterations of every layer through
+    # ets_decode_step (append + attention in one call), no rebuild in between
+    loop = None
+    T = args.loop_tokens
+    if T > 0:
+        job.reset_lengths()
+        job.decode_tokens(2)
+        torch.cuda.synchronize()
+        job.reset_lengths()
+        barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.tree_build(tree.parent, job.cap, tree.leaf_node, keep_pages_of=job.keep,
+                       stream=torch.cuda.current_stream().cuda_stream)
+        job.decode_tokens(T)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_loop = max_over_ranks(e0.elapsed_time(e1))
+        ctx.poll_status()
+        loop = {"tokens": T, "ms_per_token": ms_loop / T, "leaf_tokens_per_s": world * L * T / (ms_loop / 1000.0),
+                "what": "one ets_tree_build, then tokens x layers calls of ets_decode_step; device-resident inputs",
+                "cache": "cold (a token streams more than L2 holds)" if not flush else
+                         "warm: consecutive tokens find this tree's KV in L2"}
+
     # ---- end to end: host buffers through the *_host entry points, result read every step
     e2e = None
     if not args.no_e2e:
@@ -406,6 +433,7 @@ def run_ours(args):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": cfg, "clocks": clocks, "e2e": e2e,
             "gpu_launches": K * layers * launches_per_layer, "roofline": roofline, "cpu_baseline": cpu,
+            "decode_loop": loop,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -194,6 +194,20 @@ int32_t ets_tree_attn_decode_host(ets_ctx* ctx, int32_t layer, const void* q, vo
                                   float* lse, void* cuda_stream);
 
 /*
+ * One decode iteration of one layer in a single call (Section 1: every generated token adds KV state to
+ * its trajectory; Section 3, item 3: later steps reuse it): the new token of live leaf l (row l of
+ * k_new / v_new, bf16 [n_leaves, num_kv_heads, head_dim], DEVICE) is appended to the node the leaf
+ * sits at, then tree-decode attention runs with q / out / lse as in ets_tree_attn_decode, so that
+ * every query sees its own new token.  Lengths grow inside the capacity reserved by
+ * ets_tree_build; no rebuild is needed between iterations.  Same as ets_kv_append with
+ * (leaf_node, all ones) followed by ets_tree_attn_decode.
+ * Errors: those of the two calls; in particular ETS_ERR_INVALID_ARG when two leaves sit at the
+ * same node and ETS_ERR_POOL_EXHAUSTED when a node is full (nothing is appended then).
+ */
+int32_t ets_decode_step(ets_ctx* ctx, int32_t layer, const void* k_new, const void* v_new,
+                        const void* q, void* out, float* lse, void* cuda_stream);
+
+/*
  * Tree-decode attention for callers that cannot allocate device memory (the paper has no
  * counterpart: this is a packaging convenience, not a step of the method).  Same arguments,
  * result and errors as ets_tree_attn_decode (DEVICE pointers), but the partial results between

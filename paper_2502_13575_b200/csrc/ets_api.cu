@@ -143,6 +143,7 @@ struct ets_ctx {
     int desc_next = 0;
     // descriptors of the last short append (at most 8 tokens per node) stay on the device: a decode loop
     // repeats the same (node, count) list for every layer and step
+    std::vector<int32_t> step_ones;   // n_new of ets_decode_step: one token per leaf
     std::vector<int32_t> cache_nodes, cache_nnew;
     bool cache_valid = false;
     cudaStream_t cache_stream = nullptr;
@@ -754,6 +755,20 @@ int32_t ets_tree_attn_decode(ets_ctx* c, int32_t layer, const void* q, void* out
     if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, ETS_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
     ETS_CUDA(c, cudaSetDevice(c->cfg.device));
     if (int32_t jrc = host_join(c, (cudaStream_t)cuda_stream)) return jrc;
+    return decode_impl(c, layer, q, out, lse, (cudaStream_t)cuda_stream);
+}
+
+int32_t ets_decode_step(ets_ctx* c, int32_t layer, const void* k_new, const void* v_new, const void* q, void* out,
+                        float* lse, void* cuda_stream) {
+    if (int32_t rc = decode_check(c, layer, q, out)) return rc;
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, ETS_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
+    const ets::Tree& t = c->tree;
+    if (t.n_leaves == 0) return ETS_OK;
+    if ((int32_t)c->step_ones.size() != t.n_leaves) c->step_ones.assign((size_t)t.n_leaves, 1);
+    // the token of leaf l goes to leaf_node[l]; the append refuses a node that two leaves sit at
+    if (int32_t rc = append_impl(c, layer, t.n_leaves, t.leaf_node.data(), c->step_ones.data(), k_new, v_new, false,
+                                 (cudaStream_t)cuda_stream))
+        return rc;
     return decode_impl(c, layer, q, out, lse, (cudaStream_t)cuda_stream);
 }
 

@@ -60,6 +60,20 @@ def test_small_configs_full_comparison(name, host_api):
     run_and_check(wl.tree, wl.geometry, wl.value_seed, host_api=host_api)
 
 
+def test_forest_of_concurrent_problems_full_comparison():
+    """Eight width-16 problems in one call: one parent array with eight roots, one work list."""
+    wl = make_workload("forest_w16x8")
+    run_and_check(wl.tree, wl.geometry, wl.value_seed)
+
+
+def test_forest_of_width64_problems_sampled_leaves():
+    wl = make_workload("forest_w64x8")
+    L = wl.tree.n_leaves
+    rng = np.random.default_rng(6)
+    subset = sorted(set([0, L - 1] + [int(x) for x in rng.integers(0, L, size=8)]))
+    run_and_check(wl.tree, wl.geometry, wl.value_seed, leaves_subset=subset)
+
+
 @pytest.mark.parametrize("kernel,wide", [(0, 0), (0, 17), (0, 65), (1, 0)])
 def test_every_kernel_choice_agrees_with_the_oracle(kernel, wide):
     """Narrow tensor-core kernel only, tcgen05 kernel from 17 rows, from 65 rows, and the scalar kernel."""
@@ -243,6 +257,65 @@ def test_decode_loop_appends_one_token_per_leaf():
         ref, _ = tree_decode_attention(tree.parent, lengths, tree.leaf_node, full_k, full_v, qb, 8, 2)
         check_close(dev_to_bits(out), ref, f"step {step}")
     ctx.poll_status()
+
+
+def test_decode_step_call_over_a_search_step():
+    """ets_decode_step = append one token per leaf + attend, one call per layer and token: 40 tokens on a
+    width-16 tree with two layers, so every leaf node crosses page boundaries; checked against the oracle at
+    several tokens, and the refusals (full node, two leaves on one node) leave the state untouched."""
+    wl = make_workload("cfg2")
+    tree, g = wl.tree, wl.geometry
+    T, layers = 40, 2
+    cap = tree.tokens.copy()
+    cap[tree.leaf_node] += T
+    ctx = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, tree.parent, cap, tree.leaf_node, num_layers=layers)
+    ctx.tree_build(tree.parent, cap, tree.leaf_node)
+    full = {l: [node_kv_bits(wl.value_seed, n, int(cap[n]), g.num_kv_heads, g.head_dim, l) for n in range(tree.n_nodes)]
+            for l in range(layers)}
+    lengths = tree.tokens.copy()
+    for l in range(layers):
+        fill_layer(ctx, l, [kv[0][:t] for kv, t in zip(full[l], lengths)], [kv[1][:t] for kv, t in zip(full[l], lengths)])
+    from workloads import query_bits
+    from oracle.tree_attention import tree_decode_attention
+    from _harness import check_close
+    rng = np.random.default_rng(9)
+    for tok in range(T):
+        outs = {}
+        for l in range(layers):
+            newk = bits_to_dev(np.stack([full[l][n][0][lengths[n]] for n in tree.leaf_node]))
+            newv = bits_to_dev(np.stack([full[l][n][1][lengths[n]] for n in tree.leaf_node]))
+            qb = query_bits(wl.value_seed, 10 * tok + l, tree.n_leaves, g.num_q_heads, g.head_dim)
+            q = bits_to_dev(qb)
+            out = torch.empty_like(q)
+            ctx.decode_step(l, newk, newv, q, out, None)
+            outs[l] = (qb, out)
+        lengths[tree.leaf_node] += 1
+        if tok in (0, 7, 15, 16, 31, T - 1):
+            torch.cuda.synchronize()
+            subset = sorted(set(int(x) for x in rng.integers(0, tree.n_leaves, size=4)))
+            for l in range(layers):
+                qb, out = outs[l]
+                ref, _ = tree_decode_attention(tree.parent, lengths, tree.leaf_node, [kv[0] for kv in full[l]],
+                                               [kv[1] for kv in full[l]], qb, g.num_q_heads, g.num_kv_heads, leaves=subset)
+                check_close(dev_to_bits(out)[subset], ref[subset], f"token {tok} layer {l}")
+    ctx.poll_status()
+    assert ctx.get_node_len(1).tolist() == lengths.tolist()
+    # every leaf node is full now: one more token is refused and nothing changes
+    q = bits_to_dev(query_bits(wl.value_seed, 999, tree.n_leaves, g.num_q_heads, g.head_dim))
+    out = torch.empty_like(q)
+    one = bits_to_dev(np.zeros((tree.n_leaves, g.num_kv_heads, g.head_dim), np.uint16))
+    with pytest.raises(ets.EtsError) as e:
+        ctx.decode_step(0, one, one, q, out, None)
+    assert e.value.code == ets.ETS_ERR_POOL_EXHAUSTED
+    assert ctx.get_node_len(0).tolist() == lengths.tolist()
+    # two leaves on one node cannot both append to it in one call
+    ctx2 = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, [-1], [64], [0, 0])
+    ctx2.tree_build([-1], [64], [0, 0])
+    q2 = torch.zeros((2, g.num_q_heads, g.head_dim), dtype=torch.bfloat16, device="cuda")
+    kv2 = torch.zeros((2, g.num_kv_heads, g.head_dim), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(ets.EtsError) as e:
+        ctx2.decode_step(0, kv2, kv2, q2, torch.empty_like(q2), None)
+    assert e.value.code == ets.ETS_ERR_INVALID_ARG
 
 
 def test_append_descriptor_reuse_and_long_appends():

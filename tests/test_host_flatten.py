@@ -211,7 +211,7 @@ def test_work_decomposition_covers_everything_once(chunk_pages):
         _check_work(ctx, tree, tree.tokens, hkv, gqa)
 
 
-@pytest.mark.parametrize("name", ["cfg2", "cfg3_ets", "cfg5a", "cfg5c"])
+@pytest.mark.parametrize("name", ["cfg2", "cfg3_ets", "cfg5a", "cfg5c", "forest_w16x8"])
 def test_work_decomposition_on_configs(name):
     wl = make_workload(name)
     g = wl.geometry

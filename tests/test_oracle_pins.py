@@ -91,6 +91,28 @@ def test_leaves_split_at_root_equal_library_attention(hq, hkv, d):
         np.testing.assert_allclose(lse[i], ref_lse.numpy(), rtol=1e-12, atol=1e-13)
 
 
+def test_forest_equals_its_trees_one_at_a_time():
+    """Several problems in one call (a parent array with several roots) give, for every leaf, what the
+    leaf's own tree gives alone: nothing couples the problems."""
+    from workloads.trees import concat_trees
+    rng = np.random.default_rng(44)
+    hq, hkv, d = 4, 2, 8
+    for _ in range(10):
+        trees = [random_small_tree(rng, max_nodes=6, allow_forest=False, allow_empty_nodes=False) for _ in range(3)]
+        parts = [_rand_tree_inputs(rng, t, hq, hkv, d) for t in trees]
+        forest = concat_trees(trees)
+        k = [x for p in parts for x in p[0]]
+        v = [x for p in parts for x in p[1]]
+        q = np.concatenate([p[2] for p in parts])
+        out, lse = tree_decode_attention(forest.parent, forest.tokens, forest.leaf_node, k, v, q, hq, hkv)
+        l0 = 0
+        for t, (kk, vv, qq) in zip(trees, parts):
+            o1, s1 = tree_decode_attention(t.parent, t.tokens, t.leaf_node, kk, vv, qq, hq, hkv)
+            np.testing.assert_array_equal(out[l0:l0 + t.n_leaves], o1)
+            np.testing.assert_array_equal(lse[l0:l0 + t.n_leaves], s1)
+            l0 += t.n_leaves
+
+
 # ---------------------------------------------------------------- P3 node splitting
 def test_splitting_a_node_changes_nothing():
     rng = np.random.default_rng(3)

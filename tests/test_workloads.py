@@ -19,7 +19,29 @@ def test_bf16_rounding_is_nearest_even():
     assert np.array_equal(f32_to_bf16_bits(y), tb)
 
 
-@pytest.mark.parametrize("name", CONFIG_NAMES)
+SINGLE_TREES = [n for n in CONFIG_NAMES if not n.startswith("forest")]
+
+
+@pytest.mark.parametrize("name,width,steps", [("forest_w16x8", 16, 4), ("forest_w64x8", 64, 8)])
+def test_forest_shapes(name, width, steps):
+    """Eight concurrent problems in one parent array: eight roots, eight times the width, no edge between problems."""
+    t = make_workload(name).tree
+    assert int((t.parent == -1).sum()) == 8 and t.n_leaves == 8 * width
+    assert all(-1 <= int(p) < i for i, p in enumerate(t.parent))
+    root_of = np.arange(t.n_nodes)
+    for i, p in enumerate(t.parent):
+        if p >= 0:
+            root_of[i] = root_of[p]
+    roots = root_of[t.leaf_node]
+    assert [int((roots == r).sum()) for r in np.unique(roots)] == [width] * 8
+    st = tree_stats(t)
+    assert st["max_depth"] == steps + 1 and st["path_nodes"] == 8 * width * (steps + 1)
+    # the problems differ from one another
+    sizes = [int(t.tokens[root_of == r].sum()) for r in np.unique(root_of)]
+    assert len(set(sizes)) == 8
+
+
+@pytest.mark.parametrize("name", SINGLE_TREES)
 def test_tree_shapes(name):
     wl = make_workload(name)
     t = wl.tree

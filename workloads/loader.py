@@ -154,6 +154,19 @@ class DecodeJob:
             c.tree_attn_decode(layer, p["q"][layer], p["out"][layer], None, stream=stream)
         self.steps_done += 1
 
+    def decode_tokens(self, n_tokens: int):
+        """A search step's decode loop: n_tokens iterations of (one new token per leaf, attention) over every
+        layer through ets_decode_step, with no tree rebuild in between.  Asynchronous."""
+        if self.steps_done + n_tokens > self.headroom:
+            raise RuntimeError("step budget of this job exhausted; call reset_lengths()")
+        c = self.ctx
+        p = self._pointers()
+        stream = self.torch.cuda.current_stream().cuda_stream
+        for _ in range(n_tokens):
+            for layer in range(self.layers):
+                c.decode_step(layer, p["nk"][layer], p["nv"][layer], p["q"][layer], p["out"][layer], None, stream=stream)
+        self.steps_done += n_tokens
+
     def step_host(self):
         """Host buffers in, host buffers out, through the *_host entry points; the caller
         synchronises to read the result."""

@@ -76,6 +76,8 @@ CONFIG_NAMES = (
     "cfg5a",
     "cfg5b",
     "cfg5c",
+    "forest_w16x8",
+    "forest_w64x8",
 )
 
 _GEOM = {
@@ -189,6 +191,18 @@ def _keep_fraction(seed: int, root_tokens: int, steps: int, width: int, keep: in
     return _drop_dead_and_renumber(parent, tokens, live)
 
 
+def concat_trees(trees: List[Tree]) -> Tree:
+    """Several independent problems as one forest: node and leaf lists are concatenated, parents shifted."""
+    parent, tokens, leaves, off = [], [], [], 0
+    for t in trees:
+        parent.append(np.where(t.parent >= 0, t.parent + off, -1))
+        tokens.append(t.tokens)
+        leaves.append(t.leaf_node + off)
+        off += t.n_nodes
+    return Tree(np.concatenate(parent).astype(np.int32), np.concatenate(tokens).astype(np.int32),
+                np.concatenate(leaves).astype(np.int32))
+
+
 def _unique_tokens(tree: Tree) -> int:
     return int(tree.tokens.astype(np.int64).sum())
 
@@ -287,6 +301,19 @@ def make_workload(name: str) -> Workload:
         cid, variant = 5, 2
         tree, attempt = _branch_and_prune(TOPOLOGY_SEED_BASE + cid + 20, 1024, 6, 128, 128, 128)
         notes["attempt"] = attempt
+    elif name == "forest_w16x8":
+        # eight concurrent problems (the paper serves 4 to 32 at a time, Section 5.3), each a width-16
+        # tree drawn like cfg2 with its own seed; one parent array with eight roots
+        cid, variant = 2, 5
+        tree = concat_trees([_branch_and_prune(TOPOLOGY_SEED_BASE + cid + 10 * variant + 100 * (i + 1), 256, 4, 16, 64, 128)[0]
+                             for i in range(8)])
+        notes["problems"] = 8
+    elif name == "forest_w64x8":
+        # eight concurrent width-64 problems, each drawn like the ETS-like tree of cfg3 (keep 36 of 64)
+        cid, variant = 3, 5
+        tree = concat_trees([_keep_fraction(TOPOLOGY_SEED_BASE + cid + 10 * variant + 100 * (i + 1), 512, 8, 64, 36, 64, 128)
+                             for i in range(8)])
+        notes["problems"] = 8
     else:
         raise KeyError(f"unknown workload {name!r}; choose from {CONFIG_NAMES}")
     wl = Workload(
