@@ -22,11 +22,31 @@ __device__ __forceinline__ void merge_row(const DecodeArgs& a, int leaf, int hea
     float acc[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+    constexpr int kEarly = 8;   // o rows whose loads are started together with the (m, l) loads
     for (int base = s0; base < s1; base += 32) {
         const int cnt = min(32, s1 - base);
         const int my_slot = lane < cnt ? a.leaf_slots[base + lane] : -1;
         float2 ml = make_float2(-INFINITY, 0.f);
         if (my_slot >= 0) ml = a.part_ml[(size_t)my_slot * G + sub];
+        // the addresses of the o rows depend on the slot ids only: start the first loads now, so that
+        // they travel together with the (m, l) pairs instead of after the reduction over them
+        float early[kEarly][EPL];
+#pragma unroll
+        for (int j = 0; j < kEarly; ++j) {
+            const int slot = __shfl_sync(0xffffffffu, my_slot, j);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) early[j][e] = 0.f;
+            if (j < cnt) {
+                const float* po = a.part_o + ((size_t)slot * G + sub) * D + lane * EPL;
+                if constexpr (EPL == 4) {
+                    const float4 v = *reinterpret_cast<const float4*>(po);
+                    early[j][0] = v.x; early[j][1] = v.y; early[j][2] = v.z; early[j][3] = v.w;
+                } else {
+                    const float2 v = *reinterpret_cast<const float2*>(po);
+                    early[j][0] = v.x; early[j][1] = v.y;
+                }
+            }
+        }
         float bm = ml.y > 0.f ? ml.x : -INFINITY;
 #pragma unroll
         for (int x = 16; x > 0; x >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, x));
@@ -40,8 +60,16 @@ __device__ __forceinline__ void merge_row(const DecodeArgs& a, int leaf, int hea
 #pragma unroll
         for (int e = 0; e < EPL; ++e) acc[e] *= corr;
         ms = mn;
+#pragma unroll
+        for (int j = 0; j < kEarly; ++j) {
+            const float w = __shfl_sync(0xffffffffu, wgt, j);
+            if (j < cnt && w > 0.f) {
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) acc[e] += w * early[j][e];
+            }
+        }
 #pragma unroll 8
-        for (int j = 0; j < cnt; ++j) {
+        for (int j = kEarly; j < cnt; ++j) {
             const int slot = __shfl_sync(0xffffffffu, my_slot, j);
             const float w = __shfl_sync(0xffffffffu, wgt, j);
             const float* po = a.part_o + ((size_t)slot * G + sub) * D + lane * EPL;
