@@ -25,6 +25,11 @@ What it defines (and where each definition comes from):
   invariants (pages partition, group/path duality, hand-worked small tree in
   tests/golden/).
 
+* ``selection`` - the selection step the paper is about (Section 4, Appendix B): REBASE weights
+  (Eq. 1 / Eq. 3), the objective of Eq. 4 and its maximiser by enumeration of leaf subsets.
+  Pinned by tests/test_oracle_selection.py (weights and objective values worked by hand from
+  the equations, the lambda = 0 and large-lambda closed forms, monotonicity, relabelling).
+
 Numerical parity with values printed in the paper is unpinned by construction: the
 paper prints none for this path.  Parity is to the definition.
 """
