@@ -232,6 +232,42 @@ int32_t ets_tree_attn_decode_static(ets_ctx* ctx, int32_t layer, const void* q, 
 int32_t ets_kv_read_debug(ets_ctx* ctx, int32_t layer, int32_t node, void* k_out, void* v_out,
                           void* cuda_stream);
 
+/*
+ * Selection step of the search (host only, no context needed).  Section 4 and Appendix B: from the
+ * rewards of the live trajectories compute the REBASE weights W_i (Eq. 1: highest reward first,
+ * W_i = ceil(N_i exp(R_i / T_R) / sum over the trajectories not served yet), N_1 = width and
+ * N_{i+1} = N_i - W_i), then keep the set S of trajectories that maximises Eq. 4,
+ *     sum_{i in S} W_i / sum_i W_i  -  lambda_b |V_S| / |V_A|  +  lambda_d |C_S| / |C_A|,    |S| >= 1,
+ * where V_S are the nodes with a kept trajectory at or below them, V_A all n_nodes nodes, C_S the
+ * clusters with a kept member and C_A all clusters (a cluster counts once any member is kept, as the
+ * text of Appendix B.2 says), and finally hand the width out again over the kept trajectories
+ * (Eq. 3).  The maximiser is found exactly by branch and bound over the tree (the paper calls a
+ * general ILP solver); among equal optima the choice is unspecified.
+ *   parent[n_nodes], leaf_node[n_leaves]   HOST, as in ets_tree_build: trajectory i ends at leaf_node[i]
+ *   reward[n_leaves]                       HOST fp64, finite
+ *   cluster[n_leaves]                      HOST, nullable: cluster label of each trajectory, negative = none
+ *   weight, keep, continuations [n_leaves], node_kept [n_nodes]   HOST outputs, each nullable:
+ *                                          W_i, 0/1, W'_i (0 where pruned), 0/1 per node of the tree
+ *   result->proven_optimal                 0 when params->node_limit (0 = 2^20 search nodes) ran out:
+ *                                          `keep` is then the best set found
+ * Errors: ETS_ERR_INVALID_ARG (null array, width <= 0, temperature <= 0, negative lambda, non-finite
+ * reward), ETS_ERR_BAD_TREE.
+ */
+typedef struct ets_select_params {
+    double temperature, lambda_b, lambda_d;
+    int32_t width, reserved;
+    int64_t node_limit;
+} ets_select_params;
+typedef struct ets_select_result {
+    double objective;
+    int64_t nodes_explored;
+    int32_t proven_optimal, n_kept, n_nodes_kept, reserved;
+} ets_select_result;
+int32_t ets_select(int32_t n_nodes, const int32_t* parent, int32_t n_leaves, const int32_t* leaf_node,
+                   const double* reward, const int32_t* cluster, const ets_select_params* params,
+                   int32_t* weight, int32_t* keep, int32_t* continuations, int32_t* node_kept,
+                   ets_select_result* result);
+
 /* Counters of the current tree.  "KV size" follows Section 3: the unique KV state of the tree. */
 typedef struct ets_stats {
     int64_t n_nodes, n_leaves;

@@ -81,6 +81,16 @@ class ets_stats(C.Structure):
         "attended_tokens", "n_narrow_items")]
 
 
+class ets_select_params(C.Structure):
+    _fields_ = [("temperature", C.c_double), ("lambda_b", C.c_double), ("lambda_d", C.c_double),
+                ("width", C.c_int32), ("reserved", C.c_int32), ("node_limit", C.c_int64)]
+
+
+class ets_select_result(C.Structure):
+    _fields_ = [("objective", C.c_double), ("nodes_explored", C.c_int64), ("proven_optimal", C.c_int32),
+                ("n_kept", C.c_int32), ("n_nodes_kept", C.c_int32), ("reserved", C.c_int32)]
+
+
 # every symbol include/ets.h declares, with its C signature
 _SIGNATURES = {
     "ets_pool_bytes": (C.c_int32, [C.POINTER(ets_config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
@@ -93,6 +103,8 @@ _SIGNATURES = {
     "ets_kv_append_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, _I32P, _I32P, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_get_node_len": (C.c_int32, [C.c_void_p, C.c_int32, _I32P]),
     "ets_tree_attn_decode": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ets_select": (C.c_int32, [C.c_int32, _I32P, C.c_int32, _I32P, C.POINTER(C.c_double), _I32P,
+                               C.POINTER(ets_select_params), _I32P, _I32P, _I32P, _I32P, C.POINTER(ets_select_result)]),
     "ets_decode_step": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p]),
     "ets_tree_attn_decode_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -171,6 +183,27 @@ def make_config(num_q_heads: int, num_kv_heads: int, head_dim: int, *, num_layer
 
 def ets_version() -> str:
     return lib.ets_version().decode()
+
+
+def ets_select(parent, leaf_node, reward, cluster=None, *, width: int, temperature: float = 0.2,
+               lambda_b: float = 0.0, lambda_d: float = 0.0, node_limit: int = 0) -> Dict[str, object]:
+    """Selection step on the host (same name as the C call): REBASE weights, the kept set, the
+    continuations per kept trajectory and the kept nodes of the tree."""
+    parent, leaves = _i32(parent), _i32(leaf_node)
+    r = np.ascontiguousarray(reward, dtype=np.float64)
+    cl = None if cluster is None else _i32(cluster)
+    prm = ets_select_params(temperature, lambda_b, lambda_d, width, 0, node_limit)
+    res = ets_select_result()
+    L, n = leaves.shape[0], parent.shape[0]
+    weight, keep, cont, nodes = (np.zeros(L, np.int32), np.zeros(L, np.int32), np.zeros(L, np.int32),
+                                 np.zeros(n, np.int32))
+    rc = lib.ets_select(n, _p(parent), L, _p(leaves), r.ctypes.data_as(C.POINTER(C.c_double)), _p(cl), C.byref(prm),
+                        _p(weight), _p(keep), _p(cont), _p(nodes), C.byref(res))
+    if rc != ETS_OK:
+        raise EtsError(rc, "ets_select")
+    return {"weight": weight, "keep": keep, "continuations": cont, "node_kept": nodes, "objective": res.objective,
+            "proven_optimal": bool(res.proven_optimal), "nodes_explored": int(res.nodes_explored),
+            "n_kept": int(res.n_kept), "n_nodes_kept": int(res.n_nodes_kept)}
 
 
 def ets_pool_bytes(cfg: ets_config):
