@@ -318,6 +318,48 @@ def test_decode_step_call_over_a_search_step():
     assert e.value.code == ets.ETS_ERR_INVALID_ARG
 
 
+def test_prune_with_ets_select_then_decode_on_the_kept_tree():
+    """A search step end to end: the selection step prunes trajectories, the tree is rebuilt from the kept
+    nodes with their pages (and so their KV) carried over, and decode attention on the smaller tree equals
+    the oracle on that tree.  The kept tree's KV is what the next decode steps stream."""
+    wl = make_workload("cfg3_diverse")
+    tree, g = wl.tree, wl.geometry
+    ctx = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, tree.parent, tree.tokens, tree.leaf_node)
+    ctx.tree_build(tree.parent, tree.tokens, tree.leaf_node)
+    ks, vs = node_values(tree, g, wl.value_seed, 0)
+    fill_layer(ctx, 0, ks, vs)
+    rng = np.random.default_rng(12)
+    reward = rng.random(tree.n_leaves)
+    cluster = rng.integers(0, 6, size=tree.n_leaves)
+    sel = ets.ets_select(tree.parent, tree.leaf_node, reward, cluster, width=64, temperature=0.2, lambda_b=1.0, lambda_d=0.5)
+    assert sel["proven_optimal"] and 1 <= sel["n_kept"] < tree.n_leaves
+    kept_nodes = np.flatnonzero(sel["node_kept"])
+    new_id = -np.ones(tree.n_nodes, np.int64)
+    new_id[kept_nodes] = np.arange(kept_nodes.shape[0])
+    parent2 = np.array([new_id[tree.parent[v]] if tree.parent[v] >= 0 else -1 for v in kept_nodes], np.int32)
+    tokens2 = tree.tokens[kept_nodes].astype(np.int32)
+    kept_leaves = np.flatnonzero(sel["keep"])
+    leaves2 = new_id[tree.leaf_node[kept_leaves]].astype(np.int32)
+    before = ctx.get_stats()
+    ctx.tree_build(parent2, tokens2, leaves2, keep_pages_of=kept_nodes.astype(np.int32))
+    after = ctx.get_stats()
+    assert after["unique_tokens"] == int(tokens2.sum()) < before["unique_tokens"]
+    assert after["pages_free"] > before["pages_free"]
+    from workloads import query_bits
+    from oracle.tree_attention import tree_decode_attention
+    from _harness import check_close
+    qb = query_bits(wl.value_seed, 3, leaves2.shape[0], g.num_q_heads, g.head_dim)
+    q = bits_to_dev(qb)
+    out = torch.empty_like(q)
+    ctx.tree_attn_decode(0, q, out, None)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    subset = sorted(set([0, leaves2.shape[0] - 1] + [int(x) for x in rng.integers(0, leaves2.shape[0], size=4)]))
+    ref, _ = tree_decode_attention(parent2, tokens2, leaves2, [ks[v] for v in kept_nodes], [vs[v] for v in kept_nodes], qb,
+                                   g.num_q_heads, g.num_kv_heads, leaves=subset)
+    check_close(dev_to_bits(out)[subset], ref[subset], "kept tree")
+
+
 def test_append_descriptor_reuse_and_long_appends():
     """Short appends (at most 8 tokens per node) keep their (node, count) list on the device and read the
     start position from the device-side lengths; longer ones carry the start in the descriptor.  Mix
