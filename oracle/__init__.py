@@ -16,6 +16,11 @@ What it defines (and where each definition comes from):
   tree, independent sequences vs. a library attention routine, node splitting, brute
   force, closed forms, permutation invariance, convexity, duplicate leaves).
 
+* ``tree_attention.tree_prefill_attention`` - the same definition for the tokens of a newly
+  generated step (what scoring or prefilling a step computes): ancestors whole, the own step up
+  to a per-query limit, i.e. causal inside the step.  Pinned by a library causal-attention
+  routine on a root step, by the decode oracle on truncated trees, and by an explicit mask.
+
 * ``tree_attention.merge_partials`` - the log-sum-exp combination of per-node softmax
   partials, written out in fp64 only so that tests can show it equals the direct
   definition.  The direct function above never calls it.

@@ -93,6 +93,46 @@ def tree_decode_attention(parent: Sequence[int], node_len: Sequence[int],
     return out, lse
 
 
+def tree_prefill_attention(parent: Sequence[int], node_len: Sequence[int], leaf_node: Sequence[int],
+                           leaf_limit: Sequence[int],
+                           k_nodes: Sequence[np.ndarray], v_nodes: Sequence[np.ndarray],
+                           q_bits: np.ndarray, num_q_heads: int, num_kv_heads: int,
+                           sm_scale: Optional[float] = None,
+                           leaves: Optional[Sequence[int]] = None
+                           ) -> Tuple[np.ndarray, np.ndarray]:
+    """Attention of the tokens of a newly generated step (what the reward model and the prefill of a step
+    compute; the paper scores every new step with a PRM, Section 5.1).  Every query is a "leaf" sitting at
+    its step's node: it sees all tokens of the node's ancestors (their KV is shared, Section 4.1) and the
+    first leaf_limit[l] tokens of its own node, i.e. the causal mask inside the step: the j-th of the T new
+    tokens of a node that now holds `len` tokens has limit len - T + j + 1.  The paper prints no formula;
+    this is textbook causal softmax attention over the trajectory, evaluated on the materialised sequence.
+    With leaf_limit[l] = node_len[leaf_node[l]] it is tree_decode_attention."""
+    n_leaves = len(leaf_node)
+    head_dim = int(q_bits.shape[-1])
+    group = num_q_heads // num_kv_heads
+    scale = (1.0 / math.sqrt(head_dim)) if sm_scale is None else float(sm_scale)
+    q = bf16_bits_to_f64(q_bits)
+    out = np.full((n_leaves, num_q_heads, head_dim), np.nan, dtype=np.float64)
+    lse = np.full((n_leaves, num_q_heads), np.nan, dtype=np.float64)
+    for l in (range(n_leaves) if leaves is None else leaves):
+        own = int(leaf_node[l])
+        lim = int(leaf_limit[l])
+        if not 0 <= lim <= int(node_len[own]):
+            raise ValueError("leaf_limit must lie in [0, node_len of the leaf's node]")
+        seen = list(node_len)
+        seen[own] = lim                      # ancestors whole, own node up to the limit
+        k_path, v_path = materialise_path(parent, seen, own, k_nodes, v_nodes)
+        for a in range(num_q_heads):
+            h = a // group
+            s = scale * (k_path[:, h, :] @ q[l, a, :])
+            m = s.max()
+            w = np.exp(s - m)
+            z = w.sum()
+            out[l, a, :] = (w @ v_path[:, h, :]) / z
+            lse[l, a] = m + math.log(z)
+    return out, lse
+
+
 def node_partial(k: np.ndarray, v: np.ndarray, q: np.ndarray, scale: float
                  ) -> Tuple[float, float, np.ndarray]:
     """Softmax partial of one query over one block of tokens: (m, l, o~) with

@@ -91,6 +91,77 @@ def test_leaves_split_at_root_equal_library_attention(hq, hkv, d):
         np.testing.assert_allclose(lse[i], ref_lse.numpy(), rtol=1e-12, atol=1e-13)
 
 
+def test_prefill_of_a_root_step_is_causal_self_attention():
+    """A step at the root (no ancestors) whose T tokens are all new: the prefill oracle must equal a
+    library causal attention routine on that one sequence."""
+    import torch
+    from oracle.tree_attention import tree_prefill_attention
+    rng = np.random.default_rng(61)
+    hq, hkv, d, T = 4, 2, 8, 11
+    g = hq // hkv
+    k = [_rand_bits(rng, (T, hkv, d))]
+    v = [_rand_bits(rng, (T, hkv, d))]
+    q = _rand_bits(rng, (T, hq, d))
+    out, lse = tree_prefill_attention([-1], [T], [0] * T, list(range(1, T + 1)), k, v, q, hq, hkv)
+    kt = torch.from_numpy(bf16_bits_to_f32(k[0])).double().permute(1, 0, 2).repeat_interleave(g, dim=0)   # [hq, T, d]
+    vt = torch.from_numpy(bf16_bits_to_f32(v[0])).double().permute(1, 0, 2).repeat_interleave(g, dim=0)
+    qt = torch.from_numpy(bf16_bits_to_f32(q)).double().permute(1, 0, 2)                                  # [hq, T, d]
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, is_causal=True)                    # [hq, T, d]
+    np.testing.assert_allclose(out, ref.permute(1, 0, 2).numpy(), rtol=1e-12, atol=1e-13)
+
+
+def test_prefill_sees_ancestors_whole_and_own_step_causally():
+    """Against the decode oracle: the query with limit t on node n equals a decode query on the tree in which
+    n holds only its first t tokens; with the limit at the node's length it is the decode query itself; and
+    (brute force) with an explicit mask over the concatenated path."""
+    from oracle.tree_attention import tree_prefill_attention
+    rng = np.random.default_rng(62)
+    hq, hkv, d = 4, 2, 8
+    done = 0
+    while done < 25:
+        tree = random_small_tree(rng, max_nodes=8, allow_forest=True, allow_empty_nodes=True)
+        k, v, _ = _rand_tree_inputs(rng, tree, hq, hkv, d)
+        leaf_nodes = [int(n) for n in tree.leaf_node if tree.tokens[n] > 0]
+        if not leaf_nodes:
+            continue
+        leaves, limits = [], []
+        for n in leaf_nodes:
+            for t in sorted(set(int(x) for x in rng.integers(1, tree.tokens[n] + 1, size=2))):
+                leaves.append(n)
+                limits.append(t)
+        q = _rand_bits(rng, (len(leaves), hq, d))
+        out, lse = tree_prefill_attention(tree.parent, tree.tokens, leaves, limits, k, v, q, hq, hkv)
+        for i, (n, t) in enumerate(zip(leaves, limits)):
+            cut = tree.tokens.copy()
+            cut[n] = t
+            o1, l1 = tree_decode_attention(tree.parent, cut, [n], k, v, q[i:i + 1], hq, hkv)
+            np.testing.assert_array_equal(out[i], o1[0])
+            np.testing.assert_array_equal(lse[i], l1[0])
+            # explicit mask over the whole path with the full node
+            path = []
+            x = n
+            while x >= 0:
+                path.append(x)
+                x = int(tree.parent[x])
+            path.reverse()
+            kk = np.concatenate([bf16_bits_to_f32(k[p][:tree.tokens[p]]).astype(np.float64) for p in path])
+            vv = np.concatenate([bf16_bits_to_f32(v[p][:tree.tokens[p]]).astype(np.float64) for p in path])
+            visible = np.concatenate([np.ones(int(tree.tokens[p]), bool) if p != n else np.arange(int(tree.tokens[p])) < t
+                                      for p in path])
+            qq = bf16_bits_to_f32(q[i]).astype(np.float64)
+            for a in range(hq):
+                sc = (kk[:, a // (hq // hkv), :] @ qq[a]) / math.sqrt(d)
+                wgt = np.where(visible, np.exp(sc), 0.0)
+                np.testing.assert_allclose(out[i, a], (wgt @ vv[:, a // (hq // hkv), :]) / wgt.sum(), rtol=1e-11, atol=1e-12)
+        full = [int(tree.tokens[n]) for n in leaf_nodes]
+        qf = _rand_bits(rng, (len(leaf_nodes), hq, d))
+        a1, b1 = tree_prefill_attention(tree.parent, tree.tokens, leaf_nodes, full, k, v, qf, hq, hkv)
+        a2, b2 = tree_decode_attention(tree.parent, tree.tokens, leaf_nodes, k, v, qf, hq, hkv)
+        np.testing.assert_array_equal(a1, a2)
+        np.testing.assert_array_equal(b1, b2)
+        done += 1
+
+
 def test_forest_equals_its_trees_one_at_a_time():
     """Several problems in one call (a parent array with several roots) give, for every leaf, what the
     leaf's own tree gives alone: nothing couples the problems."""
