@@ -75,7 +75,8 @@ typedef struct ets_config {
  * pages_per_layer pages of page_size tokens for all KV heads, bf16, in a layout private to the
  * library, which spreads the pages over both buffers and keeps a page's K and V next to each
  * other) and the workspace (tables, partial results, staging).  All three must be 1024-byte
- * aligned (any cudaMalloc / torch allocation is).  Pool contents need no initialisation.
+ * aligned (cudaMalloc blocks are; a caching allocator may hand out small blocks on 512-byte
+ * boundaries).  Pool contents need no initialisation.
  */
 int32_t ets_pool_bytes(const ets_config* cfg, size_t* k_bytes, size_t* v_bytes,
                        size_t* workspace_bytes);
@@ -206,6 +207,24 @@ int32_t ets_tree_attn_decode_host(ets_ctx* ctx, int32_t layer, const void* q, vo
  */
 int32_t ets_decode_step(ets_ctx* ctx, int32_t layer, const void* k_new, const void* v_new,
                         const void* q, void* out, float* lse, void* cuda_stream);
+
+/*
+ * Attention of the tokens of newly generated steps: what prefilling a step, or scoring it with the
+ * reward model, computes (Section 5.1: every new step is scored by a PRM; Section 4.1: the steps of a
+ * trajectory share their ancestors' KV).  Every query token is a "leaf" sitting at its step's node
+ * (ets_tree_build accepts many leaves on one node): it attends to all tokens of the node's ancestors
+ * and to the first leaf_limit[l] tokens of its own node, i.e. causally inside the step.  For the j-th of
+ * T new tokens of a node that now holds len tokens, leaf_limit = len - T + j + 1; with leaf_limit =
+ * len the call equals ets_tree_attn_decode.  The step's K/V must have been appended before.
+ *   q, out, lse   as in ets_tree_attn_decode, one row per leaf (DEVICE)
+ *   leaf_limit    DEVICE int32 [n_leaves]; values are clipped to [0, current length of the node]
+ * Query groups of more than 16 rows (leaves * Hq/Hkv) that the last build classed as wide run on the
+ * tcgen05 kernel, the rest on the scalar kernel: build the tree with ETS_OPT_WIDE set to 17 so that every
+ * dense group takes the tensor cores.  A query that sees no token yields zeros and lse = -inf.
+ * Errors: as ets_tree_attn_decode.
+ */
+int32_t ets_tree_attn_prefill(ets_ctx* ctx, int32_t layer, const void* q, const int32_t* leaf_limit,
+                              void* out, float* lse, void* cuda_stream);
 
 /*
  * Tree-decode attention for callers that cannot allocate device memory (the paper has no

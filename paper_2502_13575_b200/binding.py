@@ -105,6 +105,8 @@ _SIGNATURES = {
     "ets_tree_attn_decode": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_select": (C.c_int32, [C.c_int32, _I32P, C.c_int32, _I32P, C.POINTER(C.c_double), _I32P,
                                C.POINTER(ets_select_params), _I32P, _I32P, _I32P, _I32P, C.POINTER(ets_select_result)]),
+    "ets_tree_attn_prefill": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p]),
     "ets_decode_step": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p]),
     "ets_tree_attn_decode_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -226,9 +228,11 @@ class EtsContext:
         if cfg.device >= 0:
             import torch
             dev = torch.device("cuda", cfg.device)
-            self.k_pool = torch.empty(kb, dtype=torch.uint8, device=dev)
-            self.v_pool = torch.empty(vb, dtype=torch.uint8, device=dev)
-            self.workspace = torch.empty(wb, dtype=torch.uint8, device=dev)
+            def aligned(nbytes):   # torch hands out small blocks on 512-byte boundaries; the library wants 1024
+                t = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+                off = (-t.data_ptr()) % 1024
+                return t[off:off + nbytes]
+            self.k_pool, self.v_pool, self.workspace = aligned(kb), aligned(vb), aligned(wb)
         rc = lib.ets_create(C.byref(cfg), _dev_ptr(self.k_pool), _dev_ptr(self.v_pool),
                             _dev_ptr(self.workspace), C.byref(self._h))
         if rc != ETS_OK:
@@ -309,6 +313,10 @@ class EtsContext:
     def tree_attn_decode(self, layer: int, q, out, lse=None, stream=None):
         self._check(lib.ets_tree_attn_decode(self._h, layer, _dev_ptr(q), _dev_ptr(out), _dev_ptr(lse),
                                              _stream_ptr(stream)))
+
+    def tree_attn_prefill(self, layer: int, q, leaf_limit, out, lse=None, stream=None):
+        self._check(lib.ets_tree_attn_prefill(self._h, layer, _dev_ptr(q), _dev_ptr(leaf_limit), _dev_ptr(out),
+                                              _dev_ptr(lse), _stream_ptr(stream)))
 
     def decode_step(self, layer: int, k_new, v_new, q, out, lse=None, stream=None):
         self._check(lib.ets_decode_step(self._h, layer, _dev_ptr(k_new), _dev_ptr(v_new), _dev_ptr(q), _dev_ptr(out),

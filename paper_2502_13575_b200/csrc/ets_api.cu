@@ -84,6 +84,7 @@ Layout make_layout(const ets_config* c) {
     blob += align_up(((size_t)c->max_nodes + 1) * 4, 256);          // node_page_off
     blob += align_up((size_t)c->pages_per_layer * 4, 256);          // page_ids
     blob += align_up((size_t)c->max_path_entries * 4, 256);         // node_leaves
+    blob += align_up((size_t)c->max_leaves * 4, 256);               // leaf_node
     blob += align_up(((size_t)c->max_leaves * c->num_kv_heads + 1) * 4, 256);  // leaf_slot_off
     blob += align_up((size_t)L.max_partial_slots * 4, 256);         // leaf_slots
     blob += align_up((size_t)c->num_layers * c->max_nodes * 4, 256);  // node_len
@@ -111,7 +112,7 @@ Layout make_layout(const ets_config* c) {
 }
 
 struct BlobOffsets {  // offsets of the packed tables of the current tree inside the device blob
-    size_t units, items, node_page_off, page_ids, node_leaves, leaf_slot_off, leaf_slots, node_len, total;
+    size_t units, items, node_page_off, page_ids, node_leaves, leaf_node, leaf_slot_off, leaf_slots, node_len, total;
     int32_t len_stride;
 };
 
@@ -205,6 +206,7 @@ BlobOffsets pack_offsets(const ets_ctx* c, const ets::Tree& t) {
     b.node_page_off = take(t.node_page_off.size() * 4);
     b.page_ids = take(t.page_ids.size() * 4);
     b.node_leaves = take(t.node_leaves.size() * 4);
+    b.leaf_node = take(t.leaf_node.size() * 4);
     b.leaf_slot_off = take(t.leaf_slot_off.size() * 4);
     b.leaf_slots = take(t.leaf_slots.size() * 4);
     b.len_stride = t.n_nodes > 0 ? t.n_nodes : 1;
@@ -220,6 +222,7 @@ void pack_blob(const ets_ctx* c, const ets::Tree& t, const BlobOffsets& b, char*
     put(b.node_page_off, t.node_page_off.data(), t.node_page_off.size() * 4);
     put(b.page_ids, t.page_ids.data(), t.page_ids.size() * 4);
     put(b.node_leaves, t.node_leaves.data(), t.node_leaves.size() * 4);
+    put(b.leaf_node, t.leaf_node.data(), t.leaf_node.size() * 4);
     put(b.leaf_slot_off, t.leaf_slot_off.data(), t.leaf_slot_off.size() * 4);
     put(b.leaf_slots, t.leaf_slots.data(), t.leaf_slots.size() * 4);
     for (int l = 0; l < c->cfg.num_layers; ++l)
@@ -654,7 +657,7 @@ static int32_t launch_attention(ets_ctx* c, const ets::DecodeArgs& a, cudaStream
     const int n_wide = (int)c->tree.items.size() - n_narrow;
     if (c->opt_kernel == 1) {
         if (n_wide > 0) return fail(c, ETS_ERR_STATE, "rebuild the tree after changing ETS_OPT_KERNEL");
-        ets::launch_partial_fma(a, D, s);
+        ets::launch_partial_fma(a, D, a.n_items, s);
         return ETS_OK;
     }
     // one CTA per SM; fewer when there are fewer narrow items than resident warps
@@ -686,6 +689,8 @@ static ets::DecodeArgs decode_args(const ets_ctx* c, int32_t layer, const void* 
     a.items = blob_ptr<ets::DevItem>(c, c->bo.items);
     a.node_leaves = blob_ptr<int32_t>(c, c->bo.node_leaves);
     a.node_len = blob_ptr<int32_t>(c, c->bo.node_len) + (size_t)layer * c->bo.len_stride;
+    a.leaf_node = blob_ptr<int32_t>(c, c->bo.leaf_node);
+    a.leaf_limit = nullptr;
     a.leaf_slot_off = blob_ptr<int32_t>(c, c->bo.leaf_slot_off);
     a.leaf_slots = blob_ptr<int32_t>(c, c->bo.leaf_slots);
     a.q = reinterpret_cast<const __nv_bfloat16*>(q);
@@ -770,6 +775,30 @@ int32_t ets_decode_step(ets_ctx* c, int32_t layer, const void* k_new, const void
                                  (cudaStream_t)cuda_stream))
         return rc;
     return decode_impl(c, layer, q, out, lse, (cudaStream_t)cuda_stream);
+}
+
+int32_t ets_tree_attn_prefill(ets_ctx* c, int32_t layer, const void* q, const int32_t* leaf_limit, void* out, float* lse,
+                              void* cuda_stream) {
+    if (int32_t rc = decode_check(c, layer, q, out)) return rc;
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, ETS_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
+    if (c->tree.n_leaves > 0 && !leaf_limit) return fail(c, ETS_ERR_INVALID_ARG, "null leaf_limit");
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (int32_t jrc = host_join(c, s)) return jrc;
+    const ets::Tree& t = c->tree;
+    if (t.n_leaves == 0) return ETS_OK;
+    ets::DecodeArgs a = decode_args(c, layer, q, out, lse, reinterpret_cast<float2*>(c->ws + c->lay.part_ml),
+                                    reinterpret_cast<float*>(c->ws + c->lay.part_o));
+    a.leaf_limit = leaf_limit;
+    // Query groups of more than 16 rows are dense contractions and run on the tcgen05 kernel; the few
+    // items of smaller groups (steps of a handful of tokens) take the scalar kernel, which knows the limit too.
+    const int D = c->cfg.head_dim;
+    const int n_narrow = t.n_narrow_items, n_wide = (int)t.items.size() - n_narrow;
+    ets::launch_partial_fma(a, D, n_narrow, s);
+    ets::launch_partial_wide(a, D, n_narrow, n_wide, s);
+    ets::launch_merge(a, D, s);
+    ETS_CUDA(c, cudaGetLastError());
+    return ETS_OK;
 }
 
 int32_t ets_tree_attn_decode_host(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse,

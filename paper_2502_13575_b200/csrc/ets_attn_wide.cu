@@ -157,6 +157,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 struct StageInfo {
     int32_t n_units;                 // page slots in the stage (0 = end of item)
     int32_t valid[kStageUnits];      // tokens held by each
+    int32_t node[kStageUnits];       // node it belongs to and index of its first token there: a query that
+    int32_t tok0[kStageUnits];       // is limited inside its own node (step prefill) needs them
 };
 
 struct Shared {
@@ -214,9 +216,11 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
         const uint32_t kdst = ring + s * 2 * STAGE_HALF, vdst = kdst + STAGE_HALF;
         while (n < kStageUnits && u < it.unit_count) {
             const int idx = u + lane;
-            int page = 0, valid = 0;
+            int page = 0, valid = 0, unode = -1, utok0 = 0;
             if (idx < it.unit_count) {
                 const int4 un = a.units[it.unit_begin + idx];
+                unode = un.y;
+                utok0 = un.z;
                 valid = a.node_len[un.y] - un.z;
                 valid = valid < 0 ? 0 : (valid > 16 ? 16 : valid);
                 if (valid > 0 && (un.x < 0 || (int64_t)un.x >= a.pages_per_layer)) { atomicExch(a.status, -1); valid = 0; }
@@ -230,8 +234,12 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                 live &= live - 1;
                 const int pg = __shfl_sync(0xffffffffu, page, src);
                 const int vl = __shfl_sync(0xffffffffu, valid, src);
+                const int nd = __shfl_sync(0xffffffffu, unode, src);
+                const int t0 = __shfl_sync(0xffffffffu, utok0, src);
                 if (lane == 0) {
                     sh->info[s].valid[n] = vl;
+                    sh->info[s].node[n] = nd;
+                    sh->info[s].tok0[n] = t0;
                     const char* src = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, pg, h, TB);
                     // raise the byte count first; the producer's single arrival comes after the
                     // last copy of the stage has been started, so the phase cannot end early
@@ -381,6 +389,21 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
         float m_ref = -INFINITY, l = 0.f;
         uint32_t n_stages = 0;
         bool ok = true;
+        // step prefill: this row's query sees only the first `lim` tokens of the node it sits at
+        int own_node = -1, lim = 0;
+        if (a.leaf_limit != nullptr && row < rows) {
+            const int leaf = a.node_leaves[it.leaf_list_begin + row / G];
+            own_node = a.leaf_node[leaf];
+            lim = a.leaf_limit[leaf];
+        }
+        auto row_valid = [&](uint32_t s, int c) {
+            int v = sh->info[s].valid[c];
+            if (sh->info[s].node[c] == own_node) {
+                const int x = lim - sh->info[s].tok0[c];
+                v = x < v ? (x < 0 ? 0 : x) : v;
+            }
+            return v;
+        };
         for (uint32_t st = 0;; ++st) {
             const uint32_t s = st % kStages;
             if (!wait_or_abort(smem_u32(&sh->s_ready), st & 1u, sh)) { ok = false; break; }
@@ -394,8 +417,8 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
             for (int c = 0; c < n; c += 2) {
                 float v[32];
                 tmem_ld32(tlane + kColS + 16u * c, v);
-                const int v0 = sh->info[s].valid[c];
-                const int v1 = c + 1 < n ? sh->info[s].valid[c + 1] : 0;
+                const int v0 = row_valid(s, c);
+                const int v1 = c + 1 < n ? row_valid(s, c + 1) : 0;
                 float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
@@ -434,8 +457,8 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
             for (int c = 0; c < n; c += 2) {
                 float v[32];
                 tmem_ld32(tlane + kColS + 16u * c, v);
-                const int v0 = sh->info[s].valid[c];
-                const int v1 = c + 1 < n ? sh->info[s].valid[c + 1] : 0;
+                const int v0 = row_valid(s, c);
+                const int v1 = c + 1 < n ? row_valid(s, c + 1) : 0;
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {

@@ -49,6 +49,8 @@ struct DecodeArgs {
     const DevItem* items;
     const int32_t* node_leaves;
     const int32_t* node_len;       // this layer's lengths
+    const int32_t* leaf_node;      // node each leaf sits at
+    const int32_t* leaf_limit;     // nullable: tokens of its own node each leaf's query may see (step prefill)
     const int32_t* leaf_slot_off;  // per (leaf, kv head)
     const int32_t* leaf_slots;
     const __nv_bfloat16* q;
@@ -84,7 +86,7 @@ struct AppendArgs {
 void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_t s);
 void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* page_ids_of_node, int n_tokens,
                     int64_t pages_per_layer, int Hkv, int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s);
-void launch_partial_fma(const DecodeArgs& a, int D, cudaStream_t s);
+void launch_partial_fma(const DecodeArgs& a, int D, int n_items, cudaStream_t s);
 void launch_merge(const DecodeArgs& a, int D, cudaStream_t s);
 size_t narrow_smem_bytes(int D);
 cudaError_t narrow_prepare(int D);

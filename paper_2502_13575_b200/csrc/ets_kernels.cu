@@ -120,14 +120,21 @@ __global__ void __launch_bounds__(kFmaWarps * 32) attn_partial_fma_kernel(Decode
     float q[kMaxRows][EPL];
     float o[kMaxRows][EPL];
     float m[kMaxRows], l[kMaxRows];
+    int own[kMaxRows], lim[kMaxRows];   // step prefill: node the row's leaf sits at, tokens of it the row may see
 #pragma unroll
     for (int r = 0; r < kMaxRows; ++r) {
         m[r] = -INFINITY;
         l[r] = 0.f;
 #pragma unroll
         for (int j = 0; j < EPL; ++j) { q[r][j] = 0.f; o[r][j] = 0.f; }
+        own[r] = -1;
+        lim[r] = 0;
         if (r < rows) {
             const int leaf = a.node_leaves[it.leaf_list_begin + r / G];
+            if (a.leaf_limit != nullptr) {
+                own[r] = a.leaf_node[leaf];
+                lim[r] = a.leaf_limit[leaf];
+            }
             const __nv_bfloat16* qp = a.q + ((size_t)leaf * a.Hq + h * G + r % G) * D + e0;
 #pragma unroll
             for (int j = 0; j < EPL; ++j) q[r][j] = __bfloat162float(qp[j]);
@@ -154,7 +161,7 @@ __global__ void __launch_bounds__(kFmaWarps * 32) attn_partial_fma_kernel(Decode
             for (int j = 0; j < EPL; ++j) { kf[j] = __bfloat162float(kp[j]); vf[j] = __bfloat162float(vp[j]); }
 #pragma unroll
             for (int r = 0; r < kMaxRows; ++r) {
-                if (r < rows) {
+                if (r < rows && (un.y != own[r] || un.z + t < lim[r])) {
                     float s = 0.f;
 #pragma unroll
                     for (int j = 0; j < EPL; ++j) s = fmaf(q[r][j], kf[j], s);
@@ -201,10 +208,10 @@ __global__ void __launch_bounds__(kFmaWarps * 32) attn_partial_fma_kernel(Decode
     }
 }
 
-void launch_partial_fma(const DecodeArgs& a, int D, cudaStream_t s) {
-    if (a.n_items <= 0) return;
-    if (D == 128) attn_partial_fma_kernel<128><<<a.n_items, kFmaWarps * 32, 0, s>>>(a);
-    else attn_partial_fma_kernel<64><<<a.n_items, kFmaWarps * 32, 0, s>>>(a);
+void launch_partial_fma(const DecodeArgs& a, int D, int n_items, cudaStream_t s) {
+    if (n_items <= 0) return;
+    if (D == 128) attn_partial_fma_kernel<128><<<n_items, kFmaWarps * 32, 0, s>>>(a);
+    else attn_partial_fma_kernel<64><<<n_items, kFmaWarps * 32, 0, s>>>(a);
 }
 
 // ------------------------------------------------------------------------------------
