@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--wide", type=int, default=None, help="0: no tcgen05 wide-group items")
     ap.add_argument("--loop-tokens", type=int, default=16,
                     help="decode iterations of the search-step loop figure (0 = skip it)")
+    ap.add_argument("--prefill", action="store_true",
+                    help="time step-prefill attention (all tokens of the workload's last search step as queries) "
+                         "instead of the decode step; prints its own JSON line")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time budget of the oracle sample")
@@ -440,9 +443,75 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_prefill(args):
+    """Step-prefill attention on one GPU: every token of the last search step of the workload's tree is a
+    query (a leaf on its step's node), one layer, K/V resident.  The work is a dense contraction (hundreds of
+    query rows share every K/V tile), so the bound is the tensor pipe: 4 * d flops per (query row, visible token)."""
+    import torch
+    from workloads import make_workload, node_kv_bits, query_bits
+    from paper_2502_13575_b200.runner import context_for_tree
+    import paper_2502_13575_b200 as ets
+    wl = make_workload(args.workload)
+    tree, g = wl.tree, wl.geometry
+    step_nodes = sorted(set(int(n) for n in tree.leaf_node))
+    leaves = np.concatenate([np.full(int(tree.tokens[n]), n, np.int32) for n in step_nodes])
+    limits = np.concatenate([np.arange(1, int(tree.tokens[n]) + 1, dtype=np.int32) for n in step_nodes])
+    ctx = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, tree.parent, tree.tokens, leaves)
+    ctx.set_option(ets.ETS_OPT_WIDE, 17)
+    ctx.tree_build(tree.parent, tree.tokens, leaves)
+    nodes = [n for n in range(tree.n_nodes) if tree.tokens[n] > 0]
+    kv = [node_kv_bits(wl.value_seed, n, int(tree.tokens[n]), g.num_kv_heads, g.head_dim, 0) for n in nodes]
+    k_all = torch.from_numpy(np.concatenate([x[0] for x in kv]).view(np.int16)).cuda().view(torch.bfloat16)
+    v_all = torch.from_numpy(np.concatenate([x[1] for x in kv]).view(np.int16)).cuda().view(torch.bfloat16)
+    ctx.kv_append(0, nodes, [int(tree.tokens[n]) for n in nodes], k_all, v_all)
+    L = int(leaves.shape[0])
+    q = torch.from_numpy(query_bits(wl.value_seed, 0, L, g.num_q_heads, g.head_dim).view(np.int16)).cuda().view(torch.bfloat16)
+    out = torch.empty_like(q)
+    lim = torch.from_numpy(limits).cuda()
+    stream = torch.cuda.current_stream().cuda_stream
+    for _ in range(args.warmup):
+        ctx.tree_attn_prefill(0, q, lim, out, None, stream=stream)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ctx.tree_attn_prefill(0, q, lim, out, None, stream=stream)
+    e1.record()
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ms = e0.elapsed_time(e1) / args.steps
+    # visible tokens per query: its ancestors' tokens plus its limit
+    anc = np.zeros(tree.n_nodes, np.int64)
+    for v in range(tree.n_nodes):
+        p = int(tree.parent[v])
+        anc[v] = (anc[p] + int(tree.tokens[p])) if p >= 0 else 0
+    visible = int((anc[leaves] + limits).sum())
+    flops = 4.0 * g.head_dim * visible * g.num_q_heads
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        peak, kind = float(peaks["bf16_tflops_sustained"]), "measured sustained cuBLAS bf16"
+    except Exception:
+        peak, kind = 1400.0, "fallback"
+    st = ctx.get_stats()
+    print(json.dumps({
+        "metric": "step_prefill_attention_query_tokens_per_s", "value": L / (ms / 1000.0), "unit": "query-tokens/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload + " last step as queries", "query_tokens": L, "step_nodes": len(step_nodes),
+                   "visible_tokens_per_query": visible / L, "heads": f"{g.num_q_heads}q/{g.num_kv_heads}kv x {g.head_dim}",
+                   "layers": 1, "items": st["n_items"], "narrow_items_on_scalar_kernel": st["n_narrow_items"]},
+        "roofline": {"bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                     "frac": flops / (ms * 1e-3) / 1e12 / peak, "peak_kind": kind, "traffic": None,
+                     "algorithmic_flops_per_launch": flops},
+    }), flush=True)
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.prefill:
+        run_prefill(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
