@@ -149,6 +149,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
         : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -420,10 +425,18 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                 const int v0 = row_valid(s, c);
                 const int v1 = c + 1 < n ? row_valid(s, c + 1) : 0;
                 float m0 = -INFINITY, m1 = -INFINITY;
+                if (v0 == 16 && v1 == 16) {   // two full pages, the usual case: no per-token test
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    if (i < v0) m0 = fmaxf(m0, v[i]);
-                    if (i < v1) m1 = fmaxf(m1, v[16 + i]);
+                    for (int i = 0; i < 16; ++i) {
+                        m0 = fmaxf(m0, v[i]);
+                        m1 = fmaxf(m1, v[16 + i]);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        if (i < v0) m0 = fmaxf(m0, v[i]);
+                        if (i < v1) m1 = fmaxf(m1, v[16 + i]);
+                    }
                 }
                 mx = fmaxf(mx, fmaxf(m0, m1));
             }
@@ -460,12 +473,15 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                 const int v0 = row_valid(s, c);
                 const int v1 = c + 1 < n ? row_valid(s, c + 1) : 0;
                 uint32_t pk[16];
+                const bool full = v0 == 16 && v1 == 16;
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
-                    const float a0 = i < v0 ? exp2f(fmaf(v[i], a.scale_log2, neg_ref)) : 0.f;
-                    const float a1 = i + 1 < v0 ? exp2f(fmaf(v[i + 1], a.scale_log2, neg_ref)) : 0.f;
-                    const float b0 = i < v1 ? exp2f(fmaf(v[16 + i], a.scale_log2, neg_ref)) : 0.f;
-                    const float b1 = i + 1 < v1 ? exp2f(fmaf(v[16 + i + 1], a.scale_log2, neg_ref)) : 0.f;
+                    // weights are at most 1 and are rounded to bf16 next: the approximate exponential
+                    // (2 ulp, tiny results flushed to zero) loses nothing
+                    const float a0 = (full || i < v0) ? ex2_approx(fmaf(v[i], a.scale_log2, neg_ref)) : 0.f;
+                    const float a1 = (full || i + 1 < v0) ? ex2_approx(fmaf(v[i + 1], a.scale_log2, neg_ref)) : 0.f;
+                    const float b0 = (full || i < v1) ? ex2_approx(fmaf(v[16 + i], a.scale_log2, neg_ref)) : 0.f;
+                    const float b1 = (full || i + 1 < v1) ? ex2_approx(fmaf(v[16 + i + 1], a.scale_log2, neg_ref)) : 0.f;
                     const __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1);
                     const __nv_bfloat162 pb = __floats2bfloat162_rn(b0, b1);
                     l0 += __low2float(pa) + __high2float(pa);
