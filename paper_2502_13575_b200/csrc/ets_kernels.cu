@@ -58,7 +58,21 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
 void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_t s) {
     if (n_items <= 0 || max_new <= 0) return;
     dim3 grid((max_new + kAppendTokPerBlock - 1) / kAppendTokPerBlock, n_items);
-    kv_append_kernel<<<grid, 256, 0, s>>>(a);
+    // Programmatic dependent launch: if the kernel before this one in the stream signals early (the merge
+    // kernel of the previous decode call does), the append starts while that kernel is still running.  It
+    // never waits for it: an append touches one layer's pages and lengths, which no merge kernel reads, and
+    // the attention kernels that do read them are launched normally, after the append has finished.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kv_append_kernel, a);
 }
 
 // ------------------------------------------------------------------------------------
@@ -220,6 +234,8 @@ void launch_partial_fma(const DecodeArgs& a, int D, int n_items, cudaStream_t s)
 // ------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(128) lse_merge_kernel(DecodeArgs a) {
+    // lets a dependent launch that asked for it (the next KV append) start now; see launch_kv_append
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * 4 + warp;
     if (row >= (int64_t)a.n_leaves * a.Hq) return;
