@@ -306,7 +306,7 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
 #define ETS_OPT_KERNEL        2  /* 0 tensor-core attention kernels (default), 1 scalar-FMA kernel;  */
                                  /* rebuild the tree after changing it                             */
 #define ETS_OPT_WIDE          4  /* smallest query group, in rows (leaves * Hq/Hkv, at least 17), that */
-                                 /* goes to the tcgen05 kernel (default 65); 0: none.  Next build.      */
+                                 /* goes to the tcgen05 kernel (default 33); 0: none.  Next build.      */
 #define ETS_OPT_HOST_PIPELINE 6  /* 1: the *_host calls return without making cuda_stream wait for   */
                                  /* them, so the copies of one call overlap the kernels of the next;   */
                                  /* results are valid after ets_host_join + synchronising that stream;  */

@@ -167,10 +167,10 @@ struct ets_ctx {
     // options
     int32_t opt_chunk_pages = 0;
     int32_t opt_kernel = 0;
-    // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256
-    // tree: 65 beats both 17 and "never" (below ~64 rows the per-item latency of the wide kernel
-    // costs more than the re-reads it saves).
-    int32_t opt_wide = 65;
+    // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256 tree and on
+    // eight width-64 trees: 33 beats 17, 49, 65 and "never" (below ~32 rows the per-item latency of the wide
+    // kernel costs more than the re-reads by the narrow kernel that it saves).
+    int32_t opt_wide = 33;
     bool opt_timing = false;
     // timing
     std::vector<cudaEvent_t> tev;   // 3 per timed call
