@@ -514,6 +514,27 @@ static int32_t host_join(ets_ctx* c, cudaStream_t s) {
     return ETS_OK;
 }
 
+// Everything an append launch reads, for the current tree and one layer.
+static ets::AppendArgs append_args(const ets_ctx* c, int32_t layer, const void* desc_dev, const void* ksrc, const void* vsrc) {
+    const ets::Tree& t = c->tree;
+    ets::AppendArgs a{};
+    a.desc = reinterpret_cast<const int4*>(desc_dev);
+    a.k_new = reinterpret_cast<const __nv_bfloat16*>(ksrc);
+    a.v_new = reinterpret_cast<const __nv_bfloat16*>(vsrc);
+    a.k_pool = c->k_pool + (size_t)layer * c->layer_pool_bytes;
+    a.v_pool = c->v_pool + (size_t)layer * c->layer_pool_bytes;
+    a.node_page_off = blob_ptr<int32_t>(c, c->bo.node_page_off);
+    a.page_ids = blob_ptr<int32_t>(c, c->bo.page_ids);
+    a.node_len = const_cast<int32_t*>(blob_ptr<int32_t>(c, c->bo.node_len)) + (size_t)layer * c->bo.len_stride;
+    a.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
+    a.n_nodes = t.n_nodes;
+    a.n_pages_total = (int32_t)t.page_ids.size();
+    a.pages_per_layer = c->cfg.pages_per_layer;
+    a.Hkv = c->cfg.num_kv_heads;
+    a.D = c->cfg.head_dim;
+    return a;
+}
+
 static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int32_t* node_id,
                            const int32_t* n_new, const void* k_new, const void* v_new, bool host_src,
                            cudaStream_t s) {
@@ -611,21 +632,7 @@ static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int
         ksrc = c->ws + c->lay.k_stage + hb * c->lay.kv_stride;
         vsrc = c->ws + c->lay.v_stage + hb * c->lay.kv_stride;
     }
-    ets::AppendArgs a{};
-    a.desc = reinterpret_cast<const int4*>(desc_dev);
-    a.k_new = reinterpret_cast<const __nv_bfloat16*>(ksrc);
-    a.v_new = reinterpret_cast<const __nv_bfloat16*>(vsrc);
-    a.k_pool = c->k_pool + (size_t)layer * c->layer_pool_bytes;
-    a.v_pool = c->v_pool + (size_t)layer * c->layer_pool_bytes;
-    a.node_page_off = blob_ptr<int32_t>(c, c->bo.node_page_off);
-    a.page_ids = blob_ptr<int32_t>(c, c->bo.page_ids);
-    a.node_len = const_cast<int32_t*>(blob_ptr<int32_t>(c, c->bo.node_len)) + (size_t)layer * c->bo.len_stride;
-    a.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
-    a.n_nodes = t.n_nodes;
-    a.n_pages_total = (int32_t)t.page_ids.size();
-    a.pages_per_layer = c->cfg.pages_per_layer;
-    a.Hkv = c->cfg.num_kv_heads;
-    a.D = c->cfg.head_dim;
+    const ets::AppendArgs a = append_args(c, layer, desc_dev, ksrc, vsrc);
     ets::launch_kv_append(a, n_items, max_new, s);
     ETS_CUDA(c, cudaGetLastError());
     if (host_src) {
@@ -838,6 +845,72 @@ int32_t ets_tree_attn_decode_host(ets_ctx* c, int32_t layer, const void* q, void
     else ETS_CUDA(c, cudaStreamWaitEvent(s, c->ev_out_free[hb], 0));
     c->q_used[hb] = c->out_used[hb] = true;
     ++c->n_host_decode;
+    return ETS_OK;
+}
+
+int32_t ets_decode_step_host(ets_ctx* c, int32_t layer, const void* k_new, const void* v_new, const void* q, void* out,
+                             float* lse, void* cuda_stream) {
+    if (int32_t rc = decode_check(c, layer, q, out)) return rc;
+    if (!k_new || !v_new) return fail(c, ETS_ERR_INVALID_ARG, "null k_new or v_new");
+    ets::Tree& t = c->tree;
+    if (t.n_leaves == 0) return ETS_OK;
+    if ((int32_t)c->step_ones.size() != t.n_leaves) c->step_ones.assign((size_t)t.n_leaves, 1);
+    // The short way needs the append's descriptor list (leaf_node, all ones) to be the one already on the
+    // device for the library's compute stream; otherwise take the two calls, which put it there.
+    const bool fast = c->cache_valid && c->cache_stream == c->st_comp && (int32_t)c->cache_nodes.size() == t.n_leaves &&
+                      std::memcmp(c->cache_nodes.data(), t.leaf_node.data(), (size_t)t.n_leaves * 4) == 0 &&
+                      std::memcmp(c->cache_nnew.data(), c->step_ones.data(), (size_t)t.n_leaves * 4) == 0 &&
+                      t.n_leaves <= c->lay.max_append_tokens;
+    if (!fast) {
+        if (int32_t rc = append_impl(c, layer, t.n_leaves, t.leaf_node.data(), c->step_ones.data(), k_new, v_new, true,
+                                     (cudaStream_t)cuda_stream))
+            return rc;
+        return ets_tree_attn_decode_host(c, layer, q, out, lse, cuda_stream);
+    }
+    std::vector<int32_t>& len = t.len[layer];
+    for (int32_t l = 0; l < t.n_leaves; ++l)   // the cached list has distinct nodes; only capacity can fail
+        if (len[t.leaf_node[l]] + 1 > t.cap[t.leaf_node[l]]) return fail(c, ETS_ERR_POOL_EXHAUSTED, "append beyond cap_tokens");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    const size_t rows = (size_t)t.n_leaves * c->cfg.num_q_heads;
+    const size_t qbytes = rows * c->cfg.head_dim * 2;
+    const size_t kvbytes = (size_t)t.n_leaves * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
+    const int hb = (int)(c->n_host_decode & 1u), hk = (int)(c->n_host_append & 1u);
+    char* kd = c->ws + c->lay.k_stage + hk * c->lay.kv_stride;
+    char* vd = c->ws + c->lay.v_stage + hk * c->lay.kv_stride;
+    char* qd = c->ws + c->lay.q_stage + hb * c->lay.q_stride;
+    char* od = c->ws + c->lay.out_stage + hb * c->lay.q_stride;
+    float* ld = reinterpret_cast<float*>(c->ws + c->lay.lse_stage + hb * c->lay.lse_stride);
+    if (!c->host_epoch_open) {
+        ETS_CUDA(c, cudaEventRecord(c->ev_entry, s));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_entry, 0));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_entry, 0));
+        c->host_epoch_open = c->opt_host_pipeline;
+    }
+    // all three inputs go in on one stream and are announced by one event
+    if (c->kv_used[hk]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_kv_free[hk], 0));
+    if (c->q_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_q_free[hb], 0));
+    ETS_CUDA(c, cudaMemcpyAsync(kd, k_new, kvbytes, cudaMemcpyHostToDevice, c->st_in));
+    ETS_CUDA(c, cudaMemcpyAsync(vd, v_new, kvbytes, cudaMemcpyHostToDevice, c->st_in));
+    ETS_CUDA(c, cudaMemcpyAsync(qd, q, qbytes, cudaMemcpyHostToDevice, c->st_in));
+    ETS_CUDA(c, cudaEventRecord(c->ev_q_in[hb], c->st_in));
+    ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_q_in[hb], 0));
+    if (c->out_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_out_free[hb], 0));
+    const char* desc_dev = c->ws + c->lay.desc + (size_t)kDescSlots * c->lay.desc_slot_bytes;
+    ets::launch_kv_append(append_args(c, layer, desc_dev, kd, vd), t.n_leaves, 1, c->st_comp);
+    if (int32_t rc = decode_impl(c, layer, qd, od, lse ? ld : nullptr, c->st_comp)) return rc;
+    ETS_CUDA(c, cudaEventRecord(c->ev_q_free[hb], c->st_comp));    // kernels done: the q and k/v staging is reusable, out is ready
+    ETS_CUDA(c, cudaEventRecord(c->ev_kv_free[hk], c->st_comp));
+    ETS_CUDA(c, cudaStreamWaitEvent(c->st_out, c->ev_q_free[hb], 0));
+    ETS_CUDA(c, cudaMemcpyAsync(out, od, qbytes, cudaMemcpyDeviceToHost, c->st_out));
+    if (lse) ETS_CUDA(c, cudaMemcpyAsync(lse, ld, rows * 4, cudaMemcpyDeviceToHost, c->st_out));
+    ETS_CUDA(c, cudaEventRecord(c->ev_out_free[hb], c->st_out));
+    if (c->opt_host_pipeline) c->host_pending = true;
+    else ETS_CUDA(c, cudaStreamWaitEvent(s, c->ev_out_free[hb], 0));
+    c->q_used[hb] = c->out_used[hb] = c->kv_used[hk] = true;
+    ++c->n_host_decode;
+    ++c->n_host_append;
+    for (int32_t l = 0; l < t.n_leaves; ++l) len[t.leaf_node[l]] += 1;
     return ETS_OK;
 }
 

@@ -360,6 +360,53 @@ def test_prune_with_ets_select_then_decode_on_the_kept_tree():
     check_close(dev_to_bits(out)[subset], ref[subset], "kept tree")
 
 
+@pytest.mark.parametrize("pipeline", [0, 1])
+def test_decode_step_host_equals_decode_step(pipeline):
+    """The host-buffer form of the fused step (first call through the two-call route, later ones through the
+    short one) gives the same bits as the device form, token after token, and the same lengths."""
+    wl = make_workload("cfg2")
+    tree, g = wl.tree, wl.geometry
+    T, layers, L = 6, 2, wl.tree.n_leaves
+    cap = tree.tokens.copy()
+    cap[tree.leaf_node] += T
+    ctxs = []
+    for _ in range(2):
+        c = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, tree.parent, cap, tree.leaf_node, num_layers=layers)
+        c.tree_build(tree.parent, cap, tree.leaf_node)
+        for l in range(layers):
+            ks, vs = node_values(tree, g, wl.value_seed, l)
+            fill_layer(c, l, ks, vs)
+        ctxs.append(c)
+    dev, host = ctxs
+    host.set_option(ets.ETS_OPT_HOST_PIPELINE, pipeline)
+    from workloads import query_bits
+    rng = np.random.default_rng(2)
+    for tok in range(T):
+        for l in range(layers):
+            kb = rng.integers(0, 1 << 16, size=(L, g.num_kv_heads, g.head_dim), dtype=np.uint16) & np.uint16(0xBFFF)
+            vb = rng.integers(0, 1 << 16, size=(L, g.num_kv_heads, g.head_dim), dtype=np.uint16) & np.uint16(0xBFFF)
+            qb = query_bits(wl.value_seed, 100 * tok + l, L, g.num_q_heads, g.head_dim)
+            q = bits_to_dev(qb)
+            out_d = torch.empty_like(q)
+            lse_d = torch.empty((L, g.num_q_heads), dtype=torch.float32, device="cuda")
+            dev.decode_step(l, bits_to_dev(kb), bits_to_dev(vb), q, out_d, lse_d)
+            k_h = torch.from_numpy(kb.view(np.int16)).pin_memory()
+            v_h = torch.from_numpy(vb.view(np.int16)).pin_memory()
+            q_h = torch.from_numpy(qb.view(np.int16)).pin_memory()
+            out_h = torch.empty_like(q_h).pin_memory()
+            lse_h = torch.empty((L, g.num_q_heads), dtype=torch.float32).pin_memory()
+            host.decode_step_host(l, k_h, v_h, q_h, out_h, lse_h)
+            if pipeline:
+                host.host_join()
+            torch.cuda.synchronize()
+            assert np.array_equal(out_h.numpy().view(np.uint16), dev_to_bits(out_d)), (tok, l)
+            assert np.array_equal(lse_h.numpy(), lse_d.cpu().numpy())
+    dev.poll_status()
+    host.poll_status()
+    for l in range(layers):
+        assert host.get_node_len(l).tolist() == dev.get_node_len(l).tolist()
+
+
 def test_append_descriptor_reuse_and_long_appends():
     """Short appends (at most 8 tokens per node) keep their (node, count) list on the device and read the
     start position from the device-side lengths; longer ones carry the start in the descriptor.  Mix

@@ -168,8 +168,8 @@ class DecodeJob:
         self.steps_done += n_tokens
 
     def step_host(self):
-        """Host buffers in, host buffers out, through the *_host entry points; the caller
-        synchronises to read the result."""
+        """Host buffers in, host buffers out, through ets_decode_step_host (append + attention of one layer per
+        call); the caller synchronises to read the result."""
         if self.steps_done >= self.headroom:
             raise RuntimeError("step budget of this job exhausted; call reset_lengths()")
         t = self.wl.tree
@@ -178,8 +178,8 @@ class DecodeJob:
         stream = self.torch.cuda.current_stream().cuda_stream
         c.tree_build(t.parent, self.cap, t.leaf_node, keep_pages_of=self.keep, stream=stream)
         for layer in range(self.layers):
-            c.kv_append_host(layer, self.leaf_nodes, self.ones, p["nk_h"][layer], p["nv_h"][layer], stream=stream)
-            c.tree_attn_decode_host(layer, p["q_h"][layer], p["out_h"][layer], None, stream=stream)
+            c.decode_step_host(layer, p["nk_h"][layer], p["nv_h"][layer], p["q_h"][layer], p["out_h"][layer], None,
+                               stream=stream)
         c.host_join(stream=stream)   # the step's results are complete once this stream has passed here
         self.steps_done += 1
 
