@@ -209,7 +209,8 @@ int32_t ets_decode_step(ets_ctx* ctx, int32_t layer, const void* k_new, const vo
                         const void* q, void* out, float* lse, void* cuda_stream);
 /* The same with HOST buffers (k_new, v_new, q in; out, lse back), copied through the workspace's staging
  * areas on the library's streams like ets_kv_append_host + ets_tree_attn_decode_host, in one call and
- * with one event for the three inputs.  Follows ETS_OPT_HOST_PIPELINE. */
+ * with one event for the three inputs.  When k_new, v_new and q are adjacent in host memory in this order
+ * (the output of a fused projection) they travel in one copy.  Follows ETS_OPT_HOST_PIPELINE. */
 int32_t ets_decode_step_host(ets_ctx* ctx, int32_t layer, const void* k_new, const void* v_new,
                              const void* q, void* out, float* lse, void* cuda_stream);
 

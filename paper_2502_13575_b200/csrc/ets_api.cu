@@ -33,6 +33,7 @@ struct Layout {  // byte offsets inside the workspace
     size_t part_ml, part_o;
     size_t q_stage, out_stage, lse_stage, k_stage, v_stage;   // two of each, *_stride bytes apart
     size_t q_stride, lse_stride, kv_stride;
+    size_t pk_stage, pk_stride;   // two areas for k_new | v_new | q of one call, contiguous
     size_t status;
     size_t total;
     int64_t max_partial_slots, max_items, max_units;
@@ -106,6 +107,8 @@ Layout make_layout(const ets_config* c) {
     L.kv_stride = align_up(kvb, A);
     L.k_stage = off; off += 2 * L.kv_stride;
     L.v_stage = off; off += 2 * L.kv_stride;
+    L.pk_stride = align_up(2 * kvb + qbytes, A);
+    L.pk_stage = off; off += 2 * L.pk_stride;
     L.status = off; off += A;
     L.total = off;
     return L;
@@ -879,6 +882,14 @@ int32_t ets_decode_step_host(ets_ctx* c, int32_t layer, const void* k_new, const
     char* kd = c->ws + c->lay.k_stage + hk * c->lay.kv_stride;
     char* vd = c->ws + c->lay.v_stage + hk * c->lay.kv_stride;
     char* qd = c->ws + c->lay.q_stage + hb * c->lay.q_stride;
+    // A fused projection leaves k, v and q of a layer next to each other; then one copy brings all three
+    // (a host-to-device copy of half a megabyte costs about as much in set-up as in transfer).
+    const bool packed = (const char*)v_new == (const char*)k_new + kvbytes && (const char*)q == (const char*)v_new + kvbytes;
+    if (packed) {
+        kd = c->ws + c->lay.pk_stage + hb * c->lay.pk_stride;   // guarded by the same events as the q area
+        vd = kd + kvbytes;
+        qd = vd + kvbytes;
+    }
     char* od = c->ws + c->lay.out_stage + hb * c->lay.q_stride;
     float* ld = reinterpret_cast<float*>(c->ws + c->lay.lse_stage + hb * c->lay.lse_stride);
     if (!c->host_epoch_open) {
@@ -890,9 +901,13 @@ int32_t ets_decode_step_host(ets_ctx* c, int32_t layer, const void* k_new, const
     // all three inputs go in on one stream and are announced by one event
     if (c->kv_used[hk]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_kv_free[hk], 0));
     if (c->q_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_q_free[hb], 0));
-    ETS_CUDA(c, cudaMemcpyAsync(kd, k_new, kvbytes, cudaMemcpyHostToDevice, c->st_in));
-    ETS_CUDA(c, cudaMemcpyAsync(vd, v_new, kvbytes, cudaMemcpyHostToDevice, c->st_in));
-    ETS_CUDA(c, cudaMemcpyAsync(qd, q, qbytes, cudaMemcpyHostToDevice, c->st_in));
+    if (packed) {
+        ETS_CUDA(c, cudaMemcpyAsync(kd, k_new, 2 * kvbytes + qbytes, cudaMemcpyHostToDevice, c->st_in));
+    } else {
+        ETS_CUDA(c, cudaMemcpyAsync(kd, k_new, kvbytes, cudaMemcpyHostToDevice, c->st_in));
+        ETS_CUDA(c, cudaMemcpyAsync(vd, v_new, kvbytes, cudaMemcpyHostToDevice, c->st_in));
+        ETS_CUDA(c, cudaMemcpyAsync(qd, q, qbytes, cudaMemcpyHostToDevice, c->st_in));
+    }
     ETS_CUDA(c, cudaEventRecord(c->ev_q_in[hb], c->st_in));
     ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_q_in[hb], 0));
     if (c->out_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_out_free[hb], 0));

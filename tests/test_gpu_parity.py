@@ -390,9 +390,13 @@ def test_decode_step_host_equals_decode_step(pipeline):
             out_d = torch.empty_like(q)
             lse_d = torch.empty((L, g.num_q_heads), dtype=torch.float32, device="cuda")
             dev.decode_step(l, bits_to_dev(kb), bits_to_dev(vb), q, out_d, lse_d)
-            k_h = torch.from_numpy(kb.view(np.int16)).pin_memory()
-            v_h = torch.from_numpy(vb.view(np.int16)).pin_memory()
-            q_h = torch.from_numpy(qb.view(np.int16)).pin_memory()
+            if (tok + l) % 2:   # separate buffers: three copies
+                k_h = torch.from_numpy(kb.view(np.int16)).pin_memory()
+                v_h = torch.from_numpy(vb.view(np.int16)).pin_memory()
+                q_h = torch.from_numpy(qb.view(np.int16)).pin_memory()
+            else:               # k | v | q adjacent in one buffer: one copy
+                pk = torch.from_numpy(np.concatenate([kb.ravel(), vb.ravel(), qb.ravel()]).view(np.int16)).pin_memory()
+                k_h, v_h, q_h = pk[:kb.size], pk[kb.size:2 * kb.size], pk[2 * kb.size:].view(L, g.num_q_heads, g.head_dim)
             out_h = torch.empty_like(q_h).pin_memory()
             lse_h = torch.empty((L, g.num_q_heads), dtype=torch.float32).pin_memory()
             host.decode_step_host(l, k_h, v_h, q_h, out_h, lse_h)

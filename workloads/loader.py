@@ -100,10 +100,17 @@ class DecodeJob:
         self.ones = np.ones(L, np.int32)
         if host_buffers:
             self.ctx.set_option(ets.ETS_OPT_HOST_PIPELINE, 1)
-            self.q_h = torch.from_numpy(qb.view(np.int16).copy()).pin_memory()
-            self.newk_h = torch.from_numpy(nk.view(np.int16).copy()).pin_memory()
-            self.newv_h = torch.from_numpy(nv.view(np.int16).copy()).pin_memory()
-            self.out_h = torch.empty_like(self.q_h).pin_memory()
+            # per layer one pinned buffer [k_new | v_new | q], as a fused q/k/v projection would leave it
+            kv_el = nk[0].size
+            packed = torch.empty((self.layers, 2 * kv_el + qb[0].size), dtype=torch.int16).pin_memory()
+            packed[:, :kv_el] = torch.from_numpy(nk.view(np.int16).reshape(self.layers, -1))
+            packed[:, kv_el:2 * kv_el] = torch.from_numpy(nv.view(np.int16).reshape(self.layers, -1))
+            packed[:, 2 * kv_el:] = torch.from_numpy(qb.view(np.int16).reshape(self.layers, -1))
+            self.packed_h = packed
+            self.newk_h = packed[:, :kv_el]
+            self.newv_h = packed[:, kv_el:2 * kv_el]
+            self.q_h = packed[:, 2 * kv_el:]
+            self.out_h = torch.empty(qb.shape, dtype=torch.int16).pin_memory()
         torch.cuda.synchronize(self.dev)
 
     # bytes the caller moves per step through the host-buffer entry points
