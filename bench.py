@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--prefill", action="store_true",
                     help="time step-prefill attention (all tokens of the workload's last search step as queries) "
                          "instead of the decode step; prints its own JSON line")
+    ap.add_argument("--segment-items", action="store_true",
+                    help="with --prefill: the decode work decomposition (items per segment) instead of path items")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time budget of the oracle sample")
@@ -458,6 +460,7 @@ def run_prefill(args):
     limits = np.concatenate([np.arange(1, int(tree.tokens[n]) + 1, dtype=np.int32) for n in step_nodes])
     ctx = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, tree.parent, tree.tokens, leaves)
     ctx.set_option(ets.ETS_OPT_WIDE, 17)
+    ctx.set_option(ets.ETS_OPT_PATH_ITEMS, 0 if args.segment_items else 1)
     ctx.tree_build(tree.parent, tree.tokens, leaves)
     nodes = [n for n in range(tree.n_nodes) if tree.tokens[n] > 0]
     kv = [node_kv_bits(wl.value_seed, n, int(tree.tokens[n]), g.num_kv_heads, g.head_dim, 0) for n in nodes]
@@ -500,7 +503,8 @@ def run_prefill(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload + " last step as queries", "query_tokens": L, "step_nodes": len(step_nodes),
                    "visible_tokens_per_query": visible / L, "heads": f"{g.num_q_heads}q/{g.num_kv_heads}kv x {g.head_dim}",
-                   "layers": 1, "items": st["n_items"], "narrow_items_on_scalar_kernel": st["n_narrow_items"]},
+                   "layers": 1, "items": st["n_items"], "narrow_items_on_scalar_kernel": st["n_narrow_items"],
+                   "decomposition": "segment items" if args.segment_items else "path items"},
         "roofline": {"bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
                      "frac": flops / (ms * 1e-3) / 1e12 / peak, "peak_kind": kind, "traffic": None,
                      "algorithmic_flops_per_launch": flops},

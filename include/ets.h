@@ -226,7 +226,7 @@ int32_t ets_decode_step_host(ets_ctx* ctx, int32_t layer, const void* k_new, con
  *   leaf_limit    DEVICE int32 [n_leaves]; values are clipped to [0, current length of the node]
  * Query groups of more than 16 rows (leaves * Hq/Hkv) that the last build classed as wide run on the
  * tcgen05 kernel, the rest on the scalar kernel: build the tree with ETS_OPT_WIDE set to 17 so that every
- * dense group takes the tensor cores.  A query that sees no token yields zeros and lse = -inf.
+ * dense group takes the tensor cores, or with ETS_OPT_PATH_ITEMS (faster: one item per tile and path).  A query that sees no token yields zeros and lse = -inf.
  * Errors: as ets_tree_attn_decode.
  */
 int32_t ets_tree_attn_prefill(ets_ctx* ctx, int32_t layer, const void* q, const int32_t* leaf_limit,
@@ -313,6 +313,10 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
                                  /* rebuild the tree after changing it                             */
 #define ETS_OPT_WIDE          4  /* smallest query group, in rows (leaves * Hq/Hkv, at least 17), that */
                                  /* goes to the tcgen05 kernel (default 33); 0: none.  Next build.      */
+#define ETS_OPT_PATH_ITEMS    7  /* 1: the next builds serve ets_tree_attn_prefill only: a work item is one   */
+                                 /* (node that leaves sit at, kv head, tile of its leaves) and walks the node's */
+                                 /* whole path, so a dense tile keeps its accumulator resident and leaves one  */
+                                 /* partial per row; the decode entry points then return ETS_ERR_STATE         */
 #define ETS_OPT_HOST_PIPELINE 6  /* 1: the *_host calls return without making cuda_stream wait for   */
                                  /* them, so the copies of one call overlap the kernels of the next;   */
                                  /* results are valid after ets_host_join + synchronising that stream;  */

@@ -76,7 +76,7 @@ Layout make_layout(const ets_config* c) {
     L.max_partial_slots = (c->max_path_entries + (path_pages + 3) / 4) * c->num_kv_heads +
                           (int64_t)kMaxWorkers * 4 * (16 / gqa > 0 ? 16 / gqa : 1);
     L.max_items = L.max_partial_slots;
-    L.max_units = c->pages_per_layer;
+    L.max_units = c->pages_per_layer + path_pages;   // path items (step prefill) list a node's whole path
     L.max_append_tokens = c->max_append_tokens > 0 ? c->max_append_tokens : c->max_leaves;
     const size_t A = 1024;
     size_t blob = 0;
@@ -84,7 +84,7 @@ Layout make_layout(const ets_config* c) {
     blob += align_up((size_t)L.max_items * 32, 256);
     blob += align_up(((size_t)c->max_nodes + 1) * 4, 256);          // node_page_off
     blob += align_up((size_t)c->pages_per_layer * 4, 256);          // page_ids
-    blob += align_up((size_t)c->max_path_entries * 4, 256);         // node_leaves
+    blob += align_up(((size_t)c->max_path_entries + c->max_leaves) * 4, 256);   // node_leaves (+ leaves by own node)
     blob += align_up((size_t)c->max_leaves * 4, 256);               // leaf_node
     blob += align_up(((size_t)c->max_leaves * c->num_kv_heads + 1) * 4, 256);  // leaf_slot_off
     blob += align_up((size_t)L.max_partial_slots * 4, 256);         // leaf_slots
@@ -170,6 +170,7 @@ struct ets_ctx {
     // options
     int32_t opt_chunk_pages = 0;
     int32_t opt_kernel = 0;
+    bool opt_path_items = false;
     // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256 tree and on
     // eight width-64 trees: 33 beats 17, 49, 65 and "never" (below ~32 rows the per-item latency of the wide
     // kernel costs more than the re-reads by the narrow kernel that it saves).
@@ -391,6 +392,9 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
             if (value < 0 || value > 1 << 20) return fail(c, ETS_ERR_INVALID_ARG, "wide threshold out of range");
             c->opt_wide = (int32_t)value;
             return ETS_OK;
+        case ETS_OPT_PATH_ITEMS:
+            c->opt_path_items = value != 0;
+            return ETS_OK;
         case ETS_OPT_TIMING:
             if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
             c->opt_timing = value != 0;
@@ -408,6 +412,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
     fp.chunk_pages = c->opt_chunk_pages;
     fp.wide_rows = (c->opt_wide > 0 && c->opt_kernel == 0) ? 128 : 0;
     fp.wide_min_rows = c->opt_wide;
+    fp.path_items = c->opt_path_items;
     ets::Tree next;
     std::string err;
     int32_t rc = ets::tree_build(c->tree, fp, n_nodes, parent, cap_tokens, keep_pages_of, n_leaves, leaf_node,
@@ -441,13 +446,13 @@ int32_t ets_tree_export(const ets_ctx* c, ets_tables_host* o) {
     o->n_nodes = t.n_nodes;
     o->n_leaves = t.n_leaves;
     o->n_pages = (int64_t)t.page_ids.size();
-    o->n_group = (int64_t)t.node_leaves.size();
+    o->n_group = t.node_leaf_off.empty() ? 0 : (int64_t)t.node_leaf_off.back();   // without the path-item extension
     o->n_path = (int64_t)t.leaf_path.size();
     auto cp = [](int32_t* dst, const std::vector<int32_t>& v) { if (dst && !v.empty()) std::memcpy(dst, v.data(), v.size() * 4); };
     cp(o->node_page_off, t.node_page_off);
     cp(o->page_ids, t.page_ids);
     cp(o->node_leaf_off, t.node_leaf_off);
-    cp(o->node_leaves, t.node_leaves);
+    if (o->node_leaves && o->n_group > 0) std::memcpy(o->node_leaves, t.node_leaves.data(), (size_t)o->n_group * 4);
     cp(o->leaf_path_off, t.leaf_path_off);
     cp(o->leaf_path, t.leaf_path);
     cp(o->leaf_path_pos, t.leaf_path_pos);
@@ -756,10 +761,11 @@ static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, 
     return ETS_OK;
 }
 
-static int32_t decode_check(ets_ctx* c, int32_t layer, const void* q, void* out) {
+static int32_t decode_check(ets_ctx* c, int32_t layer, const void* q, void* out, bool prefill = false) {
     if (!c) return ETS_ERR_INVALID_ARG;
     if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
     if (!c->has_tree) return fail(c, ETS_ERR_STATE, "no tree built");
+    if (c->tree.path_items && !prefill) return fail(c, ETS_ERR_STATE, "the tree was built with ETS_OPT_PATH_ITEMS: prefill only");
     if (layer < 0 || layer >= c->cfg.num_layers) return fail(c, ETS_ERR_INVALID_ARG, "layer out of range");
     if (c->tree.n_leaves > 0 && (!q || !out)) return fail(c, ETS_ERR_INVALID_ARG, "null q or out");
     return ETS_OK;
@@ -789,7 +795,7 @@ int32_t ets_decode_step(ets_ctx* c, int32_t layer, const void* k_new, const void
 
 int32_t ets_tree_attn_prefill(ets_ctx* c, int32_t layer, const void* q, const int32_t* leaf_limit, void* out, float* lse,
                               void* cuda_stream) {
-    if (int32_t rc = decode_check(c, layer, q, out)) return rc;
+    if (int32_t rc = decode_check(c, layer, q, out, true)) return rc;
     if (((uintptr_t)q | (uintptr_t)out) & 15) return fail(c, ETS_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
     if (c->tree.n_leaves > 0 && !leaf_limit) return fail(c, ETS_ERR_INVALID_ARG, "null leaf_limit");
     ETS_CUDA(c, cudaSetDevice(c->cfg.device));

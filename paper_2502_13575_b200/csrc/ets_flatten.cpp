@@ -195,7 +195,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     narrow.reserve((size_t)n_seg);
     for (int32_t s = 0; s < n_seg; ++s) {
         const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s];
-        if (nu == 0 || is_wide(s)) continue;
+        if (nu == 0 || is_wide(s) || p.path_items) continue;
         const int32_t gn = g[seg_head[s]];
         const int32_t tiles = ceil_div(gn, leaves_per_tile);
         double wsum = 0.0;
@@ -298,7 +298,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
 
     // ---- wide items: segments whose query group exceeds one narrow tile go to the tcgen05 kernel,
     // one CTA per (piece of the segment, kv head, tile of up to wide_rows query rows)
-    if (p.wide_rows > 0) {
+    if (p.wide_rows > 0 && !p.path_items) {
         const int32_t wide_leaves = std::max(1, p.wide_rows / std::max(1, p.gqa));
         // Piece length: long pieces amortise a CTA's fixed cost (TMEM allocation, Q tile, epilogue) over
         // several stages, short ones spread a small amount of wide work over more SMs.  Start long and
@@ -341,6 +341,64 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
                     }
             }
         }
+    }
+    // ---- path items (step prefill): one item per (node that leaves sit at, kv head, tile of its leaves) whose
+    // page slots are the node's whole root-to-node path.  A dense tile then walks its path once with its
+    // accumulator resident, gathers its queries once and leaves one partial per row; the ancestors' K/V is
+    // read once per tile of every node below them, as with segment items, but mostly from L2.
+    t.path_items = p.path_items;
+    if (p.path_items) {
+        t.items.clear();
+        slots = 0;
+        std::vector<int32_t> at_off((size_t)n_nodes + 1, 0);
+        for (int32_t l = 0; l < n_leaves; ++l) ++at_off[leaf_node[l] + 1];
+        for (int32_t v = 0; v < n_nodes; ++v) at_off[v + 1] += at_off[v];
+        const int32_t ext = (int32_t)t.node_leaves.size();       // leaves grouped by their own node follow the groups
+        t.node_leaves.resize((size_t)ext + n_leaves);
+        {
+            std::vector<int32_t> cur(at_off.begin(), at_off.end() - 1);
+            for (int32_t l = 0; l < n_leaves; ++l) t.node_leaves[(size_t)ext + cur[leaf_node[l]]++] = l;
+        }
+        const int32_t wide_leaves = std::max(1, std::max(p.wide_rows, 128) / std::max(1, p.gqa));
+        std::vector<int32_t> path;
+        for (int pass = 0; pass < 2; ++pass) {                   // small groups first: they are the narrow items
+            for (int32_t v = 0; v < n_nodes; ++v) {
+                const int32_t nl = at_off[v + 1] - at_off[v];
+                if (nl == 0) continue;
+                const bool dense = nl * p.gqa > p.rows_per_item;
+                if (dense != (pass == 1)) continue;
+                path.clear();
+                for (int32_t x = v; x >= 0; x = parent[x]) path.push_back(x);
+                const int32_t ub = (int32_t)(t.unit.size() / 4);
+                for (auto it = path.rbegin(); it != path.rend(); ++it)
+                    for (int32_t j = 0; j < need[*it]; ++j) {
+                        t.unit.push_back(t.page_ids[t.node_page_off[*it] + j]);
+                        t.unit.push_back(*it);
+                        t.unit.push_back(j * p.page_size);
+                        t.unit.push_back(0);
+                    }
+                const int32_t uc = (int32_t)(t.unit.size() / 4) - ub;
+                if (uc == 0) continue;
+                const int32_t per_tile = dense ? wide_leaves : leaves_per_tile;
+                for (int32_t h = 0; h < p.num_kv_heads; ++h)
+                    for (int32_t l0 = 0; l0 < nl; l0 += per_tile) {
+                        Item it;
+                        it.unit_begin = ub;
+                        it.unit_count = uc;
+                        it.kv_head = h;
+                        it.leaf_list_begin = ext + at_off[v] + l0;
+                        it.n_leaves_tile = std::min(per_tile, nl - l0);
+                        it.slot_first = (int32_t)slots;
+                        it.segment = -1;
+                        it.reserved = 0;
+                        t.items.push_back(it);
+                        slots += it.n_leaves_tile;
+                    }
+            }
+            if (pass == 0) t.n_narrow_items = (int32_t)t.items.size();
+        }
+        if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
+        for (int32_t k = 0; k <= n_workers; ++k) t.worker_off[k] = std::min(k, t.n_narrow_items);
     }
     t.n_chunks = (int64_t)t.items.size();
     t.n_partial_slots = slots;

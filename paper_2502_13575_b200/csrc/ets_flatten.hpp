@@ -33,6 +33,7 @@ struct FlattenParams {
     int32_t wide_min_rows = 17; // smallest query group (in rows) that is treated as wide
     int32_t wide_max_units = 32; // longest page run of a wide item
     int32_t wide_piece = 0;      // page run of a wide item (0 = chosen by the builder)
+    bool path_items = false;     // step prefill: items walk whole root-to-node paths (see tree_build)
     int32_t n_workers = 148 * 8; // warps the attention kernel keeps resident; they share the queue of narrow items
 };
 
@@ -58,6 +59,7 @@ struct Tree {
     std::vector<int32_t> worker_off;                  // first item of warp w: [worker_off[w], worker_off[w+1]) (one or none)
     int64_t n_segments = 0, n_chunks = 0, n_partial_slots = 0;
     int32_t chunk_pages_used = 0;
+    bool path_items = false;                // built for step prefill only
 };
 
 // Status codes mirror ets.h (kept numerically identical by a static_assert in the API file).

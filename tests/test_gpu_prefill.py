@@ -24,9 +24,10 @@ def _steps_as_leaves(tree, step_nodes, new_tokens):
     return np.array(leaves, np.int32), np.array(limits, np.int32)
 
 
-def _run(tree, geom, seed, leaves, limits, *, wide, sample, qscale=1.0, check_lse=True):
+def _run(tree, geom, seed, leaves, limits, *, wide, sample, qscale=1.0, check_lse=True, path_items=False):
     ctx = context_for_tree(geom.num_q_heads, geom.num_kv_heads, geom.head_dim, tree.parent, tree.tokens, leaves)
     ctx.set_option(ets.ETS_OPT_WIDE, wide)
+    ctx.set_option(ets.ETS_OPT_PATH_ITEMS, int(path_items))
     ctx.tree_build(tree.parent, tree.tokens, leaves)
     ks, vs = node_values(tree, geom, seed, 0)
     fill_layer(ctx, 0, ks, vs)
@@ -48,8 +49,8 @@ def _run(tree, geom, seed, leaves, limits, *, wide, sample, qscale=1.0, check_ls
     return ctx, q, lim, out
 
 
-@pytest.mark.parametrize("wide", [17, 65])
-def test_last_step_of_a_width16_tree(wide):
+@pytest.mark.parametrize("wide,path_items", [(17, False), (65, False), (17, True)])
+def test_last_step_of_a_width16_tree(wide, path_items):
     """All tokens of the last search step of cfg2 (16 nodes of 64..128 tokens) as queries: 1.5k leaves whose
     groups are dense (256..512 rows on their own node, thousands on the shared ancestors)."""
     wl = make_workload("cfg2")
@@ -59,7 +60,14 @@ def test_last_step_of_a_width16_tree(wide):
     rng = np.random.default_rng(1)
     first_of_steps = np.flatnonzero(limits == 1)[:3].tolist()
     sample = sorted(set([0, leaves.shape[0] - 1] + first_of_steps + [int(x) for x in rng.integers(0, leaves.shape[0], size=10)]))
-    _run(tree, g, wl.value_seed, leaves, limits, wide=wide, sample=sample)
+    ctx, q, lim, out = _run(tree, g, wl.value_seed, leaves, limits, wide=wide, sample=sample, path_items=path_items)
+    if path_items:
+        # one partial per (query, kv head), and the decode entry point refuses a tree built this way
+        st = ctx.get_stats()
+        assert st["n_partial_slots"] == leaves.shape[0] * g.num_kv_heads
+        with pytest.raises(ets.EtsError) as e:
+            ctx.tree_attn_decode(0, q, out, None)
+        assert e.value.code == ets.ETS_ERR_STATE
 
 
 def test_partial_steps_short_steps_and_peaked_scores():
@@ -71,8 +79,8 @@ def test_partial_steps_short_steps_and_peaked_scores():
     new = [1, 2, 3, 17, 33, 5, 64, 16] + [int(tree.tokens[n]) // 2 for n in nodes[8:]]
     leaves, limits = _steps_as_leaves(tree, nodes, new)
     sample = list(range(0, leaves.shape[0], max(1, leaves.shape[0] // 24)))
-    for qscale in (1.0, 6.0):
-        _run(tree, g, wl.value_seed, leaves, limits, wide=17, sample=sample, qscale=qscale)
+    for qscale, path_items in ((1.0, False), (6.0, False), (1.0, True), (6.0, True)):
+        _run(tree, g, wl.value_seed, leaves, limits, wide=17, sample=sample, qscale=qscale, path_items=path_items)
 
 
 def test_full_limits_equal_decode_and_random_small_trees():
@@ -86,6 +94,7 @@ def test_full_limits_equal_decode_and_random_small_trees():
             new = [int(rng.integers(1, tree.tokens[n] + 1)) for n in nodes]
             leaves, limits = _steps_as_leaves(tree, nodes, new)
             sample = list(range(leaves.shape[0]))
+            _run(tree, geom, 77, leaves, limits, wide=17, sample=sample, path_items=True)
             ctx, q, lim, out = _run(tree, geom, 77, leaves, limits, wide=17, sample=sample)
             full = torch.from_numpy(tree.tokens[leaves].astype(np.int32)).cuda()
             out_p, out_d = torch.empty_like(q), torch.empty_like(q)

@@ -256,3 +256,56 @@ def test_narrow_queue_is_ordered_longest_first(name):
             assert k not in seen
             seen.add(k)
             prev = k
+
+
+def test_path_items_cover_every_path_once():
+    """ETS_OPT_PATH_ITEMS: one item per (node that leaves sit at, kv head, tile of those leaves); its page slots
+    are the node's whole path in root-to-node order; every leaf gets exactly one partial slot per kv head; the
+    exported query groups are unchanged."""
+    rng = np.random.default_rng(17)
+    for _ in range(40):
+        hkv = int(rng.choice([1, 2]))
+        gqa = int(rng.choice([1, 4]))
+        tree = random_small_tree(rng, max_nodes=10, max_tokens=60, max_leaves=6)
+        # several query tokens per leaf node, as in a step prefill
+        leaves = np.concatenate([np.full(int(rng.integers(1, 40)), n, np.int32) for n in sorted(set(tree.leaf_node.tolist()))])
+        ctx = host_ctx(hq=hkv * gqa, hkv=hkv, max_leaves=leaves.shape[0], max_path_entries=leaves.shape[0] * 12,
+                       max_path_tokens=1 << 12)
+        ctx.tree_build(tree.parent, tree.tokens, leaves)
+        groups = ctx.tree_export()["node_leaves"].copy()
+        ctx.set_option(ets.ETS_OPT_PATH_ITEMS, 1)
+        ctx.tree_build(tree.parent, tree.tokens, leaves)
+        t, w = ctx.tree_export(), ctx.work_export()
+        assert np.array_equal(t["node_leaves"], groups)
+        seen = {}
+        for it in w["item"]:
+            ub, uc, head, lb, nl, slot0, seg, _ = (int(x) for x in it)
+            assert seg == -1 and uc >= 1
+            units = w["unit"][ub:ub + uc]
+            node = int(units[-1][1])
+            path = []
+            v = node
+            while v >= 0:
+                path.append(v)
+                v = int(tree.parent[v])
+            expect = [(int(pg), n, 16 * j) for n in reversed(path)
+                      for j, pg in enumerate(t["page_ids"][t["node_page_off"][n]:t["node_page_off"][n + 1]])]
+            assert [(int(u[0]), int(u[1]), int(u[2])) for u in units] == expect
+            for i in range(nl):
+                seen.setdefault((slot0 + i, head), 0)
+                seen[(slot0 + i, head)] += 1
+        assert all(c == 1 for c in seen.values())
+        for l in range(leaves.shape[0]):
+            for h in range(hkv):
+                k = l * hkv + h
+                n_slots = w["leaf_slot_off"][k + 1] - w["leaf_slot_off"][k]
+                has_pages = any(t["node_page_off"][n + 1] > t["node_page_off"][n] for n in _path(tree, int(leaves[l])))
+                assert n_slots == (1 if has_pages else 0)
+
+
+def _path(tree, node):
+    out = []
+    while node >= 0:
+        out.append(node)
+        node = int(tree.parent[node])
+    return out
