@@ -6,8 +6,8 @@
 // TMEM lane) instead of being re-read once per 16 rows by the narrow kernel.
 //
 // One CTA per work item, six warps:
-//   warp 0      producer: walks the item's page slots, skips empty ones, and brings up to eight
-//               K tiles and eight V tiles (128 tokens) per stage into shared memory with linear
+//   warp 0      producer: walks the item's page slots, skips empty ones, and brings up to four
+//               K tiles and four V tiles (64 tokens) per stage into shared memory with linear
 //               bulk copies; the page image in global memory already is the SWIZZLE_128B operand
 //               layout, so no tensor map is needed.  Also owns the TMEM allocation.
 //   warp 1      MMA issuer: S = Q . K^T   (A = Q from shared memory, K-major; B = K stage, K-major)
@@ -17,9 +17,11 @@
 //               reference lazily, only after it is outgrown by 2^8, saves most rescales but leaves
 //               the dominant weight off a power of two, and its bf16 rounding then shows in peaked
 //               rows whose output nearly cancels; the exact policy keeps that weight at 1.)
-// Stages are processed one after another (QK -> softmax -> PV) and a CTA holds a single stage, so a
-// CTA alone does not saturate anything; it is sized (97 KB of shared memory, 256 TMEM columns) to sit
-// on an SM next to a CTA of the narrow kernel, launched on a second stream, and the two overlap.
+// A CTA holds two stages of 64 tokens and two S buffers in tensor memory: while the softmax warps work on
+// stage s, the copies of stage s + 1 land and its S = Q K^T is already issued; the maximum pass of stage
+// s + 1 overlaps the product O += P V of stage s.  The rest of a stage is serial (softmax -> PV), so a CTA
+// alone does not saturate anything; it is sized (97 KB of shared memory, 256 TMEM columns) to sit on an SM
+// next to a CTA of the narrow kernel, launched on a second stream, and the two overlap.
 // Every wait is bounded.  A wait that runs out sets an abort flag that all roles poll, the status
 // word is raised, copies in flight are waited for (again boundedly), TMEM is released, and the CTA
 // returns.
@@ -30,13 +32,16 @@ namespace ets {
 namespace {
 
 constexpr int kWideThreads = 192;
-constexpr int kStageUnits = 8;                 // page slots (16 tokens each) per stage
-constexpr int kStages = 1;                     // one 128-token stage: leaves room for a narrow-kernel CTA on the same SM
+constexpr int kStageUnits = 4;                 // page slots (16 tokens each) per stage
+constexpr int kStages = 2;                     // two 64-token stages: the next one loads while this one is computed; same footprint as one of 128
 constexpr uint32_t kSpin = 1u << 22;
 constexpr uint32_t kTmemCols = 256;
 // P (bf16, 8 columns per 16 tokens) is written over the S columns it was computed from: chunk c of P
 // covers columns that only hold S chunks <= c/2, which the thread has consumed by then.
-constexpr uint32_t kColS = 0, kColP = 0, kColO = 128;
+// S has two buffers of 64 columns (a stage is 64 tokens): the product of the next stage is issued while the
+// softmax warps still work on this one.
+constexpr uint32_t kColS = 0, kColP = 0, kColO = 128, kColSBuf = 64;
+static_assert(kStageUnits * 16 <= (int)kColSBuf && kStages == 2, "S double buffer: 64-token stages, two of them");
 constexpr float kRescaleThreshold = 0.0f;      // log2 units; see the softmax role
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -169,7 +174,7 @@ struct StageInfo {
 struct Shared {
     uint64_t full[kStages];          // copies of a stage have landed (producer -> MMA warp)
     uint64_t empty[kStages];         // stage may be overwritten (PV product done -> producer)
-    uint64_t s_ready;                // S = Q K^T is in tensor memory (MMA -> softmax)
+    uint64_t s_ready[2];             // S = Q K^T of an even / odd stage is in tensor memory (MMA -> softmax)
     uint64_t p_ready;                // P is in tensor memory (softmax -> MMA), 4 arrivals
     uint64_t o_ready;                // O += P V done (MMA -> softmax)
     uint32_t tmem_base;
@@ -269,7 +274,8 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
     if (warp == 0) {
         if (lane == 0) {
             for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
-            mbar_init(smem_u32(&sh->s_ready), 1);
+            mbar_init(smem_u32(&sh->s_ready[0]), 1);
+            mbar_init(smem_u32(&sh->s_ready[1]), 1);
             mbar_init(smem_u32(&sh->p_ready), 4);
             mbar_init(smem_u32(&sh->o_ready), 1);
             sh->abort = 0;
@@ -339,14 +345,14 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         const uint32_t idesc_pv = instr_desc(D, true);
-        bool first = true;
-        for (uint32_t st = 0;; ++st) {
+        // S = Q K^T of stage st into S buffer st % 2 (or the end marker); returns the stage's page slots, -1 on abort
+        auto issue_qk = [&](uint32_t st) -> int {
             const uint32_t s = st % kStages;
-            if (!wait_or_abort(smem_u32(&sh->full[s]), (st / kStages) & 1u, sh)) break;
+            if (!wait_or_abort(smem_u32(&sh->full[s]), (st / kStages) & 1u, sh)) return -1;
             const int n = sh->info[s].n_units;
             if (n == 0) {   // end of item: wake the softmax warps, which then see the same marker
-                if (lane == 0) mbar_arrive(smem_u32(&sh->s_ready));
-                break;
+                if (lane == 0) mbar_arrive(smem_u32(&sh->s_ready[st & 1u]));
+                return 0;
             }
             const uint32_t kst = ring + s * 2 * STAGE_HALF, vst = kst + STAGE_HALF;
             // rows past a page's length hold stale bytes; zero them in V (0 * garbage could be NaN)
@@ -369,23 +375,33 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
                     const uint32_t koff = (uint32_t)(ks >> 2) * 1024u + (uint32_t)(ks & 3) * 32u;
-                    umma_ss(tmem + kColS, smem_desc(q_smem + koff, 16, 1024u * (D / 64)), smem_desc(kst + koff, 16, 1024u * (D / 64)),
-                            idesc_qk, ks > 0);
+                    umma_ss(tmem + kColS + kColSBuf * (st & 1u), smem_desc(q_smem + koff, 16, 1024u * (D / 64)),
+                            smem_desc(kst + koff, 16, 1024u * (D / 64)), idesc_qk, ks > 0);
                 }
-                umma_commit(smem_u32(&sh->s_ready));
+                umma_commit(smem_u32(&sh->s_ready[st & 1u]));
             }
             __syncwarp();
+            return n;
+        };
+        // The S buffer of stage st + 1 held stage st - 1, whose second product was issued by this thread
+        // before: the tensor pipe runs a thread's products in order, so the buffer is free by then.
+        int n = issue_qk(0);
+        for (uint32_t st = 0; n > 0; ++st) {
+            const uint32_t s = st % kStages;
+            const int n_next = issue_qk(st + 1);
+            if (n_next < 0) break;
+            const uint32_t vst = ring + s * 2 * STAGE_HALF + STAGE_HALF;
             if (!wait_or_abort(smem_u32(&sh->p_ready), st & 1u, sh)) break;
             tc_fence_after();
             if (lane == 0) {
                 for (int k = 0; k < n; ++k)
-                    umma_ts(tmem + kColO, tmem + kColP + 8u * k, smem_desc(vst + k * TB, 1024, 1024u * (D / 64)), idesc_pv,
-                            !(first && k == 0));
+                    umma_ts(tmem + kColO, tmem + kColP + kColSBuf * (st & 1u) + 8u * k, smem_desc(vst + k * TB, 1024, 1024u * (D / 64)),
+                            idesc_pv, !(st == 0 && k == 0));
                 umma_commit(smem_u32(&sh->empty[s]));
                 umma_commit(smem_u32(&sh->o_ready));
             }
-            first = false;
             __syncwarp();
+            n = n_next;
         }
     } else {
         // ------------------------------------------------------------------ softmax, one row per thread
@@ -411,7 +427,7 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
         };
         for (uint32_t st = 0;; ++st) {
             const uint32_t s = st % kStages;
-            if (!wait_or_abort(smem_u32(&sh->s_ready), st & 1u, sh)) { ok = false; break; }
+            if (!wait_or_abort(smem_u32(&sh->s_ready[st & 1u]), (st >> 1) & 1u, sh)) { ok = false; break; }
             // s_ready can only complete after the MMA warp saw full[s]: the stage info is visible
             const int n = sh->info[s].n_units;
             if (n == 0) break;   // end marker passed on by the MMA warp
@@ -421,7 +437,7 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
             float mx = -INFINITY;
             for (int c = 0; c < n; c += 2) {
                 float v[32];
-                tmem_ld32(tlane + kColS + 16u * c, v);
+                tmem_ld32(tlane + kColS + kColSBuf * (st & 1u) + 16u * c, v);
                 const int v0 = row_valid(s, c);
                 const int v1 = c + 1 < n ? row_valid(s, c + 1) : 0;
                 float m0 = -INFINITY, m1 = -INFINITY;
@@ -441,6 +457,13 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                 mx = fmaxf(mx, fmaxf(m0, m1));
             }
             mx *= a.scale_log2;
+            // O must hold the previous stage's product before it is rescaled, and that product must have read
+            // its P before this stage's P is handed over: wait for it here, after the maximum pass, which
+            // thereby overlaps the product
+            if (st > 0) {
+                if (!wait_or_abort(smem_u32(&sh->o_ready), (st - 1) & 1u, sh)) { ok = false; break; }
+                tc_fence_after();
+            }
             // raise the reference (and rescale O, l) when the maximum outgrew it by the threshold
             const bool need = mx > m_ref + kRescaleThreshold;
             const bool any_need = __any_sync(0xffffffffu, need);
@@ -469,7 +492,7 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
             const float neg_ref = -m_ref;
             for (int c = 0; c < n; c += 2) {
                 float v[32];
-                tmem_ld32(tlane + kColS + 16u * c, v);
+                tmem_ld32(tlane + kColS + kColSBuf * (st & 1u) + 16u * c, v);
                 const int v0 = row_valid(s, c);
                 const int v1 = c + 1 < n ? row_valid(s, c + 1) : 0;
                 uint32_t pk[16];
@@ -489,7 +512,7 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                     pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pa);
                     pk[8 + (i >> 1)] = *reinterpret_cast<const uint32_t*>(&pb);
                 }
-                tmem_st16(tlane + kColP + 8u * c, pk);
+                tmem_st16(tlane + kColP + kColSBuf * (st & 1u) + 8u * c, pk);
             }
             l += l0 + l1;
             tmem_wait_st();
@@ -497,7 +520,10 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready));
             ++n_stages;
-            if (!wait_or_abort(smem_u32(&sh->o_ready), st & 1u, sh)) { ok = false; break; }
+        }
+        // the last stage's product must be in O before the epilogue reads it
+        if (ok && n_stages > 0) {
+            if (!wait_or_abort(smem_u32(&sh->o_ready), (n_stages - 1) & 1u, sh)) ok = false;
             tc_fence_after();
         }
         // epilogue: partial (m_ref, l, O) of this row
