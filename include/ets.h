@@ -317,6 +317,13 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
                                  /* (node that leaves sit at, kv head, tile of its leaves) and walks the node's */
                                  /* whole path, so a dense tile keeps its accumulator resident and leaves one  */
                                  /* partial per row; the decode entry points then return ETS_ERR_STATE         */
+#define ETS_OPT_OVERLAP_APPEND 8 /* 1: ets_kv_append / ets_decode_step may start their append while the kernel    */
+                                 /* before it in the stream is still running, if that kernel signals early    */
+                                 /* (programmatic dependent launch; the library's merge kernel does, so in a   */
+                                 /* loop over layers the append runs under the previous call's merge).  Only   */
+                                 /* for callers whose k_new / v_new are complete when the call is made: not    */
+                                 /* when the kernel that writes them is the one before the call in the stream   */
+                                 /* and signals early itself.  Default 0.                                      */
 #define ETS_OPT_HOST_PIPELINE 6  /* 1: the *_host calls return without making cuda_stream wait for   */
                                  /* them, so the copies of one call overlap the kernels of the next;   */
                                  /* results are valid after ets_host_join + synchronising that stream;  */

@@ -171,6 +171,7 @@ struct ets_ctx {
     int32_t opt_chunk_pages = 0;
     int32_t opt_kernel = 0;
     bool opt_path_items = false;
+    bool opt_overlap_append = false;
     // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256 tree and on
     // eight width-64 trees: 33 beats 17, 49, 65 and "never" (below ~32 rows the per-item latency of the wide
     // kernel costs more than the re-reads by the narrow kernel that it saves).
@@ -391,6 +392,9 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
         case ETS_OPT_WIDE:
             if (value < 0 || value > 1 << 20) return fail(c, ETS_ERR_INVALID_ARG, "wide threshold out of range");
             c->opt_wide = (int32_t)value;
+            return ETS_OK;
+        case ETS_OPT_OVERLAP_APPEND:
+            c->opt_overlap_append = value != 0;
             return ETS_OK;
         case ETS_OPT_PATH_ITEMS:
             c->opt_path_items = value != 0;
@@ -641,7 +645,7 @@ static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int
         vsrc = c->ws + c->lay.v_stage + hb * c->lay.kv_stride;
     }
     const ets::AppendArgs a = append_args(c, layer, desc_dev, ksrc, vsrc);
-    ets::launch_kv_append(a, n_items, max_new, s);
+    ets::launch_kv_append(a, n_items, max_new, c->opt_overlap_append && !host_src, s);
     ETS_CUDA(c, cudaGetLastError());
     if (host_src) {
         ETS_CUDA(c, cudaEventRecord(c->ev_kv_free[hb], c->st_comp));
@@ -918,7 +922,7 @@ int32_t ets_decode_step_host(ets_ctx* c, int32_t layer, const void* k_new, const
     ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_q_in[hb], 0));
     if (c->out_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_out_free[hb], 0));
     const char* desc_dev = c->ws + c->lay.desc + (size_t)kDescSlots * c->lay.desc_slot_bytes;
-    ets::launch_kv_append(append_args(c, layer, desc_dev, kd, vd), t.n_leaves, 1, c->st_comp);
+    ets::launch_kv_append(append_args(c, layer, desc_dev, kd, vd), t.n_leaves, 1, false, c->st_comp);
     if (int32_t rc = decode_impl(c, layer, qd, od, lse ? ld : nullptr, c->st_comp)) return rc;
     ETS_CUDA(c, cudaEventRecord(c->ev_q_free[hb], c->st_comp));    // kernels done: the q and k/v staging is reusable, out is ready
     ETS_CUDA(c, cudaEventRecord(c->ev_kv_free[hk], c->st_comp));

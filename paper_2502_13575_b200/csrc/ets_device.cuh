@@ -83,7 +83,7 @@ struct AppendArgs {
     int32_t Hkv, D;
 };
 
-void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_t s);
+void launch_kv_append(const AppendArgs& a, int n_items, int max_new, bool may_start_early, cudaStream_t s);
 void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* page_ids_of_node, int n_tokens,
                     int64_t pages_per_layer, int Hkv, int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s);
 void launch_partial_fma(const DecodeArgs& a, int D, int n_items, cudaStream_t s);

@@ -55,13 +55,15 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
     if (blockIdx.x == 0 && threadIdx.x == 0) a.node_len[node] = start + n_new;
 }
 
-void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_t s) {
+void launch_kv_append(const AppendArgs& a, int n_items, int max_new, bool may_start_early, cudaStream_t s) {
     if (n_items <= 0 || max_new <= 0) return;
     dim3 grid((max_new + kAppendTokPerBlock - 1) / kAppendTokPerBlock, n_items);
-    // Programmatic dependent launch: if the kernel before this one in the stream signals early (the merge
-    // kernel of the previous decode call does), the append starts while that kernel is still running.  It
-    // never waits for it: an append touches one layer's pages and lengths, which no merge kernel reads, and
-    // the attention kernels that do read them are launched normally, after the append has finished.
+    // Programmatic dependent launch (only when the caller allows it): if the kernel before this one in the
+    // stream signals early (the merge kernel of the previous decode call does), the append starts while that
+    // kernel is still running.  It never waits for it: an append touches one layer's pages and lengths, which
+    // no merge kernel reads, and the attention kernels that do read them are launched normally, after the
+    // append has finished.  The caller must not allow it when the kernel that produces k_new / v_new is the
+    // one before this in the stream and signals early itself.
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(256);
@@ -71,7 +73,7 @@ void launch_kv_append(const AppendArgs& a, int n_items, int max_new, cudaStream_
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = may_start_early ? 1 : 0;
     cudaLaunchKernelEx(&cfg, kv_append_kernel, a);
 }
 

@@ -74,6 +74,8 @@ class DecodeJob:
             self.ctx.set_option(ets.ETS_OPT_KERNEL, kernel)
         if wide is not None:
             self.ctx.set_option(ets.ETS_OPT_WIDE, wide)
+        # the step inputs below are resident before any call: appends may run under the preceding merge kernel
+        self.ctx.set_option(ets.ETS_OPT_OVERLAP_APPEND, 1)
         self.keep = np.arange(tree.n_nodes, dtype=np.int32)
         self.ctx.tree_build(tree.parent, self.cap, tree.leaf_node)
         # pools
