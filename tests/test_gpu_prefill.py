@@ -106,3 +106,39 @@ def test_full_limits_equal_decode_and_random_small_trees():
             # different kernels serve the narrow items in the two calls: equal within twice the parity bar
             excess = ((out_p.float() - out_d.float()).abs() - (4e-3 + 2e-2 * out_d.float().abs())).max().item()
             assert excess <= 0, excess
+
+
+@pytest.mark.parametrize("path_items", [False, True])
+def test_limits_of_zero_and_beyond_the_node(path_items):
+    """A limit of 0 hides the own node entirely (only ancestors are seen; at a root: nothing, which gives zeros
+    and lse = -inf); a limit beyond the node's length is clipped to it."""
+    geom = Geometry(8, 2, 128)
+    parent = np.array([-1, 0, 0], np.int32)
+    tokens = np.array([40, 33, 20], np.int32)
+    from workloads import Tree
+    tree = Tree(parent, tokens, np.array([1, 2], np.int32))
+    #        leaf node:  root  root  1    1    1     2    2
+    leaves = np.array([0, 0, 1, 1, 1, 2, 2] * 3, np.int32)          # 21 leaves: dense groups
+    limits = np.array([0, 7, 0, 33, 99, 1, 20] * 3, np.int32)
+    ctx = context_for_tree(geom.num_q_heads, geom.num_kv_heads, geom.head_dim, parent, tokens, leaves)
+    ctx.set_option(ets.ETS_OPT_WIDE, 17)
+    ctx.set_option(ets.ETS_OPT_PATH_ITEMS, int(path_items))
+    ctx.tree_build(parent, tokens, leaves)
+    ks, vs = node_values(tree, geom, 5, 0)
+    fill_layer(ctx, 0, ks, vs)
+    qb = query_bits(5, 0, leaves.shape[0], geom.num_q_heads, geom.head_dim)
+    q = bits_to_dev(qb)
+    out = torch.empty_like(q)
+    lse = torch.empty((leaves.shape[0], geom.num_q_heads), dtype=torch.float32, device="cuda")
+    ctx.tree_attn_prefill(0, q, torch.from_numpy(limits).cuda(), out, lse)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    blind = np.flatnonzero((leaves == 0) & (limits == 0))
+    assert np.all(dev_to_bits(out)[blind] == 0) and np.all(np.isneginf(lse.cpu().numpy()[blind]))
+    seeing = [i for i in range(leaves.shape[0]) if i not in set(blind.tolist())]
+    clipped = np.minimum(limits, tokens[leaves])
+    ref, ref_lse = tree_prefill_attention(parent, tokens, leaves, clipped, ks, vs, qb, geom.num_q_heads, geom.num_kv_heads,
+                                          leaves=seeing)
+    check_close(dev_to_bits(out)[seeing], ref[seeing], "limits")
+    got = lse.cpu().numpy().astype(np.float64)[seeing]
+    assert np.all(np.abs(got - ref_lse[seeing]) <= 1e-3 + 1e-3 * np.abs(ref_lse[seeing]))
