@@ -216,52 +216,56 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
     const int G = a.G, h = it.kv_head;
     const int rows = it.n_leaves_tile * G;
 
-    // Producer step: gather up to 8 page slots of the item that hold tokens (lane-parallel look-ahead
-    // over 32 slots), start their copies into stage st % kStages and publish the stage.  Returns the
-    // number of slots (0 = end marker).  Called by all lanes of warp 0.
-    int u = 0;
+    // Producer step: take the next page slots of the item that hold tokens (up to kStageUnits), start their
+    // copies into stage st % kStages and publish the stage.  Returns the number of slots (0 = end marker).
+    // Called by all lanes of warp 0.  The descriptors of 32 consecutive page slots, one per lane, are kept in
+    // registers between calls: the two dependent table loads behind them are paid once per 32 slots, not once
+    // per stage.
+    int u = 0, win_base = -32;
+    int w_page = 0, w_valid = 0, w_node = -1, w_tok0 = 0;
+    uint32_t w_live = 0;
     auto produce = [&](uint32_t st) -> int {
         const uint32_t s = st % kStages;
         int n = 0;
         const uint32_t kdst = ring + s * 2 * STAGE_HALF, vdst = kdst + STAGE_HALF;
         while (n < kStageUnits && u < it.unit_count) {
-            const int idx = u + lane;
-            int page = 0, valid = 0, unode = -1, utok0 = 0;
-            if (idx < it.unit_count) {
-                const int4 un = a.units[it.unit_begin + idx];
-                unode = un.y;
-                utok0 = un.z;
-                valid = a.node_len[un.y] - un.z;
-                valid = valid < 0 ? 0 : (valid > 16 ? 16 : valid);
-                if (valid > 0 && (un.x < 0 || (int64_t)un.x >= a.pages_per_layer)) { atomicExch(a.status, -1); valid = 0; }
-                page = un.x;
-            }
-            uint32_t live = __ballot_sync(0xffffffffu, valid > 0);
-            int consumed = 32;
-            while (live) {
-                const int src = __ffs(live) - 1;
-                if (n == kStageUnits) { consumed = src; break; }
-                live &= live - 1;
-                const int pg = __shfl_sync(0xffffffffu, page, src);
-                const int vl = __shfl_sync(0xffffffffu, valid, src);
-                const int nd = __shfl_sync(0xffffffffu, unode, src);
-                const int t0 = __shfl_sync(0xffffffffu, utok0, src);
-                if (lane == 0) {
-                    sh->info[s].valid[n] = vl;
-                    sh->info[s].node[n] = nd;
-                    sh->info[s].tok0[n] = t0;
-                    const char* src = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, pg, h, TB);
-                    // raise the byte count first; the producer's single arrival comes after the
-                    // last copy of the stage has been started, so the phase cannot end early
-                    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"(2 * TB) : "memory");
-                    bulk_g2s(kdst + n * TB, src, TB, smem_u32(&sh->full[s]));
-                    bulk_g2s(vdst + n * TB, src + TB, TB, smem_u32(&sh->full[s]));
+            if (u >= win_base + 32) {
+                win_base = u;
+                const int idx = u + lane;
+                w_page = 0; w_valid = 0; w_node = -1; w_tok0 = 0;
+                if (idx < it.unit_count) {
+                    const int4 un = a.units[it.unit_begin + idx];
+                    w_node = un.y;
+                    w_tok0 = un.z;
+                    w_valid = a.node_len[un.y] - un.z;
+                    w_valid = w_valid < 0 ? 0 : (w_valid > 16 ? 16 : w_valid);
+                    if (w_valid > 0 && (un.x < 0 || (int64_t)un.x >= a.pages_per_layer)) { atomicExch(a.status, -1); w_valid = 0; }
+                    w_page = un.x;
                 }
-                ++n;
+                w_live = __ballot_sync(0xffffffffu, w_valid > 0);
             }
-            u += consumed;
-            if (u > it.unit_count) u = it.unit_count;
+            const uint32_t rest = w_live >> (u - win_base);      // live slots of the window from u on
+            if (rest == 0) { u = win_base + 32; continue; }
+            const int src = (u - win_base) + __ffs(rest) - 1;
+            u = win_base + src + 1;
+            const int pg = __shfl_sync(0xffffffffu, w_page, src);
+            const int vl = __shfl_sync(0xffffffffu, w_valid, src);
+            const int nd = __shfl_sync(0xffffffffu, w_node, src);
+            const int t0 = __shfl_sync(0xffffffffu, w_tok0, src);
+            if (lane == 0) {
+                sh->info[s].valid[n] = vl;
+                sh->info[s].node[n] = nd;
+                sh->info[s].tok0[n] = t0;
+                const char* tile = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, pg, h, TB);
+                // raise the byte count first; the producer's single arrival comes after the
+                // last copy of the stage has been started, so the phase cannot end early
+                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"(2 * TB) : "memory");
+                bulk_g2s(kdst + n * TB, tile, TB, smem_u32(&sh->full[s]));
+                bulk_g2s(vdst + n * TB, tile + TB, TB, smem_u32(&sh->full[s]));
+            }
+            ++n;
         }
+        if (u > it.unit_count) u = it.unit_count;
         if (lane == 0) {
             sh->info[s].n_units = n;                 // n == 0: end marker
             mbar_arrive(smem_u32(&sh->full[s]));      // publishes the stage info with release semantics
