@@ -234,12 +234,17 @@ void launch_partial_fma(const DecodeArgs& a, int D, int n_items, cudaStream_t s)
 // Log-sum-exp merge along each leaf's path: one warp per (leaf, query head); plenty of warps,
 // because each one is a short chain of dependent loads.
 // ------------------------------------------------------------------------------------
+#ifndef ETS_MERGE_WARPS
+#define ETS_MERGE_WARPS 4
+#endif
+constexpr int kMergeWarps = ETS_MERGE_WARPS;
+
 template <int D>
-__global__ void __launch_bounds__(128) lse_merge_kernel(DecodeArgs a) {
+__global__ void __launch_bounds__(kMergeWarps * 32) lse_merge_kernel(DecodeArgs a) {
     // lets a dependent launch that asked for it (the next KV append) start now; see launch_kv_append
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * 4 + warp;
+    const int64_t row = (int64_t)blockIdx.x * kMergeWarps + warp;
     if (row >= (int64_t)a.n_leaves * a.Hq) return;
     merge_row<D>(a, (int)(row / a.Hq), (int)(row % a.Hq), lane);
 }
@@ -247,9 +252,9 @@ __global__ void __launch_bounds__(128) lse_merge_kernel(DecodeArgs a) {
 void launch_merge(const DecodeArgs& a, int D, cudaStream_t s) {
     const int64_t rows = (int64_t)a.n_leaves * a.Hq;
     if (rows <= 0) return;
-    const int blocks = (int)((rows + 3) / 4);
-    if (D == 128) lse_merge_kernel<128><<<blocks, 128, 0, s>>>(a);
-    else lse_merge_kernel<64><<<blocks, 128, 0, s>>>(a);
+    const int blocks = (int)((rows + kMergeWarps - 1) / kMergeWarps);
+    if (D == 128) lse_merge_kernel<128><<<blocks, kMergeWarps * 32, 0, s>>>(a);
+    else lse_merge_kernel<64><<<blocks, kMergeWarps * 32, 0, s>>>(a);
 }
 
 }  // namespace ets
