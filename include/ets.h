@@ -207,6 +207,17 @@ int32_t ets_tree_attn_decode_host(ets_ctx* ctx, int32_t layer, const void* q, vo
  */
 int32_t ets_decode_step(ets_ctx* ctx, int32_t layer, const void* k_new, const void* v_new,
                         const void* q, void* out, float* lse, void* cuda_stream);
+/*
+ * For callers that capture ets_decode_step into a CUDA graph and replay it: a replay appends on the device
+ * (the captured append reads the node lengths there), but the library's host-side record of the lengths,
+ * which the capacity checks and the next ets_tree_build use, only saw the captured call.  Tell it that
+ * `times` further decode steps of `layer` have run (host only, no launch).  Capture after one ordinary call
+ * of the same step (the first call uploads the append's descriptor list), with ETS_OPT_OVERLAP_APPEND and
+ * ETS_OPT_TIMING off; the caller keeps the replays inside cap_tokens (the device-side append refuses and
+ * raises the status word otherwise).  Errors: ETS_ERR_POOL_EXHAUSTED if the count cannot have fitted.
+ */
+int32_t ets_note_decode_steps(ets_ctx* ctx, int32_t layer, int32_t times);
+
 /* The same with HOST buffers (k_new, v_new, q in; out, lse back), copied through the workspace's staging
  * areas on the library's streams like ets_kv_append_host + ets_tree_attn_decode_host, in one call and
  * with one event for the three inputs.  When k_new, v_new and q are adjacent in host memory in this order

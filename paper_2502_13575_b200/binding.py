@@ -111,6 +111,7 @@ _SIGNATURES = {
                                           C.c_void_p]),
     "ets_decode_step": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p]),
+    "ets_note_decode_steps": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),
     "ets_decode_step_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p]),
     "ets_tree_attn_decode_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -325,6 +326,9 @@ class EtsContext:
     def decode_step(self, layer: int, k_new, v_new, q, out, lse=None, stream=None):
         self._check(lib.ets_decode_step(self._h, layer, _dev_ptr(k_new), _dev_ptr(v_new), _dev_ptr(q), _dev_ptr(out),
                                         _dev_ptr(lse), _stream_ptr(stream)))
+
+    def note_decode_steps(self, layer: int, times: int):
+        self._check(lib.ets_note_decode_steps(self._h, layer, times))
 
     def decode_step_host(self, layer: int, k_new, v_new, q, out, lse=None, stream=None):
         self._check(lib.ets_decode_step_host(self._h, layer, _dev_ptr(k_new), _dev_ptr(v_new), _dev_ptr(q),

@@ -861,6 +861,20 @@ int32_t ets_tree_attn_decode_host(ets_ctx* c, int32_t layer, const void* q, void
     return ETS_OK;
 }
 
+int32_t ets_note_decode_steps(ets_ctx* c, int32_t layer, int32_t times) {
+    if (!c) return ETS_ERR_INVALID_ARG;
+    if (!c->has_tree) return fail(c, ETS_ERR_STATE, "no tree built");
+    if (layer < 0 || layer >= c->cfg.num_layers || times < 0) return fail(c, ETS_ERR_INVALID_ARG, "layer or count");
+    ets::Tree& t = c->tree;
+    std::vector<int32_t>& len = t.len[layer];
+    std::vector<int32_t> add((size_t)t.n_nodes, 0);
+    for (int32_t l = 0; l < t.n_leaves; ++l) add[t.leaf_node[l]] += times;
+    for (int32_t v = 0; v < t.n_nodes; ++v)
+        if ((int64_t)len[v] + add[v] > t.cap[v]) return fail(c, ETS_ERR_POOL_EXHAUSTED, "the replayed steps ran beyond cap_tokens");
+    for (int32_t v = 0; v < t.n_nodes; ++v) len[v] += add[v];
+    return ETS_OK;
+}
+
 int32_t ets_decode_step_host(ets_ctx* c, int32_t layer, const void* k_new, const void* v_new, const void* q, void* out,
                              float* lse, void* cuda_stream) {
     if (int32_t rc = decode_check(c, layer, q, out)) return rc;

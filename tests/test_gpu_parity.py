@@ -360,6 +360,67 @@ def test_prune_with_ets_select_then_decode_on_the_kept_tree():
     check_close(dev_to_bits(out)[subset], ref[subset], "kept tree")
 
 
+def test_decode_step_replayed_from_a_cuda_graph():
+    """One decode iteration over all layers captured into a CUDA graph and replayed: every replay appends the
+    (same) new token at the lengths the device holds and attends; after telling the library about the replays
+    the result equals the oracle on the grown tree, and an ordinary call continues from there."""
+    wl = make_workload("cfg2")
+    tree, g = wl.tree, wl.geometry
+    layers, L, R = 2, wl.tree.n_leaves, 5
+    cap = tree.tokens.copy()
+    cap[tree.leaf_node] += R + 3
+    ctx = context_for_tree(g.num_q_heads, g.num_kv_heads, g.head_dim, tree.parent, cap, tree.leaf_node, num_layers=layers)
+    ctx.tree_build(tree.parent, cap, tree.leaf_node)
+    vals = {l: node_values(tree, g, wl.value_seed, l) for l in range(layers)}
+    for l in range(layers):
+        fill_layer(ctx, l, *vals[l])
+    from workloads import query_bits
+    from oracle.tree_attention import tree_decode_attention
+    from _harness import check_close
+    rng = np.random.default_rng(4)
+    kb = {l: rng.integers(0, 1 << 16, size=(L, g.num_kv_heads, g.head_dim), dtype=np.uint16) & np.uint16(0xBFFF) for l in range(layers)}
+    vb = {l: rng.integers(0, 1 << 16, size=(L, g.num_kv_heads, g.head_dim), dtype=np.uint16) & np.uint16(0xBFFF) for l in range(layers)}
+    qb = {l: query_bits(wl.value_seed, 50 + l, L, g.num_q_heads, g.head_dim) for l in range(layers)}
+    k_d = {l: bits_to_dev(kb[l]) for l in range(layers)}
+    v_d = {l: bits_to_dev(vb[l]) for l in range(layers)}
+    q_d = {l: bits_to_dev(qb[l]) for l in range(layers)}
+    out = {l: torch.empty_like(q_d[l]) for l in range(layers)}
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for l in range(layers):     # an ordinary call first: it puts the append's descriptor list on the device
+            ctx.decode_step(l, k_d[l], v_d[l], q_d[l], out[l], None, stream=side.cuda_stream)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for l in range(layers):
+            ctx.decode_step(l, k_d[l], v_d[l], q_d[l], out[l], None, stream=side.cuda_stream)
+    # the capture itself counted as one call on the host but ran nothing; the replays run on the device
+    for _ in range(R):
+        graph.replay()
+    torch.cuda.synchronize()
+    for l in range(layers):
+        ctx.note_decode_steps(l, R - 1)
+    ctx.poll_status()
+    steps = 1 + R
+    lengths = tree.tokens.copy()
+    lengths[tree.leaf_node] += steps
+    assert ctx.get_node_len(0).tolist() == lengths.tolist()
+    subset = [0, L // 2, L - 1]
+    for l in range(layers):
+        ks = [np.concatenate([vals[l][0][n]] + ([np.repeat(kb[l][list(tree.leaf_node).index(n)][None], steps, 0)] if n in set(tree.leaf_node.tolist()) else []))
+              for n in range(tree.n_nodes)]
+        vs = [np.concatenate([vals[l][1][n]] + ([np.repeat(vb[l][list(tree.leaf_node).index(n)][None], steps, 0)] if n in set(tree.leaf_node.tolist()) else []))
+              for n in range(tree.n_nodes)]
+        ref, _ = tree_decode_attention(tree.parent, lengths, tree.leaf_node, ks, vs, qb[l], g.num_q_heads, g.num_kv_heads, leaves=subset)
+        check_close(dev_to_bits(out[l])[subset], ref[subset], f"layer {l} after {R} replays")
+    # an ordinary call continues from the lengths the replays left
+    ctx.decode_step(0, k_d[0], v_d[0], q_d[0], out[0], None)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    lengths[tree.leaf_node] += 1
+    assert ctx.get_node_len(0).tolist() == lengths.tolist()
+
+
 @pytest.mark.parametrize("pipeline", [0, 1])
 def test_decode_step_host_equals_decode_step(pipeline):
     """The host-buffer form of the fused step (first call through the two-call route, later ones through the
