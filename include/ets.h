@@ -220,8 +220,8 @@ int32_t ets_note_decode_steps(ets_ctx* ctx, int32_t layer, int32_t times);
 
 /* The same with HOST buffers (k_new, v_new, q in; out, lse back), copied through the workspace's staging
  * areas on the library's streams like ets_kv_append_host + ets_tree_attn_decode_host, in one call and
- * with one event for the three inputs.  When k_new, v_new and q are adjacent in host memory in this order
- * (the output of a fused projection) they travel in one copy.  Follows ETS_OPT_HOST_PIPELINE. */
+ * with one event for the three inputs.  With ETS_OPT_PACKED_INPUTS set, k_new, v_new and q that are
+ * adjacent in host memory in this order (the output of a fused projection) travel in one copy.  Follows ETS_OPT_HOST_PIPELINE. */
 int32_t ets_decode_step_host(ets_ctx* ctx, int32_t layer, const void* k_new, const void* v_new,
                              const void* q, void* out, float* lse, void* cuda_stream);
 
@@ -335,6 +335,10 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
                                  /* for callers whose k_new / v_new are complete when the call is made: not    */
                                  /* when the kernel that writes them is the one before the call in the stream   */
                                  /* and signals early itself.  Default 0.                                      */
+#define ETS_OPT_PACKED_INPUTS 9  /* 1: the caller promises that whenever k_new, v_new and q of ets_decode_step_host  */
+                                 /* are adjacent in this order they lie in ONE host allocation, so one copy may  */
+                                 /* span them (two pinned allocations that merely touch must not be copied as    */
+                                 /* one).  Default 0: three copies.                                             */
 #define ETS_OPT_HOST_PIPELINE 6  /* 1: the *_host calls return without making cuda_stream wait for   */
                                  /* them, so the copies of one call overlap the kernels of the next;   */
                                  /* results are valid after ets_host_join + synchronising that stream;  */

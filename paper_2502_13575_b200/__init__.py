@@ -10,7 +10,7 @@ _BINDING_NAMES = (
     "EtsContext", "EtsError", "ets_config", "ets_pool_bytes", "ets_select", "ets_version", "make_config", "lib",
     "ETS_OK", "ETS_ERR_INVALID_ARG", "ETS_ERR_BAD_TREE", "ETS_ERR_POOL_EXHAUSTED", "ETS_ERR_UNSUPPORTED",
     "ETS_ERR_STATE", "ETS_ERR_CUDA", "ETS_ERR_DEVICE_TIMEOUT",
-    "ETS_OPT_CHUNK_PAGES", "ETS_OPT_KERNEL", "ETS_OPT_TIMING", "ETS_OPT_WIDE", "ETS_OPT_HOST_PIPELINE", "ETS_OPT_PATH_ITEMS", "ETS_OPT_OVERLAP_APPEND",
+    "ETS_OPT_CHUNK_PAGES", "ETS_OPT_KERNEL", "ETS_OPT_TIMING", "ETS_OPT_WIDE", "ETS_OPT_HOST_PIPELINE", "ETS_OPT_PATH_ITEMS", "ETS_OPT_OVERLAP_APPEND", "ETS_OPT_PACKED_INPUTS",
 )
 
 

@@ -31,6 +31,7 @@ ETS_OPT_WIDE = 4
 ETS_OPT_HOST_PIPELINE = 6
 ETS_OPT_PATH_ITEMS = 7
 ETS_OPT_OVERLAP_APPEND = 8
+ETS_OPT_PACKED_INPUTS = 9
 
 _ERR_NAMES = {
     -1: "ETS_ERR_INVALID_ARG", -2: "ETS_ERR_BAD_TREE", -3: "ETS_ERR_POOL_EXHAUSTED",

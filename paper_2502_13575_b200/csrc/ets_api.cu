@@ -172,6 +172,7 @@ struct ets_ctx {
     int32_t opt_kernel = 0;
     bool opt_path_items = false;
     bool opt_overlap_append = false;
+    bool opt_packed_inputs = false;
     // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256 tree and on
     // eight width-64 trees: 33 beats 17, 49, 65 and "never" (below ~32 rows the per-item latency of the wide
     // kernel costs more than the re-reads by the narrow kernel that it saves).
@@ -395,6 +396,9 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
             return ETS_OK;
         case ETS_OPT_OVERLAP_APPEND:
             c->opt_overlap_append = value != 0;
+            return ETS_OK;
+        case ETS_OPT_PACKED_INPUTS:
+            c->opt_packed_inputs = value != 0;
             return ETS_OK;
         case ETS_OPT_PATH_ITEMS:
             c->opt_path_items = value != 0;
@@ -907,8 +911,10 @@ int32_t ets_decode_step_host(ets_ctx* c, int32_t layer, const void* k_new, const
     char* vd = c->ws + c->lay.v_stage + hk * c->lay.kv_stride;
     char* qd = c->ws + c->lay.q_stage + hb * c->lay.q_stride;
     // A fused projection leaves k, v and q of a layer next to each other; then one copy brings all three
-    // (a host-to-device copy of half a megabyte costs about as much in set-up as in transfer).
-    const bool packed = (const char*)v_new == (const char*)k_new + kvbytes && (const char*)q == (const char*)v_new + kvbytes;
+    // (a host-to-device copy of half a megabyte costs about as much in set-up as in transfer).  Adjacent
+    // addresses alone do not prove one allocation (two pinned blocks can touch, and a copy may not span
+    // them), so the caller has to promise it.
+    const bool packed = c->opt_packed_inputs && (const char*)v_new == (const char*)k_new + kvbytes && (const char*)q == (const char*)v_new + kvbytes;
     if (packed) {
         kd = c->ws + c->lay.pk_stage + hb * c->lay.pk_stride;   // guarded by the same events as the q area
         vd = kd + kvbytes;

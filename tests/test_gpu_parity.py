@@ -390,6 +390,8 @@ def test_decode_step_replayed_from_a_cuda_graph():
         for l in range(layers):     # an ordinary call first: it puts the append's descriptor list on the device
             ctx.decode_step(l, k_d[l], v_d[l], q_d[l], out[l], None, stream=side.cuda_stream)
     side.synchronize()
+    import gc
+    gc.collect()    # a context of an earlier test collected during the capture would synchronise the device inside it
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph, stream=side):
         for l in range(layers):
@@ -451,7 +453,8 @@ def test_decode_step_host_equals_decode_step(pipeline):
             out_d = torch.empty_like(q)
             lse_d = torch.empty((L, g.num_q_heads), dtype=torch.float32, device="cuda")
             dev.decode_step(l, bits_to_dev(kb), bits_to_dev(vb), q, out_d, lse_d)
-            if (tok + l) % 2:   # separate buffers: three copies
+            host.set_option(ets.ETS_OPT_PACKED_INPUTS, 1 - (tok + l) % 2)
+            if (tok + l) % 2:   # separate buffers (which may happen to touch): three copies
                 k_h = torch.from_numpy(kb.view(np.int16)).pin_memory()
                 v_h = torch.from_numpy(vb.view(np.int16)).pin_memory()
                 q_h = torch.from_numpy(qb.view(np.int16)).pin_memory()

@@ -76,6 +76,7 @@ class DecodeJob:
             self.ctx.set_option(ets.ETS_OPT_WIDE, wide)
         # the step inputs below are resident before any call: appends may run under the preceding merge kernel
         self.ctx.set_option(ets.ETS_OPT_OVERLAP_APPEND, 1)
+        self.ctx.set_option(ets.ETS_OPT_PACKED_INPUTS, 1)   # decode_tokens() packs k | v | q of a layer in one pinned buffer
         self.keep = np.arange(tree.n_nodes, dtype=np.int32)
         self.ctx.tree_build(tree.parent, self.cap, tree.leaf_node)
         # pools
