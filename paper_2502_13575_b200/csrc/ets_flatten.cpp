@@ -75,7 +75,12 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             if (o < 0) continue;
             int32_t have = prev.node_page_off[o + 1] - prev.node_page_off[o];
             claimed_old[o] = std::min(have, need[i]);
-            for (int32_t l = 0; l < L; ++l) t.len[l][i] = std::min(prev.len[l][o], cap_tokens[i]);
+        }
+        for (int32_t l = 0; l < L; ++l) {
+            int32_t* dst = t.len[l].data();
+            const int32_t* src = prev.len[l].data();
+            for (int32_t i = 0; i < n_nodes; ++i)
+                if (keep_pages_of[i] >= 0) dst[i] = std::min(src[keep_pages_of[i]], cap_tokens[i]);
         }
     }
     t.free_heap = prev.free_heap;
@@ -137,17 +142,19 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     // ---- segments: a node continues its parent's segment iff both have the same leaves below
     std::vector<int32_t> seg_of((size_t)n_nodes, -1);
     std::vector<int32_t> seg_head;                 // first node of each segment
-    std::vector<std::vector<int32_t>> seg_nodes;   // nodes in root-to-leaf order
+    std::vector<int32_t> seg_last;                 // last node of each segment so far
+    std::vector<int32_t> seg_next((size_t)n_nodes, -1);   // the segment's next node towards the leaves
     for (int32_t i = 0; i < n_nodes; ++i) {
         if (g[i] == 0) continue;
         int32_t pa = parent[i];
         if (pa >= 0 && g[pa] == g[i]) {
             seg_of[i] = seg_of[pa];
-            seg_nodes[seg_of[i]].push_back(i);
+            seg_next[seg_last[seg_of[i]]] = i;
+            seg_last[seg_of[i]] = i;
         } else {
             seg_of[i] = (int32_t)seg_head.size();
             seg_head.push_back(i);
-            seg_nodes.push_back({i});
+            seg_last.push_back(i);
         }
     }
     const int32_t n_seg = (int32_t)seg_head.size();
@@ -157,14 +164,14 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     std::vector<int32_t> seg_unit_off((size_t)n_seg + 1, 0);
     for (int32_t s = 0; s < n_seg; ++s) {
         int32_t cnt = 0;
-        for (int32_t v : seg_nodes[s]) cnt += need[v];
+        for (int32_t v = seg_head[s]; v >= 0; v = seg_next[v]) cnt += need[v];
         seg_unit_off[s + 1] = seg_unit_off[s] + cnt;
     }
     const int64_t n_units = seg_unit_off[n_seg];
     t.unit.resize((size_t)n_units * 4);
     for (int32_t s = 0; s < n_seg; ++s) {
         int32_t u = seg_unit_off[s];
-        for (int32_t v : seg_nodes[s])
+        for (int32_t v = seg_head[s]; v >= 0; v = seg_next[v])
             for (int32_t j = 0; j < need[v]; ++j, ++u) {
                 t.unit[4 * (size_t)u + 0] = t.page_ids[t.node_page_off[v] + j];
                 t.unit[4 * (size_t)u + 1] = v;
@@ -243,7 +250,16 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     }
     std::vector<Part> best_parts;
     {
-        auto by_len = [](const Part& a, const Part& b) { return a.len > b.len; };
+        // stable order by falling length (a piece holds at most 32 page slots): a counting sort
+        std::vector<Part> sorted;
+        auto sort_by_len = [&](std::vector<Part>& v) {
+            size_t first[34] = {};
+            for (const Part& q : v) ++first[32 - q.len + 1];
+            for (int k = 1; k < 34; ++k) first[k] += first[k - 1];
+            sorted.resize(v.size());
+            for (const Part& q : v) sorted[first[32 - q.len]++] = q;
+            v.swap(sorted);
+        };
         auto cut = [](std::vector<Part>& out, int32_t seg, int32_t begin, int32_t len, int32_t c) {
             const int32_t np_ = (len + c - 1) / c;
             for (int32_t k = 0; k < np_; ++k) {
@@ -257,7 +273,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             mult_of[q.seg] = q.mult;
             cut(best_parts, q.seg, 0, q.nu, cap);
         }
-        std::stable_sort(best_parts.begin(), best_parts.end(), by_len);
+        sort_by_len(best_parts);
         for (const Part& q : best_parts) total_pieces += mult_of[q.seg];
         if (tail_cap < cap && total_pieces > n_workers) {
             // the parts that hold the last n_workers pieces of the queue are cut down to tail_cap
@@ -268,10 +284,15 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             for (size_t k = first; k < best_parts.size(); ++k) cut(tail, best_parts[k].seg, best_parts[k].begin, best_parts[k].len, tail_cap);
             best_parts.resize(first);
             best_parts.insert(best_parts.end(), tail.begin(), tail.end());
-            std::stable_sort(best_parts.begin(), best_parts.end(), by_len);
+            sort_by_len(best_parts);
         }
     }
     int64_t slots = 0;
+    {
+        size_t n_items_narrow = 0;
+        for (const Part& q : best_parts) n_items_narrow += (size_t)p.num_kv_heads * ceil_div(g[seg_head[q.seg]], leaves_per_tile);
+        t.items.reserve(n_items_narrow + 64);
+    }
     for (const Part& q : best_parts) {
         const int32_t head_node = seg_head[q.seg];
         const int32_t gn = g[head_node];
