@@ -324,6 +324,9 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
                                  /* rebuild the tree after changing it                             */
 #define ETS_OPT_WIDE          4  /* smallest query group, in rows (leaves * Hq/Hkv, at least 17), that */
                                  /* goes to the tcgen05 kernel (default 33); 0: none.  Next build.      */
+                                 /* While the option is untouched, a tree so small that a warp of the    */
+                                 /* streaming kernel would read four page slots or fewer gets no such    */
+                                 /* items (the second kernel's launch costs more than it saves there).   */
 #define ETS_OPT_PATH_ITEMS    7  /* 1: the next builds serve ets_tree_attn_prefill only: a work item is one   */
                                  /* (node that leaves sit at, kv head, tile of its leaves) and walks the node's */
                                  /* whole path, so a dense tile keeps its accumulator resident and leaves one  */

@@ -172,6 +172,7 @@ struct ets_ctx {
     int32_t opt_kernel = 0;
     bool opt_path_items = false;
     bool opt_overlap_append = false;
+    bool opt_wide_set = false;   // the caller chose the wide threshold: no small-tree exception
     bool opt_packed_inputs = false;
     // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256 tree and on
     // eight width-64 trees: 33 beats 17, 49, 65 and "never" (below ~32 rows the per-item latency of the wide
@@ -393,6 +394,7 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
         case ETS_OPT_WIDE:
             if (value < 0 || value > 1 << 20) return fail(c, ETS_ERR_INVALID_ARG, "wide threshold out of range");
             c->opt_wide = (int32_t)value;
+            c->opt_wide_set = true;
             return ETS_OK;
         case ETS_OPT_OVERLAP_APPEND:
             c->opt_overlap_append = value != 0;
@@ -420,6 +422,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
     fp.chunk_pages = c->opt_chunk_pages;
     fp.wide_rows = (c->opt_wide > 0 && c->opt_kernel == 0) ? 128 : 0;
     fp.wide_min_rows = c->opt_wide;
+    if (c->opt_wide_set) fp.wide_min_work = 0;
     fp.path_items = c->opt_path_items;
     ets::Tree next;
     std::string err;

@@ -190,9 +190,19 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     const int32_t leaves_per_tile = std::max(1, p.rows_per_item / std::max(1, p.gqa));
     const int32_t n_workers = std::max(1, p.n_workers);
     const int32_t max_run = std::min(32, p.chunk_pages > 0 ? p.chunk_pages : 32);
+    // A very small tree is left to the narrow kernel alone: the second kernel costs a fork and a join of
+    // streams, a few microseconds, which is more than it saves when a warp has only a handful of page
+    // slots to read anyway (measured on a width-16 tree: 16.8 us without, 20.5 us with the second kernel).
+    bool wide_pays = p.wide_rows > 0;
+    if (wide_pays && !p.path_items) {
+        int64_t all_narrow = 0;   // (page slot, kv head, leaf tile) visits if every segment were narrow
+        for (int32_t s = 0; s < n_seg; ++s)
+            all_narrow += (int64_t)(seg_unit_off[s + 1] - seg_unit_off[s]) * p.num_kv_heads * ceil_div(g[seg_head[s]], leaves_per_tile);
+        wide_pays = all_narrow > (int64_t)p.wide_min_work * n_workers;
+    }
     auto is_wide = [&](int32_t s) {
         const int32_t r = g[seg_head[s]] * p.gqa;
-        return p.wide_rows > 0 && r > p.rows_per_item && r >= p.wide_min_rows;
+        return wide_pays && r > p.rows_per_item && r >= p.wide_min_rows;
     };
     struct Part { int32_t seg, begin, len; };
     // per narrow segment: page slots, pieces per part (heads x leaf tiles), mean weight of a page slot

@@ -258,6 +258,29 @@ def test_narrow_queue_is_ordered_longest_first(name):
             prev = k
 
 
+def test_small_trees_get_no_wide_items_unless_asked():
+    """A tree on which a warp of the streaming kernel would visit four page slots or fewer is left to that
+    kernel alone (the second kernel's launch costs more than it saves); setting the threshold explicitly
+    switches the exception off, and larger trees keep their wide items."""
+    def items(name, wide=None):
+        wl = make_workload(name)
+        g = wl.geometry
+        ctx = host_ctx(g.num_q_heads, g.num_kv_heads, g.head_dim, pages=1 << 15, max_path_entries=1 << 14)
+        if wide is not None:
+            ctx.set_option(ets.ETS_OPT_WIDE, wide)
+        ctx.tree_build(wl.tree.parent, wl.tree.tokens, wl.tree.leaf_node)
+        n_narrow = ctx.get_stats()["n_narrow_items"]
+        item = ctx.work_export()["item"]
+        _check_work(ctx, wl.tree, wl.tree.tokens, g.num_kv_heads, g.gqa)
+        return n_narrow, len(item)
+    n_narrow, n_items = items("cfg2")
+    assert n_narrow == n_items                  # root group of 64 rows, but only ~2.4 page slots per warp
+    n_narrow, n_items = items("cfg2", wide=33)
+    assert n_narrow < n_items
+    n_narrow, n_items = items("cfg3_ets")
+    assert n_narrow < n_items
+
+
 def test_path_items_cover_every_path_once():
     """ETS_OPT_PATH_ITEMS: one item per (node that leaves sit at, kv head, tile of those leaves); its page slots
     are the node's whole path in root-to-node order; every leaf gets exactly one partial slot per kv head; the
