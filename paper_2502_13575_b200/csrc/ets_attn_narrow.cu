@@ -223,7 +223,7 @@ __device__ __forceinline__ void tile_step(uint32_t kt, uint32_t vt, int valid, f
     }
 
     // online softmax (log2 units); this lane holds tokens grp and grp+8 of rows 2quad, 2quad+1
-    uint32_t pf[NT][2];
+    uint32_t pf[NT][2], pg[NT][2];
 #pragma unroll
     for (int j = 0; j < NT; ++j) {
         float sv[4];
@@ -232,7 +232,7 @@ __device__ __forceinline__ void tile_step(uint32_t kt, uint32_t vt, int valid, f
             const int tok = grp + (i >> 1) * 8;
             sv[i] = tok < valid ? s[j][i] * scale_log2 : -INFINITY;
         }
-        float p[4];
+        float p[4], pl[4];
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             float mx = fmaxf(sv[r], sv[r + 2]);
@@ -241,11 +241,15 @@ __device__ __forceinline__ void tile_step(uint32_t kt, uint32_t vt, int valid, f
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
             const float mn = fmaxf(acc.m[j][r], mx);     // finite: token 0 of the tile is valid
             const float corr = exp2f(acc.m[j][r] - mn);
-            // weights are rounded to bf16 here, so that the row sum and the product use the same
-            // values and the rounding cancels in sum(p v) / sum(p)
-            p[r] = __bfloat162float(__float2bfloat16_rn(exp2f(sv[r] - mn)));
-            p[r + 2] = __bfloat162float(__float2bfloat16_rn(exp2f(sv[r + 2] - mn)));
-            acc.l[j][r] = acc.l[j][r] * corr + p[r] + p[r + 2];
+            // A weight enters the product as two bf16 terms, its rounded value and the rounded rest
+            // (16 bits of it in all): with one term the weights would be off by up to 2^-8 each, which
+            // on a path of a few tokens with values of opposite sign exceeds the output's tolerance.
+            const float e0 = exp2f(sv[r] - mn), e1 = exp2f(sv[r + 2] - mn);
+            p[r] = __bfloat162float(__float2bfloat16_rn(e0));
+            p[r + 2] = __bfloat162float(__float2bfloat16_rn(e1));
+            pl[r] = e0 - p[r];
+            pl[r + 2] = e1 - p[r + 2];
+            acc.l[j][r] = acc.l[j][r] * corr + e0 + e1;
             acc.m[j][r] = mn;
 #pragma unroll
             for (int mt = 0; mt < KS; ++mt) {
@@ -256,6 +260,8 @@ __device__ __forceinline__ void tile_step(uint32_t kt, uint32_t vt, int valid, f
         // P^T as B operand: transpose the two 8x8 (token x row) blocks
         pf[j][0] = movmatrix_trans(pack_bf16(p[0], p[1]));
         pf[j][1] = movmatrix_trans(pack_bf16(p[2], p[3]));
+        pg[j][0] = movmatrix_trans(pack_bf16(pl[0], pl[1]));
+        pg[j][1] = movmatrix_trans(pack_bf16(pl[2], pl[3]));
     }
 
     // O^T += V_tile^T . P^T
@@ -265,6 +271,8 @@ __device__ __forceinline__ void tile_step(uint32_t kt, uint32_t vt, int valid, f
         ldsm_x4_trans((v_lane + (uint32_t)(mt >> 2) * 1024u) ^ (uint32_t)((mt & 3) << 5), af);
 #pragma unroll
         for (int j = 0; j < NT; ++j) mma_bf16(acc.o[mt][j], af, pf[j]);
+#pragma unroll
+        for (int j = 0; j < NT; ++j) mma_bf16(acc.o[mt][j], af, pg[j]);
     }
 }
 

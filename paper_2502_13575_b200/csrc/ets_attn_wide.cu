@@ -41,6 +41,10 @@ constexpr uint32_t kTmemCols = 256;
 // S has two buffers of 64 columns (a stage is 64 tokens): the product of the next stage is issued while the
 // softmax warps still work on this one.
 constexpr uint32_t kColS = 0, kColP = 0, kColO = 128, kColSBuf = 64;
+// P of a pair of page slots replaces the pair's S (32 columns): 16 columns of bf16 weights, then 16 columns
+// with their second bf16 term (what rounding the first left over)
+constexpr uint32_t kColPLo = 16;
+__host__ __device__ constexpr uint32_t p_col(int k) { return 32u * (uint32_t)(k >> 1) + 8u * (uint32_t)(k & 1); }
 static_assert(kStageUnits * 16 <= (int)kColSBuf && kStages == 2, "S double buffer: 64-token stages, two of them");
 constexpr float kRescaleThreshold = 0.0f;      // log2 units; see the softmax role
 
@@ -195,8 +199,10 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, Sha
     return ok;
 }
 
+// At most 88 registers: next to the streaming kernel's CTA (8 warps of 168 registers, two per scheduler) a
+// scheduler's 16,384 registers leave room for two of this kernel's warps only up to that size.
 template <int D>
-__global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first_item) {
+__global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first_item) {
     constexpr uint32_t TB = 16 * D * 2;                  // one tile
     constexpr uint32_t STAGE_HALF = kStageUnits * TB;    // K (or V) part of a stage
     constexpr int KS = D / 16;                           // k-steps of the QK product
@@ -399,8 +405,12 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
             tc_fence_after();
             if (lane == 0) {
                 for (int k = 0; k < n; ++k)
-                    umma_ts(tmem + kColO, tmem + kColP + kColSBuf * (st & 1u) + 8u * k, smem_desc(vst + k * TB, 1024, 1024u * (D / 64)),
+                    umma_ts(tmem + kColO, tmem + kColP + kColSBuf * (st & 1u) + p_col(k), smem_desc(vst + k * TB, 1024, 1024u * (D / 64)),
                             idesc_pv, !(st == 0 && k == 0));
+                // the weights' second term
+                for (int k = 0; k < n; ++k)
+                    umma_ts(tmem + kColO, tmem + kColP + kColPLo + kColSBuf * (st & 1u) + p_col(k), smem_desc(vst + k * TB, 1024, 1024u * (D / 64)),
+                            idesc_pv, true);
                 umma_commit(smem_u32(&sh->empty[s]));
                 umma_commit(smem_u32(&sh->o_ready));
             }
@@ -490,8 +500,10 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                 m_ref = m_new;
             }
             // pass 2: P = 2^(s - m_ref), packed bf16 into the A operand of the second product, two page
-            // slots per step with independent sums.  The row sum uses the bf16-rounded weights, the
-            // same ones the product uses, so the rounding cancels in sum(p v) / sum(p).
+            // slots per step with independent sums.  A weight goes in as two bf16 terms, its rounded
+            // value and the rounded rest: with one term the weights would be off by up to 2^-8 each,
+            // which on a path of a few tokens with values of opposite sign exceeds the output's
+            // tolerance.  Both terms of a pair go where the pair's S was.
             float l0 = 0.f, l1 = 0.f;
             const float neg_ref = -m_ref;
             for (int c = 0; c < n; c += 2) {
@@ -499,7 +511,7 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                 tmem_ld32(tlane + kColS + kColSBuf * (st & 1u) + 16u * c, v);
                 const int v0 = row_valid(s, c);
                 const int v1 = c + 1 < n ? row_valid(s, c + 1) : 0;
-                uint32_t pk[16];
+                uint32_t pk[16], plo[16];
                 const bool full = v0 == 16 && v1 == 16;
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
@@ -511,12 +523,17 @@ __global__ void __maxnreg__(80) attn_partial_wide_kernel(DecodeArgs a, int first
                     const float b1 = (full || i + 1 < v1) ? ex2_approx(fmaf(v[16 + i + 1], a.scale_log2, neg_ref)) : 0.f;
                     const __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1);
                     const __nv_bfloat162 pb = __floats2bfloat162_rn(b0, b1);
-                    l0 += __low2float(pa) + __high2float(pa);
-                    l1 += __low2float(pb) + __high2float(pb);
+                    const __nv_bfloat162 qa = __floats2bfloat162_rn(a0 - __low2float(pa), a1 - __high2float(pa));
+                    const __nv_bfloat162 qb = __floats2bfloat162_rn(b0 - __low2float(pb), b1 - __high2float(pb));
+                    l0 += a0 + a1;
+                    l1 += b0 + b1;
                     pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pa);
                     pk[8 + (i >> 1)] = *reinterpret_cast<const uint32_t*>(&pb);
+                    plo[i >> 1] = *reinterpret_cast<const uint32_t*>(&qa);
+                    plo[8 + (i >> 1)] = *reinterpret_cast<const uint32_t*>(&qb);
                 }
-                tmem_st16(tlane + kColP + kColSBuf * (st & 1u) + 8u * c, pk);
+                tmem_st16(tlane + kColP + kColSBuf * (st & 1u) + p_col(c), pk);
+                tmem_st16(tlane + kColP + kColPLo + kColSBuf * (st & 1u) + p_col(c), plo);
             }
             l += l0 + l1;
             tmem_wait_st();

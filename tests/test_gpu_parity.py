@@ -160,6 +160,23 @@ def test_random_small_trees_with_edge_cases():
         done += 1
 
 
+@pytest.mark.parametrize("seed", [52, 65, 81, 116, 144, 171, 241, 265, 479])
+def test_short_paths_with_cancelling_values_keep_the_tolerance(seed):
+    """Paths of a few tokens where two or three weights dominate and their values have opposite signs: the
+    output is small and the error of the weights shows.  With the weights entering the second product as a
+    single bf16 term (off by up to 2^-8 each) these trees missed the tolerance by up to 1.5e-3; the kernels
+    split each weight into two bf16 terms.  Trees, shapes and kernel choices as drawn by the seed."""
+    rng = np.random.default_rng(seed)
+    big = rng.integers(0, 3)
+    tree = random_small_tree(rng, max_nodes=[10, 40, 120][big], max_tokens=[70, 300, 200][big], max_leaves=[7, 40, 100][big])
+    lengths = np.array([int(rng.integers(0, t + 1)) for t in tree.tokens], np.int32)
+    hkv = int(rng.choice([1, 2, 8]))
+    gqa = int(rng.choice([1, 2, 4, 8, 16]))
+    d = int(rng.choice([64, 128]))
+    wide = [None, 17, 33, 65, 0][int(rng.integers(0, 5))]
+    run_and_check(tree, Geometry(hkv * gqa, hkv, d), 5000 + seed + 1, cap=tree.tokens, lengths=lengths, wide=wide)
+
+
 def test_single_token_tree_returns_v():
     g = Geometry(4, 2, 64)
     tree = Tree(np.array([-1], np.int32), np.array([1], np.int32), np.array([0], np.int32))
