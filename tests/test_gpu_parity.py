@@ -160,12 +160,8 @@ def test_random_small_trees_with_edge_cases():
         done += 1
 
 
-@pytest.mark.parametrize("seed", [52, 65, 81, 116, 144, 171, 241, 265, 479])
-def test_short_paths_with_cancelling_values_keep_the_tolerance(seed):
-    """Paths of a few tokens where two or three weights dominate and their values have opposite signs: the
-    output is small and the error of the weights shows.  With the weights entering the second product as a
-    single bf16 term (off by up to 2^-8 each) these trees missed the tolerance by up to 1.5e-3; the kernels
-    split each weight into two bf16 terms.  Trees, shapes and kernel choices as drawn by the seed."""
+def _seeded_case(seed):
+    """A random tree with random lengths below capacity, head shape and kernel choice, all drawn from the seed."""
     rng = np.random.default_rng(seed)
     big = rng.integers(0, 3)
     tree = random_small_tree(rng, max_nodes=[10, 40, 120][big], max_tokens=[70, 300, 200][big], max_leaves=[7, 40, 100][big])
@@ -174,7 +170,34 @@ def test_short_paths_with_cancelling_values_keep_the_tolerance(seed):
     gqa = int(rng.choice([1, 2, 4, 8, 16]))
     d = int(rng.choice([64, 128]))
     wide = [None, 17, 33, 65, 0][int(rng.integers(0, 5))]
-    run_and_check(tree, Geometry(hkv * gqa, hkv, d), 5000 + seed + 1, cap=tree.tokens, lengths=lengths, wide=wide)
+    return tree, lengths, Geometry(hkv * gqa, hkv, d), wide
+
+
+def test_random_trees_of_mixed_size():
+    """Sixty seeded trees of up to 120 nodes and 100 leaves (forests, repeated and internal leaves, empty nodes),
+    G from 1 to 16, 1 to 8 kv heads, both head sizes, wide threshold default / 17 / 33 / 65 / off."""
+    done, seed = 0, 3000
+    while done < 60:
+        tree, lengths, geom, wide = _seeded_case(seed)
+        seed += 1
+        path_tokens = np.zeros(tree.n_nodes, np.int64)
+        for v in range(tree.n_nodes):
+            p = int(tree.parent[v])
+            path_tokens[v] = int(lengths[v]) + (path_tokens[p] if p >= 0 else 0)
+        if np.any(path_tokens[tree.leaf_node] == 0):   # every leaf needs a token on its path
+            continue
+        run_and_check(tree, geom, 5000 + seed, cap=tree.tokens, lengths=lengths, wide=wide)
+        done += 1
+
+
+@pytest.mark.parametrize("seed", [52, 65, 81, 116, 144, 171, 241, 265, 479])
+def test_short_paths_with_cancelling_values_keep_the_tolerance(seed):
+    """Paths of a few tokens where two or three weights dominate and their values have opposite signs: the
+    output is small and the error of the weights shows.  With the weights entering the second product as a
+    single bf16 term (off by up to 2^-8 each) these trees missed the tolerance by up to 1.5e-3; the kernels
+    split each weight into two bf16 terms.  Trees, shapes and kernel choices as drawn by the seed."""
+    tree, lengths, geom, wide = _seeded_case(seed)
+    run_and_check(tree, geom, 5000 + seed + 1, cap=tree.tokens, lengths=lengths, wide=wide)
 
 
 def test_single_token_tree_returns_v():
