@@ -175,9 +175,10 @@ struct ets_ctx {
     bool opt_wide_set = false;   // the caller chose the wide threshold: no small-tree exception
     bool opt_packed_inputs = false;
     // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256 tree and on
-    // eight width-64 trees: 33 beats 17, 49, 65 and "never" (below ~32 rows the per-item latency of the wide
-    // kernel costs more than the re-reads by the narrow kernel that it saves).
-    int32_t opt_wide = 33;
+    // eight width-64 trees: 33, 49 and 65 are within a microsecond of each other per layer, 17 and "never" are
+    // 20 % slower (below ~32 rows the per-item latency of the wide kernel costs more than the re-reads by the
+    // narrow kernel that it saves); 49 gives the shortest whole step on the width-256 tree.
+    int32_t opt_wide = 49;
     bool opt_timing = false;
     // timing
     std::vector<cudaEvent_t> tev;   // 3 per timed call
