@@ -17,7 +17,7 @@ Plain, slow restatement of Section 4 and Appendix B of the paper in fp64:
   ets_step         weights -> selection -> weights again over the kept trajectories (Eq. 3).
 
 Pins: tests/test_oracle_selection.py (hand-worked trees, lambda = 0 and large-lambda closed forms,
-monotonicity in lambda_b, invariance under relabelling).
+monotonicity in lambda_b, invariance under relabelling; ets_step as a whole on a hand-worked six-node tree).
 """
 from __future__ import annotations
 

@@ -49,7 +49,8 @@ def check_close(gpu_bits, oracle, what=""):
 
 
 def run_and_check(tree, geom, value_seed, *, layers=(0,), qscale=1.0, chunk_pages=None, kernel=None, wide=None,
-                  cap=None, lengths=None, leaves_subset=None, host_api=False, sm_scale=0.0, ctx=None):
+                  cap=None, lengths=None, leaves_subset=None, host_api=False, sm_scale=0.0, ctx=None,
+                  aligned_q=False):
     """Build, fill, decode every requested layer, compare with the oracle.  Returns the context."""
     cap = tree.tokens if cap is None else cap
     lengths = tree.tokens if lengths is None else lengths
@@ -67,7 +68,7 @@ def run_and_check(tree, geom, value_seed, *, layers=(0,), qscale=1.0, chunk_page
     for layer in layers:
         ks, vs = node_values(tree, geom, value_seed, layer, lengths)
         fill_layer(ctx, layer, ks, vs)
-        qb = query_bits(value_seed, layer, L, geom.num_q_heads, geom.head_dim, qscale)
+        qb = query_bits(value_seed, layer, L, geom.num_q_heads, geom.head_dim, qscale, aligned_with_node2=aligned_q)
         if host_api:
             q_h = torch.from_numpy(qb.view(np.int16)).pin_memory()
             out_h = torch.empty_like(q_h).pin_memory()

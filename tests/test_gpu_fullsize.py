@@ -1,7 +1,8 @@
-"""Full-size parity in the launch configuration bench.py times: the width-256, 32-layer workload
-driven through workloads.loader.DecodeJob.step (flatten + append + decode per layer), checked
-on sampled leaves and layers that the oracle computes one by one; plus properties that hold at
-any size (finite outputs, convexity bounds are covered by the sampled comparison)."""
+"""Full-size parity in the launch configuration bench.py times: every workload driven through
+workloads.loader.DecodeJob.step (flatten + append + decode per layer) and compared with the oracle on
+EVERY leaf: all 256 leaves of the width-256 tree on its first, a middle and its last layer, all leaves
+of layer 0 for the others.  A defect tied to a single work item (a tail piece, a re-read tile) touches
+a few rows only; sampling a handful of leaves would let it through."""
 import numpy as np
 import pytest
 import torch
@@ -26,16 +27,14 @@ def _check_job(job, layers, leaves):
     assert torch.isfinite(job.out.float()).all()
 
 
-def test_cfg4_all_layers_sampled():
+def test_cfg4_every_leaf_on_three_layers():
     wl = make_workload("cfg4")
     job = DecodeJob(wl, headroom=4, device=0, host_buffers=False)
     for _ in range(2):
         job.step()
     torch.cuda.synchronize()
     job.ctx.poll_status()
-    rng = np.random.default_rng(3)
-    leaves = sorted(set([0, wl.tree.n_leaves - 1] + [int(x) for x in rng.integers(0, wl.tree.n_leaves, 4)]))
-    _check_job(job, [0, 13, 31], leaves)
+    _check_job(job, [0, 13, 31], list(range(wl.tree.n_leaves)))
     st = job.ctx.get_stats()
     assert st["unique_tokens"] == int(wl.tree.tokens.sum()) + 2 * wl.tree.n_leaves
     # the host-buffer entry points give the same bytes as the device ones
@@ -50,12 +49,11 @@ def test_cfg4_all_layers_sampled():
     assert np.array_equal(a, b)
 
 
-@pytest.mark.parametrize("name", ["cfg3_diverse", "cfg3_ets", "cfg5a", "cfg5c"])
+@pytest.mark.parametrize("name", ["cfg3_diverse", "cfg3_ets", "cfg5a", "cfg5b", "cfg5c", "forest_w64x8"])
 def test_other_configs_through_the_step_path(name):
     wl = make_workload(name)
     job = DecodeJob(wl, headroom=3, device=0, host_buffers=False)
     job.step()
     torch.cuda.synchronize()
     job.ctx.poll_status()
-    L = wl.tree.n_leaves
-    _check_job(job, [0], [0, L // 3, L - 1])
+    _check_job(job, [0], list(range(wl.tree.n_leaves)))

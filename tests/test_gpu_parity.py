@@ -190,14 +190,17 @@ def test_random_trees_of_mixed_size():
         done += 1
 
 
+@pytest.mark.parametrize("aligned_q", [True, False])
 @pytest.mark.parametrize("seed", [52, 65, 81, 116, 144, 171, 241, 265, 479])
-def test_short_paths_with_cancelling_values_keep_the_tolerance(seed):
+def test_short_paths_with_cancelling_values_keep_the_tolerance(seed, aligned_q):
     """Paths of a few tokens where two or three weights dominate and their values have opposite signs: the
     output is small and the error of the weights shows.  With the weights entering the second product as a
     single bf16 term (off by up to 2^-8 each) these trees missed the tolerance by up to 1.5e-3; the kernels
-    split each weight into two bf16 terms.  Trees, shapes and kernel choices as drawn by the seed."""
+    split each weight into two bf16 terms.  Trees, shapes and kernel choices as drawn by the seed.  The nine
+    seeds were found with queries that repeat node 2's K rows (query_bits(aligned_with_node2=True)), which
+    makes the softmax below that node sharply peaked; they are run that way and with independent queries."""
     tree, lengths, geom, wide = _seeded_case(seed)
-    run_and_check(tree, geom, 5000 + seed + 1, cap=tree.tokens, lengths=lengths, wide=wide)
+    run_and_check(tree, geom, 5000 + seed + 1, cap=tree.tokens, lengths=lengths, wide=wide, aligned_q=aligned_q)
 
 
 def test_single_token_tree_returns_v():

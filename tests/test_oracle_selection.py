@@ -74,6 +74,33 @@ def test_objective_by_hand():
     assert keep == [2] and val == pytest.approx(-0.1)
 
 
+def test_ets_step_by_hand():
+    """The whole step on the six-node tree, every value worked out from Eq. 1, Eq. 4 and Eq. 3.
+    exp(R/T) = 5, 2, 6 and eight continuations (no product below lands on an integer, where the ceiling
+    would hang on the last bit of exp).  Eq. 1: leaf 2 first, ceil(8*6/13) = ceil(3.69) = 4; then leaf 0,
+    ceil(4*5/7) = ceil(2.86) = 3; then leaf 1, ceil(1*2/2) = 1."""
+    r = [math.log(5.0), math.log(2.0), math.log(6.0)]
+    # lambda_b = 1.2: {2} gives 4/8 - 1.2*3/6 = -0.1, the best (see test_objective_by_hand); Eq. 3 hands all
+    # eight continuations to the one kept trajectory
+    w, keep, w2, val = ets_step(PARENT, LEAVES, r, None, 8, 1.0, 1.2, 0.0)
+    assert w.tolist() == [3, 1, 4] and keep == [2] and w2.tolist() == [0, 0, 8] and val == pytest.approx(-0.1)
+    # lambda_b = 0.9: {0,2}: 7/8 - 0.9*5/6 = 0.125; {0,1,2}: 1 - 0.9 = 0.1; {2}: 0.5 - 0.45 = 0.05; {1,2}: 5/8 - 0.75 < 0;
+    # {0}: 3/8 - 0.45 < 0; {1}: 1/8 - 0.45 < 0; {0,1}: 0.5 - 0.6 < 0.  Eq. 3 over {0, 2}: leaf 2 gets
+    # ceil(8*6/11) = ceil(4.36) = 5, leaf 0 ceil(3*5/5) = 3; the pruned leaf gets nothing
+    w, keep, w2, val = ets_step(PARENT, LEAVES, r, None, 8, 1.0, 0.9, 0.0)
+    assert w.tolist() == [3, 1, 4] and keep == [0, 2] and w2.tolist() == [3, 0, 5] and val == pytest.approx(0.125)
+    # clusters {0,1} and {2}, lambda_b = 1.2, lambda_d = 0.5: {0,2}: 7/8 - 1 + 0.5 = 0.375; {0,1,2}: 1 - 1.2 + 0.5 = 0.3;
+    # {2}: -0.1 + 0.25 = 0.15; {1,2}: 5/8 - 1 + 0.5 = 0.125; {0}: 3/8 - 0.6 + 0.25 = 0.025; {0,1}: 0.5 - 0.8 + 0.25 < 0;
+    # {1}: 1/8 - 0.6 + 0.25 < 0
+    w, keep, w2, val = ets_step(PARENT, LEAVES, r, [7, 7, 9], 8, 1.0, 1.2, 0.5)
+    assert keep == [0, 2] and w2.tolist() == [3, 0, 5] and val == pytest.approx(0.375)
+    # a colder temperature changes Eq. 1 and with it the choice: T = 0.5 squares the ratios (25, 4, 36):
+    # ceil(8*36/65) = ceil(4.43) = 5, ceil(3*25/29) = ceil(2.59) = 3, nothing left for leaf 1; at lambda_b = 0.9:
+    # {0,2}: 8/8 - 0.75 = 0.25 wins over {2}: 5/8 - 0.45 and {0,1,2}: 1 - 0.9; Eq. 3: ceil(8*36/61) = 5, then 3
+    w, keep, w2, val = ets_step(PARENT, LEAVES, r, None, 8, 0.5, 0.9, 0.0)
+    assert w.tolist() == [3, 0, 5] and keep == [0, 2] and w2.tolist() == [3, 0, 5] and val == pytest.approx(0.25)
+
+
 def test_lambda_zero_keeps_every_weighted_leaf_and_large_lambda_keeps_one():
     rng = np.random.default_rng(5)
     for _ in range(30):

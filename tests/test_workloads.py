@@ -103,3 +103,39 @@ def test_values_look_standard_normal():
     k, v = node_kv_bits(11, 0, 4096, 2, 64)
     x = bf16_bits_to_f32(k).astype(np.float64)
     assert abs(x.mean()) < 0.01 and abs(x.std() - 1.0) < 0.01
+
+
+def _row_set(bits):
+    return {r.tobytes() for r in bits.reshape(-1, bits.shape[-1])}
+
+
+def test_queries_share_no_row_with_any_node():
+    """The query stream has a key of its own: on cfg2 no query row of any of the first layers equals a K or V
+    row of any node in that layer (they once shared node 2's key, which peaked every softmax below it)."""
+    wl = make_workload("cfg2")
+    g, tree = wl.geometry, wl.tree
+    for layer in (0, 1, 2):
+        kv_rows = set()
+        for n in range(tree.n_nodes):
+            k, v = node_kv_bits(wl.value_seed, n, int(tree.tokens[n]), g.num_kv_heads, g.head_dim, layer)
+            kv_rows |= _row_set(k) | _row_set(v)
+        q = query_bits(wl.value_seed, layer, tree.n_leaves, g.num_q_heads, g.head_dim)
+        assert not (_row_set(q) & kv_rows)
+    # the deliberately aligned variant is what the name says: its rows are node 2's K rows
+    qa = query_bits(wl.value_seed, 0, tree.n_leaves, g.num_q_heads, g.head_dim, aligned_with_node2=True)
+    k2, _ = node_kv_bits(wl.value_seed, 2, int(tree.tokens[2]), g.num_kv_heads, g.head_dim, 0)
+    n = min(qa.size, k2.size)
+    assert np.array_equal(qa.reshape(-1)[:n], k2.reshape(-1)[:n])
+
+
+def test_queries_look_standard_normal_and_unpeaked():
+    """With independent N(0,1) queries the scores q.k/sqrt(d) are N(0,1): no leaf of cfg2 sees a score near
+    |q|^2/sqrt(d) = 11."""
+    from workloads import bf16_bits_to_f32 as f32
+    wl = make_workload("cfg2")
+    g, tree = wl.geometry, wl.tree
+    q = f32(query_bits(wl.value_seed, 0, tree.n_leaves, g.num_q_heads, g.head_dim)).astype(np.float64)
+    assert abs(q.mean()) < 0.02 and abs(q.std() - 1.0) < 0.02
+    k2, _ = node_kv_bits(wl.value_seed, 2, int(tree.tokens[2]), g.num_kv_heads, g.head_dim, 0)
+    s = np.einsum("lad,thd->lath", q, f32(k2).astype(np.float64)) / np.sqrt(g.head_dim)
+    assert np.abs(s).max() < 6.0

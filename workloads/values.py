@@ -9,7 +9,8 @@ not depend on how many rows are drawn in total (a node that grows keeps its old 
 Layer l > 0 re-uses the layer-0 rows with the feature axis rotated by l positions and
 the sign flipped on odd layers: exact bf16 operations that a device can repeat on its
 own copy, which keeps a 32-layer pool cheap to fill while every layer holds different
-bytes.  Queries are drawn independently per layer.
+bytes.  Queries are drawn per layer from streams of their own: their seed key has a
+fourth element, which no (value_seed, node, K|V) key of a node has.
 """
 from __future__ import annotations
 
@@ -57,11 +58,20 @@ def node_kv_bits(value_seed: int, node: int, n_tokens: int, num_kv_heads: int, h
     return layer_transform_bits(k, layer), layer_transform_bits(v, layer)
 
 
+QUERY_STREAM_TAG = 0x51554552   # fourth element of a query stream's seed key
+
+
 def query_bits(value_seed: int, layer: int, n_leaves: int, num_q_heads: int, head_dim: int,
-               scale: float = 1.0) -> np.ndarray:
+               scale: float = 1.0, aligned_with_node2: bool = False) -> np.ndarray:
     """One decode query per leaf: uint16 [n_leaves, num_q_heads, head_dim].  `scale`
-    multiplies the N(0,1) draw before rounding (peaked-softmax test cases use 4 and 8)."""
-    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([value_seed, 2, layer])))
+    multiplies the N(0,1) draw before rounding (peaked-softmax test cases use 4 and 8).
+
+    `aligned_with_node2` draws from the key (value_seed, 2, layer) instead, which is also the key of
+    node 2's K rows (layer 0) and V rows (layer 1): the query rows then repeat those rows bit for bit,
+    every leaf below node 2 meets keys with score |q|^2/sqrt(d), and its softmax is sharply peaked.
+    Kept as a deliberately hard case for the tests; no workload uses it."""
+    key = [value_seed, 2, layer] if aligned_with_node2 else [value_seed, layer, 1, QUERY_STREAM_TAG]
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence(key)))
     x = rng.standard_normal((n_leaves, num_q_heads, head_dim), dtype=np.float32)
     if scale != 1.0:
         x = x * np.float32(scale)
