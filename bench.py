@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--chunk-pages", type=int, default=None)
     ap.add_argument("--kernel", type=int, default=None)
     ap.add_argument("--wide", type=int, default=None, help="0: no tcgen05 wide-group items")
+    ap.add_argument("--chain", type=int, default=None, help="0: ordinary launches instead of the programmatic-dependent chain")
     ap.add_argument("--loop-tokens", type=int, default=16,
                     help="decode iterations of the search-step loop figure (0 = skip it)")
     ap.add_argument("--prefill", action="store_true",
@@ -70,44 +71,125 @@ def workload_description(wl, layers):
 
 
 # ----------------------------------------------------------------------------- oracle timing
-def oracle_sample(wl, layers, budget_s, max_leaves=None):
-    """Time the oracle, as it stands, on a bounded sample: whole leaves of layer 0, as many as
-    fit the budget.  Returns (leaf-queries/s for a full step over `layers` layers, threads, text)."""
+# The oracle is timed as it stands.  Its unit of work is one leaf (all query heads of one layer): the leaf's
+# whole path is materialised and softmax attention is evaluated per head in fp64.  Leaves are independent, so
+# the all-cores figure runs them on a pool of worker processes, one BLAS thread each, and `cores` is the number
+# of workers that really ran; the one-core figure runs the same leaves in one process with one BLAS thread.
+_ORACLE = {}
+
+
+def _oracle_worker_init(path):
+    """Worker start-up: one BLAS thread, K/V of the sampled paths mapped from the file the parent wrote."""
+    try:
+        from threadpoolctl import threadpool_limits
+        _ORACLE["limit"] = threadpool_limits(limits=1)
+    except Exception:
+        pass
+    meta = np.load(os.path.join(path, "meta.npz"))
+    k_all = np.load(os.path.join(path, "k.npy"), mmap_mode="r")
+    v_all = np.load(os.path.join(path, "v.npy"), mmap_mode="r")
+    off = meta["off"]
+    n_nodes = int(meta["parent"].shape[0])
+    _ORACLE.update(parent=meta["parent"], tokens=meta["tokens"], leaf_node=meta["leaf_node"], q=meta["q"],
+                   hq=int(meta["heads"][0]), hkv=int(meta["heads"][1]),
+                   k=[k_all[off[n]:off[n + 1]] for n in range(n_nodes)],
+                   v=[v_all[off[n]:off[n + 1]] for n in range(n_nodes)])
+
+
+def _oracle_worker_leaf(leaf):
+    """One leaf of one layer through the oracle; returns the seconds it took (-1.0: start-up probe)."""
+    if leaf < 0:
+        return -1.0
     from oracle.tree_attention import tree_decode_attention
+    o = _ORACLE
+    t0 = time.perf_counter()
+    tree_decode_attention(o["parent"], o["tokens"], o["leaf_node"], o["k"], o["v"], o["q"], o["hq"], o["hkv"],
+                          leaves=[int(leaf)])
+    return time.perf_counter() - t0
+
+
+def _oracle_sample_files(wl, leaves, path):
+    """K/V of every node on the sampled leaves' paths (layer 0), written where the workers can map them."""
     from workloads import node_kv_bits, query_bits
     tree, g = wl.tree, wl.geometry
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([int(p.get("num_threads", 1)) for p in threadpool_info()] or [1])
-    except Exception:
-        threads = 1
-    qb = query_bits(wl.value_seed, 0, tree.n_leaves, g.num_q_heads, g.head_dim)
-    empty = np.zeros((0, g.num_kv_heads, g.head_dim), np.uint16)
-    k_nodes = [empty] * tree.n_nodes
-    v_nodes = [empty] * tree.n_nodes
-    order = np.random.default_rng(0).permutation(tree.n_leaves)
-    if max_leaves:
-        order = order[:max_leaves]
-    done, spent = 0, 0.0
-    for l in order:
+    need = set()
+    for l in leaves:
         v = int(tree.leaf_node[l])
-        while v >= 0:  # inputs are generated outside the timed part
-            if k_nodes[v] is empty and tree.tokens[v] > 0:
-                k_nodes[v], v_nodes[v] = node_kv_bits(wl.value_seed, v, int(tree.tokens[v]), g.num_kv_heads,
-                                                      g.head_dim, 0)
+        while v >= 0 and v not in need:
+            need.add(v)
             v = int(tree.parent[v])
-        t0 = time.perf_counter()
-        tree_decode_attention(tree.parent, tree.tokens, tree.leaf_node, k_nodes, v_nodes, qb,
-                              g.num_q_heads, g.num_kv_heads, leaves=[int(l)])
-        spent += time.perf_counter() - t0
-        done += 1
-        if spent >= budget_s:
-            break
-    per_leaf_layer = spent / done
-    value = 1.0 / (per_leaf_layer * layers)
-    text = (f"{done} of {tree.n_leaves} leaves of {wl.name}, layer 0 only ({spent:.1f} s of oracle time); "
-            f"a full step is {layers} layers x {tree.n_leaves} leaves, scaled linearly")
-    return value, threads, text, spent
+    off = np.zeros(tree.n_nodes + 1, np.int64)
+    ks, vs = [], []
+    for n in range(tree.n_nodes):
+        t = int(tree.tokens[n]) if n in need else 0
+        off[n + 1] = off[n] + t
+        if t:
+            k, v = node_kv_bits(wl.value_seed, n, t, g.num_kv_heads, g.head_dim, 0)
+            ks.append(k)
+            vs.append(v)
+    np.save(os.path.join(path, "k.npy"), np.concatenate(ks))
+    np.save(os.path.join(path, "v.npy"), np.concatenate(vs))
+    tokens = np.where(np.isin(np.arange(tree.n_nodes), list(need)), tree.tokens, 0).astype(np.int64)
+    np.savez(os.path.join(path, "meta.npz"), parent=np.asarray(tree.parent), tokens=tokens,
+             leaf_node=np.asarray(tree.leaf_node), off=off,
+             q=query_bits(wl.value_seed, 0, tree.n_leaves, g.num_q_heads, g.head_dim),
+             heads=np.array([g.num_q_heads, g.num_kv_heads]))
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def oracle_sample(wl, layers, budget_s, workers=None):
+    """Time the oracle, as it stands, on a bounded sample of whole leaves of layer 0: first on one core, then on
+    a pool of `workers` processes (default: every core this process may use).  Returns a dict with
+    leaf-queries/s of a full step over `layers` layers for both, the worker count and a description."""
+    import multiprocessing as mp
+    import shutil
+    tree = wl.tree
+    workers = workers or host_cores()
+    order = [int(x) for x in np.random.default_rng(0).permutation(tree.n_leaves)]
+    # enough leaves to keep every worker busy for the budget; the paths' K/V is generated outside the timed part
+    n_sample = min(tree.n_leaves, max(2 * workers, 8))
+    sample = order[:n_sample]
+    tmp = tempfile.mkdtemp(prefix="ets_oracle_")
+    try:
+        _oracle_sample_files(wl, sample, tmp)
+        # ---- one core
+        _oracle_worker_init(tmp)
+        one_budget = max(1.0, 0.3 * budget_s)
+        spent1, done1 = 0.0, 0
+        for l in sample:
+            spent1 += _oracle_worker_leaf(l)
+            done1 += 1
+            if spent1 >= one_budget:
+                break
+        lim = _ORACLE.pop("limit", None)
+        if lim is not None:
+            lim.restore_original_limits()
+        per_leaf_1 = spent1 / done1
+        # ---- all cores: a spawned pool (a fork after CUDA start-up would hang), warmed up before the clock starts
+        ctx = mp.get_context("spawn")
+        with ctx.Pool(workers, initializer=_oracle_worker_init, initargs=(tmp,)) as pool:
+            pool.map(_oracle_worker_leaf, [-1] * (4 * workers))
+            rounds = max(1, int(round(0.7 * budget_s / max(per_leaf_1 * 1.5 * max(1, n_sample // workers), 1e-3))))
+            jobs = (sample * rounds)[:max(n_sample, rounds * n_sample)]
+            t0 = time.perf_counter()
+            pool.map(_oracle_worker_leaf, jobs, chunksize=1)
+            wall = time.perf_counter() - t0
+        per_leaf_all = wall / len(jobs)
+    finally:
+        shutil.rmtree(tmp, ignore_errors=True)
+    return {
+        "value": 1.0 / (per_leaf_all * layers), "value_one_core": 1.0 / (per_leaf_1 * layers), "cores": workers,
+        "sample": (f"{len(jobs)} leaf evaluations ({n_sample} distinct leaves of {tree.n_leaves}) of {wl.name}, layer 0 only, "
+                   f"on {workers} worker processes with one BLAS thread each ({wall:.1f} s wall); one core: {done1} leaves "
+                   f"in {spent1:.1f} s; a full step is {layers} layers x {tree.n_leaves} leaves, scaled linearly"),
+        "seconds": wall + spent1,
+    }
 
 
 def run_reference(args):
@@ -118,14 +200,14 @@ def run_reference(args):
     from workloads import make_workload
     wl = make_workload(args.workload)
     layers = args.layers or wl.geometry.num_layers
-    per_step_budget = max(0.5, min(6.0, 90.0 / max(1, args.steps + args.warmup)))
-    vals, spent_all = [], []
-    threads, text = 1, ""
+    per_step_budget = max(1.0, min(8.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, ones = [], []
+    res = None
     for i in range(args.warmup + args.steps):
-        value, threads, text, spent = oracle_sample(wl, layers, per_step_budget)
+        res = oracle_sample(wl, layers, per_step_budget)
         if i >= args.warmup:
-            vals.append(value)
-            spent_all.append(spent)
+            vals.append(res["value"])
+            ones.append(res["value_one_core"])
     value = len(vals) / sum(1.0 / v for v in vals)
     ms = 1000.0 * wl.tree.n_leaves / value
     line = {
@@ -133,8 +215,9 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_description(wl, layers),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                         "sample": "each step: " + text},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": res["cores"], "kind": "oracle",
+                         "value_one_core": len(ones) / sum(1.0 / v for v in ones),
+                         "sample": "each step: " + res["sample"]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -293,7 +376,7 @@ def run_ours(args):
     K, W = args.steps, args.warmup
     headroom = max(K + W + 2, args.loop_tokens + 4)
     job = DecodeJob(wl, headroom=headroom, device=local, layers=layers, chunk_pages=args.chunk_pages,
-                    kernel=args.kernel, wide=args.wide, host_buffers=not args.no_e2e)
+                    kernel=args.kernel, wide=args.wide, host_buffers=not args.no_e2e, chain=args.chain)
     ctx = job.ctx
     stats = ctx.get_stats()
     L = tree.n_leaves
@@ -420,8 +503,9 @@ def run_ours(args):
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline and world == 1:
-        v, threads, text, _ = oracle_sample(wl, layers, args.cpu_seconds)
-        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": text}
+        res = oracle_sample(wl, layers, args.cpu_seconds)
+        cpu = {"value": res["value"], "unit": UNIT, "cores": res["cores"], "kind": "oracle",
+               "value_one_core": res["value_one_core"], "sample": res["sample"]}
 
     # kernels of the library per layer: append, narrow attention, merge, and the wide attention kernel when
     # the tree has wide query groups

@@ -250,8 +250,9 @@ int32_t ets_tree_attn_prefill(ets_ctx* ctx, int32_t layer, const void* q, const 
  * the attention and merge kernels live in an 8 MiB array built into the library instead of the
  * caller's workspace.  Meant for embedders whose host application owns the memory budget or
  * forbids allocation calls on its hot path (a cudaMalloc may synchronise the device).
- *   - Limit: partial_slots * (Hq/Hkv) * (head_dim + 2) * 4 bytes (see ets_get_stats) must fit in
- *     8 MiB; larger trees are refused with ETS_ERR_POOL_EXHAUSTED and a message.
+ *   - Limit: with rows = partial_slots * (Hq/Hkv) (see ets_get_stats), rows * 8 bytes rounded up to a
+ *     multiple of 256, plus rows * head_dim * 4 bytes, must fit in 8 MiB; larger trees are refused
+ *     with ETS_ERR_POOL_EXHAUSTED and a message.  ETS_OPT_TIMING is ignored by this call.
  *   - The first call on each device looks up the array's device address; make it before starting
  *     any stream capture.  The call itself makes no allocation of any kind.
  *   - One array per GPU, shared by every call and context: calls that overlap in time on the
@@ -348,6 +349,19 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
                                  /* the calls are ordered after cuda_stream's work only as of the first */
                                  /* *_host call following a join                                        */
 #define ETS_OPT_TIMING        3  /* 1: bracket the attention and merge kernels with events      */
+#define ETS_OPT_LAUNCH_CHAIN 10  /* 1 (default): the kernels of a call go to cuda_stream as a chain of programmatic  */
+                                 /* dependent launches: each may become resident and run its set-up (barriers,      */
+                                 /* table reads) under the tail of the one before, and waits for it before it       */
+                                 /* touches anything that kernel writes; the tcgen05 kernel runs beside the          */
+                                 /* streaming kernel on the same stream.  Every kernel waits for its predecessor     */
+                                 /* before it ends, so work queued behind a call is ordered behind all of it.        */
+                                 /* 0: ordinary launches, the tcgen05 kernel on a library stream forked from and     */
+                                 /* joined into cuda_stream.                                                         */
+#define ETS_OPT_TEST_FIRST_WAIT_POLLS 11 /* for tests of the time-out path: number of polls after which the FIRST   */
+                                 /* wait for data of every worker of the attention kernels gives up (0: at once);   */
+                                 /* the worker then raises ETS_ERR_DEVICE_TIMEOUT (ets_poll_status), starts nothing  */
+                                 /* new, waits with the ordinary bound for the copies it had started, and returns;   */
+                                 /* that call's outputs are undefined.  Negative: the ordinary bound (default).      */
 int32_t ets_set_option(ets_ctx* ctx, int32_t key, int64_t value);
 
 /*
@@ -367,6 +381,22 @@ int32_t ets_timing_read(ets_ctx* ctx, double* attn_ms, double* merge_ms, int64_t
  * skipped an out-of-range table entry.  Clears the word.
  */
 int32_t ets_poll_status(ets_ctx* ctx, void* cuda_stream);
+
+/*
+ * Measurement probes (the paper has no counterpart; bench.py reports them beside the attention numbers).
+ * ets_probe_stream_read: a persistent kernel with the streaming attention kernel's data path and no
+ * arithmetic reads `bytes` of `buf` (DEVICE, 1024-byte aligned) once: n_ctas CTAs of 8 warps, every warp
+ * keeping `depth` (1..8) linear bulk copies of chunk_bytes (a multiple of 1024) in flight into shared
+ * memory (8 * depth * chunk_bytes must fit in 227 KiB).  Timed by the caller with events on cuda_stream.
+ * ets_probe_empty_launch: a kernel that does nothing, n_ctas CTAs of 256 threads with smem_bytes of
+ * dynamic shared memory: what a launch of that shape costs.
+ *   scratch   DEVICE, 8 KiB, 1024-byte aligned, zeroed by the caller; the int32 at byte 4096 is set to
+ *             ETS_ERR_DEVICE_TIMEOUT if a bounded wait of the probe ran out
+ * Asynchronous.  Errors: ETS_ERR_INVALID_ARG, ETS_ERR_CUDA.
+ */
+int32_t ets_probe_stream_read(const void* buf, size_t bytes, int32_t chunk_bytes, int32_t depth,
+                              int32_t n_ctas, void* scratch, void* cuda_stream);
+int32_t ets_probe_empty_launch(int32_t n_ctas, size_t smem_bytes, void* scratch, void* cuda_stream);
 
 const char* ets_last_error(const ets_ctx* ctx);
 const char* ets_version(void);

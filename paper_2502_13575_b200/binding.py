@@ -32,6 +32,8 @@ ETS_OPT_HOST_PIPELINE = 6
 ETS_OPT_PATH_ITEMS = 7
 ETS_OPT_OVERLAP_APPEND = 8
 ETS_OPT_PACKED_INPUTS = 9
+ETS_OPT_LAUNCH_CHAIN = 10
+ETS_OPT_TEST_FIRST_WAIT_POLLS = 11
 
 _ERR_NAMES = {
     -1: "ETS_ERR_INVALID_ARG", -2: "ETS_ERR_BAD_TREE", -3: "ETS_ERR_POOL_EXHAUSTED",
@@ -123,6 +125,8 @@ _SIGNATURES = {
     "ets_host_join": (C.c_int32, [C.c_void_p, C.c_void_p]),
     "ets_timing_read": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "ets_poll_status": (C.c_int32, [C.c_void_p, C.c_void_p]),
+    "ets_probe_stream_read": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "ets_probe_empty_launch": (C.c_int32, [C.c_int32, C.c_size_t, C.c_void_p, C.c_void_p]),
     "ets_last_error": (C.c_char_p, [C.c_void_p]),
     "ets_version": (C.c_char_p, []),
 }
@@ -212,6 +216,20 @@ def ets_select(parent, leaf_node, reward, cluster=None, *, width: int, temperatu
     return {"weight": weight, "keep": keep, "continuations": cont, "node_kept": nodes, "objective": res.objective,
             "proven_optimal": bool(res.proven_optimal), "nodes_explored": int(res.nodes_explored),
             "n_kept": int(res.n_kept), "n_nodes_kept": int(res.n_nodes_kept)}
+
+
+def ets_probe_stream_read(buf, nbytes: int, chunk_bytes: int, depth: int, n_ctas: int, scratch, stream=None):
+    """Measurement probe (same name as the C call): streams `nbytes` of `buf` once through the bulk-copy ring."""
+    rc = lib.ets_probe_stream_read(_dev_ptr(buf), nbytes, chunk_bytes, depth, n_ctas, _dev_ptr(scratch), _stream_ptr(stream))
+    if rc != ETS_OK:
+        raise EtsError(rc, "ets_probe_stream_read")
+
+
+def ets_probe_empty_launch(n_ctas: int, smem_bytes: int, scratch, stream=None):
+    """Measurement probe (same name as the C call): launches a kernel that does nothing."""
+    rc = lib.ets_probe_empty_launch(n_ctas, smem_bytes, _dev_ptr(scratch), _stream_ptr(stream))
+    if rc != ETS_OK:
+        raise EtsError(rc, "ets_probe_empty_launch")
 
 
 def ets_pool_bytes(cfg: ets_config):

@@ -3,6 +3,7 @@
 #include "../../include/ets.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -174,6 +175,10 @@ struct ets_ctx {
     bool opt_overlap_append = false;
     bool opt_wide_set = false;   // the caller chose the wide threshold: no small-tree exception
     bool opt_packed_inputs = false;
+    // One call's kernels are launched as a chain of programmatic dependents on one stream (see pdl_wait in
+    // ets_device.cuh); 0: ordinary launches, the wide kernel on a second stream forked from the caller's.
+    bool opt_chain = true;
+    uint32_t opt_first_wait_polls = ets::kWaitPolls;
     // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256 tree and on
     // eight width-64 trees: 33, 49 and 65 are within a microsecond of each other per layer, 17 and "never" are
     // 20 % slower (below ~32 rows the per-item latency of the wide kernel costs more than the re-reads by the
@@ -406,6 +411,13 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
         case ETS_OPT_PATH_ITEMS:
             c->opt_path_items = value != 0;
             return ETS_OK;
+        case ETS_OPT_LAUNCH_CHAIN:
+            c->opt_chain = value != 0;
+            return ETS_OK;
+        case ETS_OPT_TEST_FIRST_WAIT_POLLS:
+            if (value > (int64_t)ets::kWaitPolls) return fail(c, ETS_ERR_INVALID_ARG, "poll limit out of range");
+            c->opt_first_wait_polls = value < 0 ? ets::kWaitPolls : (uint32_t)value;
+            return ETS_OK;
         case ETS_OPT_TIMING:
             if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
             c->opt_timing = value != 0;
@@ -552,6 +564,7 @@ static ets::AppendArgs append_args(const ets_ctx* c, int32_t layer, const void* 
     a.pages_per_layer = c->cfg.pages_per_layer;
     a.Hkv = c->cfg.num_kv_heads;
     a.D = c->cfg.head_dim;
+    a.overlap = 0;
     return a;
 }
 
@@ -652,8 +665,9 @@ static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int
         ksrc = c->ws + c->lay.k_stage + hb * c->lay.kv_stride;
         vsrc = c->ws + c->lay.v_stage + hb * c->lay.kv_stride;
     }
-    const ets::AppendArgs a = append_args(c, layer, desc_dev, ksrc, vsrc);
-    ets::launch_kv_append(a, n_items, max_new, c->opt_overlap_append && !host_src, s);
+    ets::AppendArgs a = append_args(c, layer, desc_dev, ksrc, vsrc);
+    a.overlap = (c->opt_chain && c->opt_overlap_append && !host_src) ? 1 : 0;
+    ets::launch_kv_append(a, n_items, max_new, c->opt_chain, s);
     ETS_CUDA(c, cudaGetLastError());
     if (host_src) {
         ETS_CUDA(c, cudaEventRecord(c->ev_kv_free[hb], c->st_comp));
@@ -690,19 +704,30 @@ static int32_t launch_attention(ets_ctx* c, const ets::DecodeArgs& a, cudaStream
     // one CTA per SM; fewer when there are fewer narrow items than resident warps
     const int n_ctas = std::min((c->fp.n_workers + ets::kNarrowWarps - 1) / ets::kNarrowWarps,
                                 (n_narrow + ets::kNarrowWarps - 1) / ets::kNarrowWarps);
-    if (n_wide > 0 && n_narrow > 0) {
-        // the two kernels write disjoint partial slots and are sized to share an SM: the wide one
-        // runs on a second stream, forked from and joined back into the caller's stream
+    const bool chain = c->opt_chain;
+    if (n_wide > 0 && n_narrow > 0 && chain) {
+        // The two kernels write disjoint partial slots and are sized to share an SM.  Both go to the caller's
+        // stream, the wide one as the programmatic dependent of the narrow one: it starts as soon as every
+        // CTA of the narrow kernel (one per SM, all resident at once) has passed its wait for the kernels
+        // ahead, runs beside it, and its last CTA waits for the narrow kernel before it leaves, so whatever
+        // follows in the stream is ordered behind both.
+        ets::DecodeArgs aw = a;
+        aw.wide_behind_narrow = 1;
+        ets::launch_partial_narrow(a, D, n_ctas, true, s);
+        ets::launch_partial_wide(aw, D, n_narrow, n_wide, true, s);
+    } else if (n_wide > 0 && n_narrow > 0) {
+        // ordinary launches: the wide kernel runs on a second stream, forked from and joined back into
+        // the caller's stream
         ETS_CUDA(c, cudaEventRecord(c->ev_fork, s));
         ETS_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
-        ets::launch_partial_narrow(a, D, n_ctas, s);
-        ets::launch_partial_wide(a, D, n_narrow, n_wide, c->side);
+        ets::launch_partial_narrow(a, D, n_ctas, false, s);
+        ets::launch_partial_wide(a, D, n_narrow, n_wide, false, c->side);
         ETS_CUDA(c, cudaEventRecord(c->ev_join, c->side));
         ETS_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));
     } else if (n_wide > 0) {
-        ets::launch_partial_wide(a, D, n_narrow, n_wide, s);
+        ets::launch_partial_wide(a, D, n_narrow, n_wide, chain, s);
     } else if (n_narrow > 0) {
-        ets::launch_partial_narrow(a, D, n_ctas, s);
+        ets::launch_partial_narrow(a, D, n_ctas, chain, s);
     }
     return ETS_OK;
 }
@@ -738,6 +763,8 @@ static ets::DecodeArgs decode_args(const ets_ctx* c, int32_t layer, const void* 
     a.G = c->cfg.num_q_heads / c->cfg.num_kv_heads;
     a.pages_per_layer = c->cfg.pages_per_layer;
     a.scale_log2 = c->scale_log2;
+    a.first_wait_polls = c->opt_first_wait_polls;
+    a.wide_behind_narrow = 0;
     return a;
 }
 
@@ -764,7 +791,7 @@ static int32_t decode_impl(ets_ctx* c, int32_t layer, const void* q, void* out, 
     }
     if (int32_t rc = launch_attention(c, a, s)) return rc;
     if (ev) ETS_CUDA(c, cudaEventRecord(ev[1], s));
-    ets::launch_merge(a, c->cfg.head_dim, s);
+    ets::launch_merge(a, c->cfg.head_dim, c->opt_chain, s);
     if (ev) {
         ETS_CUDA(c, cudaEventRecord(ev[2], s));
         c->timed_calls++;
@@ -823,8 +850,8 @@ int32_t ets_tree_attn_prefill(ets_ctx* c, int32_t layer, const void* q, const in
     const int D = c->cfg.head_dim;
     const int n_narrow = t.n_narrow_items, n_wide = (int)t.items.size() - n_narrow;
     ets::launch_partial_fma(a, D, n_narrow, s);
-    ets::launch_partial_wide(a, D, n_narrow, n_wide, s);
-    ets::launch_merge(a, D, s);
+    ets::launch_partial_wide(a, D, n_narrow, n_wide, false, s);
+    ets::launch_merge(a, D, false, s);
     ETS_CUDA(c, cudaGetLastError());
     return ETS_OK;
 }
@@ -946,7 +973,7 @@ int32_t ets_decode_step_host(ets_ctx* c, int32_t layer, const void* k_new, const
     ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_q_in[hb], 0));
     if (c->out_used[hb]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_out_free[hb], 0));
     const char* desc_dev = c->ws + c->lay.desc + (size_t)kDescSlots * c->lay.desc_slot_bytes;
-    ets::launch_kv_append(append_args(c, layer, desc_dev, kd, vd), t.n_leaves, 1, false, c->st_comp);
+    ets::launch_kv_append(append_args(c, layer, desc_dev, kd, vd), t.n_leaves, 1, c->opt_chain, c->st_comp);
     if (int32_t rc = decode_impl(c, layer, qd, od, lse ? ld : nullptr, c->st_comp)) return rc;
     ETS_CUDA(c, cudaEventRecord(c->ev_q_free[hb], c->st_comp));    // kernels done: the q and k/v staging is reusable, out is ready
     ETS_CUDA(c, cudaEventRecord(c->ev_kv_free[hk], c->st_comp));
@@ -988,7 +1015,9 @@ namespace {
 constexpr size_t kStaticScratchBytes = (size_t)8 << 20;
 constexpr int kStaticMaxDevices = 64;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-unsigned char* g_static_scratch_addr[kStaticMaxDevices] = {};
+// device address of the array per device ordinal; contexts on different host threads may race to fill an
+// entry, so it is an atomic (every thread would store the same value)
+std::atomic<unsigned char*> g_static_scratch_addr[kStaticMaxDevices];
 }  // namespace
 
 int32_t ets_tree_attn_decode_static(ets_ctx* c, int32_t layer, const void* q, void* out, float* lse,
@@ -1001,25 +1030,29 @@ int32_t ets_tree_attn_decode_static(ets_ctx* c, int32_t layer, const void* q, vo
     const int G = c->cfg.num_q_heads / c->cfg.num_kv_heads;
     const int D = c->cfg.head_dim;
     const size_t rows = (size_t)t.n_partial_slots * G;
-    const size_t ml_bytes = align_up(rows * sizeof(float2), 256);
+    const size_t ml_bytes = align_up(rows * sizeof(float2), 256);   // the o part starts on a 256-byte boundary
     const size_t need = ml_bytes + rows * D * sizeof(float);
     if (need > kStaticScratchBytes)
         return fail(c, ETS_ERR_POOL_EXHAUSTED,
                     "tree needs " + std::to_string(need) + " bytes of partial results; the built-in scratch holds " +
                         std::to_string(kStaticScratchBytes) + " (use ets_tree_attn_decode with a workspace)");
     ETS_CUDA(c, cudaSetDevice(dev));
-    if (!g_static_scratch_addr[dev]) {
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // like every device entry point: pipelined host-buffer calls still in flight on the library's streams
+    // (they append to the pools and use the same item queue) are joined first
+    if (int32_t jrc = host_join(c, s)) return jrc;
+    unsigned char* scratch = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
         void* p = nullptr;
         ETS_CUDA(c, cudaGetSymbolAddress(&p, g_static_scratch));
-        g_static_scratch_addr[dev] = static_cast<unsigned char*>(p);
+        scratch = static_cast<unsigned char*>(p);
+        g_static_scratch_addr[dev].store(scratch, std::memory_order_release);
     }
     if (t.n_leaves == 0) return ETS_OK;
-    unsigned char* scratch = g_static_scratch_addr[dev];
-    cudaStream_t s = (cudaStream_t)cuda_stream;
     const ets::DecodeArgs a = decode_args(c, layer, q, out, lse, reinterpret_cast<float2*>(scratch),
                                           reinterpret_cast<float*>(scratch + ml_bytes));
     if (int32_t rc = launch_attention(c, a, s)) return rc;
-    ets::launch_merge(a, D, s);
+    ets::launch_merge(a, D, c->opt_chain, s);
     ETS_CUDA(c, cudaGetLastError());
     return ETS_OK;
 }

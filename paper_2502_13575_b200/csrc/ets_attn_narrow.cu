@@ -34,7 +34,7 @@ constexpr int kWarps = kNarrowWarps;
 #define ETS_DEPTH 2
 #endif
 constexpr int kDepth = ETS_DEPTH;   // measured as fast as 3; 2 leaves shared memory for a wide-kernel CTA on the same SM
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = kWaitPolls;
 #ifndef ETS_CLAIM_AHEAD
 #define ETS_CLAIM_AHEAD 6
 #endif
@@ -60,8 +60,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t polls = kSpinLimit) {
+    for (uint32_t i = 0; i < polls; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -322,12 +322,13 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
     const int grp = lane >> 2;
     const int G = a.G;
 
-    if (base & 127u) {   // the swizzled tile rows must start on 128-byte boundaries
-        if (threadIdx.x == 0) atomicExch(a.status, -1);
-    } else if (worker < a.n_narrow) {
+    const bool aligned = (base & 127u) == 0;   // the swizzled tile rows must start on 128-byte boundaries
+    const bool active = aligned && worker < a.n_narrow;
+    if (!aligned && threadIdx.x == 0) atomicExch(a.status, -1);
+    {
         const uint32_t ring = base + (uint32_t)warp * kDepth * 2 * TB;
         const uint32_t bars = base + (uint32_t)kWarps * kDepth * 2 * TB + (uint32_t)warp * kDepth * 8;
-        if (lane == 0) {
+        if (active && lane == 0) {
 #pragma unroll
             for (int s = 0; s < kDepth; ++s) mbar_init(bars + s * 8, 1);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -428,13 +429,26 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
             }
         };
 
-        // the first item of this warp is its own index in the queue
-        nx.idx = worker;
-        nx.it = a.items[worker];
-        nx.stage = 2;
-        fetch_finish();
+        // The first item of this warp is its own index in the queue.  Its descriptor, page slots and leaf
+        // ids come from the tables, which no kernel writes: they are fetched before the wait for the
+        // kernel ahead in the stream (launched as its programmatic dependent, this part runs under that
+        // kernel's tail).  Node lengths, K/V, the queue counter and the partial results are touched
+        // only after the wait; only then may the kernel behind this one (the wide-group kernel) start,
+        // so that its start implies that the appended K/V and lengths are complete.
+        if (active) {
+            nx.idx = worker;
+            nx.it = a.items[worker];
+            nx.stage = 2;
+            fetch_step();
+        } else {
+            nx.idx = INT_MAX;
+        }
+        pdl_wait();
+        pdl_launch_dependents();
+        if (active) fetch_finish();
 
         bool dead = false;
+        bool first_wait = true;
         while (nx.idx != INT_MAX && !dead) {
             // make the fetched item the current one and start fetching its successor
             cur = nx.it;
@@ -477,7 +491,9 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
                     const uint32_t slot = n_consumed % kDepth;
                     const uint32_t parity = (n_consumed / kDepth) & 1u;
                     ++n_consumed;
-                    if (!__all_sync(FULL, mbar_wait_bounded(bars + slot * 8, parity))) {   // same answer in every lane
+                    const uint32_t polls = first_wait ? a.first_wait_polls : kSpinLimit;
+                    first_wait = false;
+                    if (!__all_sync(FULL, mbar_wait_bounded(bars + slot * 8, parity, polls))) {   // same answer in every lane
                         if (lane == 0) atomicExch(a.status, -7);
                         dead = true;
                         return;
@@ -502,7 +518,10 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
         }
         if (dead) {
             // gave up: nothing new is started; wait (boundedly) for the copies already started, so that
-            // none lands after the CTA has gone.  The slot whose wait ran out counts as consumed.
+            // none lands after the CTA has gone.  The slot whose wait ran out counts as consumed.  A claim
+            // on the item queue that is still in flight is waited for too (by using its value), so that it
+            // cannot land after the last warp has rewound the counter.
+            if (nx.stage == 1 && __shfl_sync(FULL, nx.claim, 0) < 0) atomicExch(a.status, -1);
             while (n_consumed < n_issued) {
                 mbar_wait_bounded(bars + (n_consumed % kDepth) * 8, (n_consumed / kDepth) & 1u);
                 ++n_consumed;
@@ -539,10 +558,11 @@ cudaError_t narrow_prepare(int D) {
     return e;
 }
 
-void launch_partial_narrow(const DecodeArgs& a, int D, int n_ctas, cudaStream_t s) {
+void launch_partial_narrow(const DecodeArgs& a, int D, int n_ctas, bool chained, cudaStream_t s) {
     if (a.n_narrow <= 0 || n_ctas <= 0) return;
-    if (D == 128) attn_partial_narrow_kernel<128><<<n_ctas, kWarps * 32, narrow_smem_bytes(128), s>>>(a);
-    else attn_partial_narrow_kernel<64><<<n_ctas, kWarps * 32, narrow_smem_bytes(64), s>>>(a);
+    ChainLaunch l(dim3(n_ctas), dim3(kWarps * 32), narrow_smem_bytes(D), s, chained);
+    if (D == 128) cudaLaunchKernelEx(&l.cfg, attn_partial_narrow_kernel<128>, a);
+    else cudaLaunchKernelEx(&l.cfg, attn_partial_narrow_kernel<64>, a);
 }
 
 }  // namespace ets

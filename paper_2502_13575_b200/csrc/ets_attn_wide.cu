@@ -34,7 +34,7 @@ namespace {
 constexpr int kWideThreads = 192;
 constexpr int kStageUnits = 4;                 // page slots (16 tokens each) per stage
 constexpr int kStages = 2;                     // two 64-token stages: the next one loads while this one is computed; same footprint as one of 128
-constexpr uint32_t kSpin = 1u << 22;
+constexpr uint32_t kSpin = kWaitPolls;
 constexpr uint32_t kTmemCols = 256;
 // P (bf16, 8 columns per 16 tokens) is written over the S columns it was computed from: chunk c of P
 // covers columns that only hold S chunks <= c/2, which the thread has consumed by then.
@@ -188,9 +188,9 @@ struct Shared {
 
 // Called by all 32 lanes of a warp together; the answer is the same in every lane, so that the
 // warp-collective tcgen05 instructions that follow are never reached by only part of a warp.
-__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, Shared* sh) {
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, Shared* sh, uint32_t polls = kSpin) {
     bool ok = false;
-    for (uint32_t i = 0; i < kSpin; ++i) {
+    for (uint32_t i = 0; i < polls; ++i) {
         if (mbar_try_wait(bar, parity)) { ok = true; break; }
         if ((i & 255u) == 255u && sh->abort) break;
     }
@@ -214,8 +214,19 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
     Shared* sh = reinterpret_cast<Shared*>(base_ptr + 128u * D * 2u + kStages * 2u * STAGE_HALF);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Launch order (see pdl_wait in ets_device.cuh).  The merge kernel behind this one may become resident
+    // at once; it waits for this kernel to complete before it reads a partial result.  Launched on its own,
+    // this kernel waits here for the kernel ahead of it (an append, or the previous call's merge) before it
+    // reads lengths, K/V or queries.  Launched behind the narrow kernel of the same call it must not: that
+    // wait would last until the narrow kernel has finished, and the two are meant to share the SMs.  It
+    // needs none then: the narrow kernel lets it start only after its own wait, i.e. when everything
+    // earlier in the stream has completed.  Completion stays transitive because the CTA that finishes
+    // last waits for the narrow kernel before it leaves (at the end of this function).
+    pdl_launch_dependents();
+    if (!a.wide_behind_narrow) pdl_wait();
     if (base & 1023u) {   // the swizzled operand layout needs 1024-byte aligned tiles
         if (threadIdx.x == 0) atomicExch(a.status, -1);
+        pdl_wait();
         return;
     }
     const DevItem it = a.items[first_item + blockIdx.x];
@@ -358,7 +369,7 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
         // S = Q K^T of stage st into S buffer st % 2 (or the end marker); returns the stage's page slots, -1 on abort
         auto issue_qk = [&](uint32_t st) -> int {
             const uint32_t s = st % kStages;
-            if (!wait_or_abort(smem_u32(&sh->full[s]), (st / kStages) & 1u, sh)) return -1;
+            if (!wait_or_abort(smem_u32(&sh->full[s]), (st / kStages) & 1u, sh, st == 0 ? a.first_wait_polls : kSpin)) return -1;
             const int n = sh->info[s].n_units;
             if (n == 0) {   // end of item: wake the softmax warps, which then see the same marker
                 if (lane == 0) mbar_arrive(smem_u32(&sh->s_ready[st & 1u]));
@@ -590,6 +601,14 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+    // behind the narrow kernel: the CTA that finishes last waits for that kernel, so that this grid
+    // completes after it (the others leave at once and free their SM for the CTAs still queued)
+    if (a.wide_behind_narrow && threadIdx.x == 0) {
+        if (atomicAdd(a.queue + 2, 1) == (int)gridDim.x - 1) {
+            a.queue[2] = 0;
+            pdl_wait();
+        }
+    }
 }
 
 size_t wide_smem_bytes_impl(int D) {
@@ -616,10 +635,11 @@ cudaError_t wide_prepare(int D) {
     return e;
 }
 
-void launch_partial_wide(const DecodeArgs& a, int D, int first_item, int n_wide, cudaStream_t s) {
+void launch_partial_wide(const DecodeArgs& a, int D, int first_item, int n_wide, bool chained, cudaStream_t s) {
     if (n_wide <= 0) return;
-    if (D == 128) attn_partial_wide_kernel<128><<<n_wide, kWideThreads, wide_smem_bytes_impl(128), s>>>(a, first_item);
-    else attn_partial_wide_kernel<64><<<n_wide, kWideThreads, wide_smem_bytes_impl(64), s>>>(a, first_item);
+    ChainLaunch l(dim3(n_wide), dim3(kWideThreads), wide_smem_bytes_impl(D), s, chained);
+    if (D == 128) cudaLaunchKernelEx(&l.cfg, attn_partial_wide_kernel<128>, a, first_item);
+    else cudaLaunchKernelEx(&l.cfg, attn_partial_wide_kernel<64>, a, first_item);
 }
 
 }  // namespace ets

@@ -60,13 +60,28 @@ struct DecodeArgs {
     const char* v_pool;
     float2* part_ml;               // [slot][G]  (m in log2 units, l); a slot belongs to one kv head
     float* part_o;                 // [slot][G][D]
-    int32_t* queue;                // [0] narrow items handed out beyond the first per warp, [1] warps that have finished
+    int32_t* queue;                // [0] narrow items handed out beyond the first per warp, [1] warps that have finished,
+                                   // [2] CTAs of the wide kernel that have finished (each rewound by the last to report)
     int32_t* status;
     int32_t n_items, n_narrow, n_leaves, n_units;   // narrow items come first in `items`
     int32_t Hq, Hkv, G;
     int64_t pages_per_layer;
     float scale_log2;              // sm_scale * log2(e)
+    uint32_t first_wait_polls;     // give-up limit of each worker's first wait for data (kWaitPolls unless a test lowers it)
+    int32_t wide_behind_narrow;    // wide kernel: launched as the narrow kernel's programmatic dependent (see launch_attention)
 };
+
+constexpr uint32_t kWaitPolls = 1u << 22;   // polls after which a device-side wait gives up
+
+// Programmatic dependent launch (PTX griddepcontrol).  A kernel launched with the programmatic-serialization
+// attribute may start while the kernel before it in the stream is still running, once every CTA of that
+// kernel has executed pdl_launch_dependents() or exited.  pdl_wait() returns when that kernel has completed
+// and its writes are visible; it returns at once in a kernel that was launched the ordinary way.  Rule kept by
+// every kernel here that can be launched this way: nothing an earlier kernel writes is read, and nothing an
+// earlier kernel reads is written, before pdl_wait(); and every such kernel executes pdl_wait() before it
+// ends, so that "this kernel has completed" always implies "everything before it in the stream has".
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 struct AppendArgs {
     const int4* desc;              // per item: node, start, n_new, src token offset
@@ -81,18 +96,35 @@ struct AppendArgs {
     int32_t n_nodes, n_pages_total;
     int64_t pages_per_layer;
     int32_t Hkv, D;
+    int32_t overlap;               // 1: copy first, wait for the preceding kernel at the end (see launch_kv_append)
 };
 
-void launch_kv_append(const AppendArgs& a, int n_items, int max_new, bool may_start_early, cudaStream_t s);
+void launch_kv_append(const AppendArgs& a, int n_items, int max_new, bool chained, cudaStream_t s);
 void launch_kv_read(const char* k_pool, const char* v_pool, const int32_t* page_ids_of_node, int n_tokens,
                     int64_t pages_per_layer, int Hkv, int D, __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t s);
 void launch_partial_fma(const DecodeArgs& a, int D, int n_items, cudaStream_t s);
-void launch_merge(const DecodeArgs& a, int D, cudaStream_t s);
+void launch_merge(const DecodeArgs& a, int D, bool chained, cudaStream_t s);
 size_t narrow_smem_bytes(int D);
 cudaError_t narrow_prepare(int D);
-void launch_partial_narrow(const DecodeArgs& a, int D, int n_ctas, cudaStream_t s);
+void launch_partial_narrow(const DecodeArgs& a, int D, int n_ctas, bool chained, cudaStream_t s);
 size_t wide_smem_bytes(int D);
 cudaError_t wide_prepare(int D);
-void launch_partial_wide(const DecodeArgs& a, int D, int first_item, int n_wide, cudaStream_t s);
+void launch_partial_wide(const DecodeArgs& a, int D, int first_item, int n_wide, bool chained, cudaStream_t s);
+
+// launch configuration with or without the programmatic-serialization attribute
+struct ChainLaunch {
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    ChainLaunch(dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool chained) {
+        cfg.gridDim = grid;
+        cfg.blockDim = block;
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = chained ? 1 : 0;
+    }
+};
 
 }  // namespace ets

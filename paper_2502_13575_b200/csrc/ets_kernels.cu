@@ -11,7 +11,7 @@ namespace ets {
 // ------------------------------------------------------------------------------------
 constexpr int kAppendTokPerBlock = 8;
 
-__global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
+__device__ __forceinline__ void kv_append_block(const AppendArgs& a) {
     const int4 d = a.desc[blockIdx.y];
     const int node = d.x, n_new = d.z, src_off = d.w;
     const int t0 = blockIdx.x * kAppendTokPerBlock;
@@ -55,26 +55,26 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
     if (blockIdx.x == 0 && threadIdx.x == 0) a.node_len[node] = start + n_new;
 }
 
-void launch_kv_append(const AppendArgs& a, int n_items, int max_new, bool may_start_early, cudaStream_t s) {
+// Launched with the programmatic-serialization attribute when the caller chains its launches (see
+// pdl_wait in ets_device.cuh).  The kernel behind it (an attention kernel) may begin at once: it reads
+// nothing this kernel writes before its own pdl_wait.  Ordinarily this kernel waits for the one before
+// it and then copies.  With `overlap` it copies first and waits at the end: an append touches one
+// layer's pages and lengths, which the kernel that signalled (the merge kernel of the previous decode
+// call, whose attention kernels have completed by then) does not read, and k_new / v_new are complete
+// by the caller's promise; the wait at the end keeps completion transitive, so that the attention
+// kernel behind this append cannot overwrite partial results the merge kernel is still reading.
+__global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
+    pdl_launch_dependents();
+    if (!a.overlap) pdl_wait();
+    kv_append_block(a);
+    if (a.overlap) pdl_wait();
+}
+
+void launch_kv_append(const AppendArgs& a, int n_items, int max_new, bool chained, cudaStream_t s) {
     if (n_items <= 0 || max_new <= 0) return;
     dim3 grid((max_new + kAppendTokPerBlock - 1) / kAppendTokPerBlock, n_items);
-    // Programmatic dependent launch (only when the caller allows it): if the kernel before this one in the
-    // stream signals early (the merge kernel of the previous decode call does), the append starts while that
-    // kernel is still running.  It never waits for it: an append touches one layer's pages and lengths, which
-    // no merge kernel reads, and the attention kernels that do read them are launched normally, after the
-    // append has finished.  The caller must not allow it when the kernel that produces k_new / v_new is the
-    // one before this in the stream and signals early itself.
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = may_start_early ? 1 : 0;
-    cudaLaunchKernelEx(&cfg, kv_append_kernel, a);
+    ChainLaunch l(grid, dim3(256), 0, s, chained);
+    cudaLaunchKernelEx(&l.cfg, kv_append_kernel, a);
 }
 
 // ------------------------------------------------------------------------------------
@@ -241,20 +241,27 @@ constexpr int kMergeWarps = ETS_MERGE_WARPS;
 
 template <int D>
 __global__ void __launch_bounds__(kMergeWarps * 32) lse_merge_kernel(DecodeArgs a) {
-    // lets a dependent launch that asked for it (the next KV append) start now; see launch_kv_append
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * kMergeWarps + warp;
-    if (row >= (int64_t)a.n_leaves * a.Hq) return;
-    merge_row<D>(a, (int)(row / a.Hq), (int)(row % a.Hq), lane);
+    const bool active = row < (int64_t)a.n_leaves * a.Hq;
+    // Before the wait: the slot list of this row (tables; no kernel writes them).  Launched as a programmatic
+    // dependent, the CTA may be resident while the attention kernels still run; it reads partial results
+    // only after the wait, and only then lets the kernel behind it (the next append) start, so that
+    // kernel runs when the attention kernels have completed.
+    MergeList ml{};
+    if (active) ml = merge_list(a, (int)(row / a.Hq), (int)(row % a.Hq), lane);
+    pdl_wait();
+    pdl_launch_dependents();
+    if (active) merge_row<D>(a, (int)(row / a.Hq), (int)(row % a.Hq), lane, ml);
 }
 
-void launch_merge(const DecodeArgs& a, int D, cudaStream_t s) {
+void launch_merge(const DecodeArgs& a, int D, bool chained, cudaStream_t s) {
     const int64_t rows = (int64_t)a.n_leaves * a.Hq;
     if (rows <= 0) return;
     const int blocks = (int)((rows + kMergeWarps - 1) / kMergeWarps);
-    if (D == 128) lse_merge_kernel<128><<<blocks, kMergeWarps * 32, 0, s>>>(a);
-    else lse_merge_kernel<64><<<blocks, kMergeWarps * 32, 0, s>>>(a);
+    ChainLaunch l(dim3(blocks), dim3(kMergeWarps * 32), 0, s, chained);
+    if (D == 128) cudaLaunchKernelEx(&l.cfg, lse_merge_kernel<128>, a);
+    else cudaLaunchKernelEx(&l.cfg, lse_merge_kernel<64>, a);
 }
 
 }  // namespace ets

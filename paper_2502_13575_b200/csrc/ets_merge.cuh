@@ -12,12 +12,25 @@ namespace ets {
 
 // One (leaf, query head) per warp.  Lanes fetch the slot ids and then the (m, l) pairs in parallel;
 // after that the addresses of all o rows are known and their loads do not depend on each other.
+// The partial slots of one (leaf, query head): bounds of its list and this lane's entry of the first 32.
+// Read from the tables only, so a caller may fetch it before the partial results exist.
+struct MergeList {
+    int s0, s1, first_slot;
+};
+__device__ __forceinline__ MergeList merge_list(const DecodeArgs& a, int leaf, int head, int lane) {
+    MergeList m;
+    const int list = leaf * a.Hkv + head / a.G;
+    m.s0 = a.leaf_slot_off[list];
+    m.s1 = a.leaf_slot_off[list + 1];
+    m.first_slot = m.s0 + lane < m.s1 ? a.leaf_slots[m.s0 + lane] : -1;
+    return m;
+}
+
 template <int D>
-__device__ __forceinline__ void merge_row(const DecodeArgs& a, int leaf, int head, int lane) {
+__device__ __forceinline__ void merge_row(const DecodeArgs& a, int leaf, int head, int lane, const MergeList& list) {
     constexpr int EPL = D / 32;  // features per lane
     const int G = a.G, sub = head % G;
-    const int list = leaf * a.Hkv + head / G;
-    const int s0 = a.leaf_slot_off[list], s1 = a.leaf_slot_off[list + 1];
+    const int s0 = list.s0, s1 = list.s1;
     float ms = -INFINITY, ls = 0.f;
     float acc[EPL];
 #pragma unroll
@@ -25,7 +38,7 @@ __device__ __forceinline__ void merge_row(const DecodeArgs& a, int leaf, int hea
     constexpr int kEarly = 8;   // o rows whose loads are started together with the (m, l) loads
     for (int base = s0; base < s1; base += 32) {
         const int cnt = min(32, s1 - base);
-        const int my_slot = lane < cnt ? a.leaf_slots[base + lane] : -1;
+        const int my_slot = base == s0 ? list.first_slot : (lane < cnt ? a.leaf_slots[base + lane] : -1);
         float2 ml = make_float2(-INFINITY, 0.f);
         if (my_slot >= 0) ml = a.part_ml[(size_t)my_slot * G + sub];
         // the addresses of the o rows depend on the slot ids only: start the first loads now, so that

@@ -54,7 +54,7 @@ class DecodeJob:
 
     def __init__(self, wl: Workload, *, headroom: int, device: int = 0, layers: Optional[int] = None,
                  chunk_pages: Optional[int] = None, kernel: Optional[int] = None, wide: Optional[int] = None,
-                 host_buffers: bool = True):
+                 host_buffers: bool = True, chain: Optional[int] = None, overlap_append: int = 1):
         import torch
         from paper_2502_13575_b200.runner import context_for_tree
         import paper_2502_13575_b200 as ets
@@ -74,8 +74,10 @@ class DecodeJob:
             self.ctx.set_option(ets.ETS_OPT_KERNEL, kernel)
         if wide is not None:
             self.ctx.set_option(ets.ETS_OPT_WIDE, wide)
+        if chain is not None:
+            self.ctx.set_option(ets.ETS_OPT_LAUNCH_CHAIN, chain)
         # the step inputs below are resident before any call: appends may run under the preceding merge kernel
-        self.ctx.set_option(ets.ETS_OPT_OVERLAP_APPEND, 1)
+        self.ctx.set_option(ets.ETS_OPT_OVERLAP_APPEND, overlap_append)
         self.ctx.set_option(ets.ETS_OPT_PACKED_INPUTS, 1)   # decode_tokens() packs k | v | q of a layer in one pinned buffer
         self.keep = np.arange(tree.n_nodes, dtype=np.int32)
         self.ctx.tree_build(tree.parent, self.cap, tree.leaf_node)
