@@ -49,6 +49,9 @@ def parse_args():
                          "instead of the decode step; prints its own JSON line")
     ap.add_argument("--segment-items", action="store_true",
                     help="with --prefill: the decode work decomposition (items per segment) instead of path items")
+    ap.add_argument("--repeats", type=int, default=5, help="times the K-step timed loop is repeated (median reported)")
+    ap.add_argument("--no-table", action="store_true", help="skip the per-workload table and the probes of the default run")
+    ap.add_argument("--table-only", action="store_true", help="only the per-workload table and the probes")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time budget of the oracle sample")
@@ -175,8 +178,9 @@ def oracle_sample(wl, layers, budget_s, workers=None):
         ctx = mp.get_context("spawn")
         with ctx.Pool(workers, initializer=_oracle_worker_init, initargs=(tmp,)) as pool:
             pool.map(_oracle_worker_leaf, [-1] * (4 * workers))
-            rounds = max(1, int(round(0.7 * budget_s / max(per_leaf_1 * 1.5 * max(1, n_sample // workers), 1e-3))))
-            jobs = (sample * rounds)[:max(n_sample, rounds * n_sample)]
+            # about 0.7 of the budget if the workers scaled perfectly; at least every sampled leaf once
+            n_jobs = max(n_sample, int(0.7 * budget_s * workers / max(per_leaf_1, 1e-4)))
+            jobs = [sample[i % n_sample] for i in range(n_jobs)]
             t0 = time.perf_counter()
             pool.map(_oracle_worker_leaf, jobs, chunksize=1)
             wall = time.perf_counter() - t0
@@ -347,6 +351,188 @@ def aggregate_value(leaves_per_rank: int, world: int, ms_per_step: float) -> flo
     return world * leaves_per_rank / (ms_per_step / 1000.0)
 
 
+# ----------------------------------------------------------------------------- probes and the per-workload table
+TABLE_WORKLOADS = ("cfg1", "cfg2", "cfg3_diverse", "cfg3_ets", "cfg5a", "cfg5b", "cfg5c", "forest_w16x8", "forest_w64x8",
+                   "search_w64_rebase", "search_w64_ets", "search_w256_rebase", "search_w256_ets")
+NOMINAL_HBM_GBS = 8000.0
+
+
+def _event_ms(torch, fn, reps):
+    """Median over `reps` of the time of fn() between two events on the current stream."""
+    out = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        out.append(e0.elapsed_time(e1))
+    return statistics.median(out)
+
+
+def run_probes(torch, device):
+    """What the GPU gives a kernel of the streaming attention kernel's shape with no arithmetic (read-only, linear
+    bulk copies into per-warp shared-memory rings), and what a launch costs."""
+    import paper_2502_13575_b200 as ets
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
+    nbytes = 2 << 30                                  # far beyond L2: every launch reads from DRAM
+    buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    buf.zero_()
+    scratch = torch.zeros(8192, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    reads = []
+    for chunk, depth in ((8192, 2), (8192, 3), (16384, 1), (4096, 4), (4096, 6), (2048, 8)):   # 8 warps x depth x chunk <= 227 KiB
+        def launch():
+            ets.ets_probe_stream_read(buf, nbytes, chunk, depth, sms, scratch, stream)
+        for _ in range(3):
+            launch()
+        torch.cuda.synchronize()
+        ms = _event_ms(torch, launch, 9)
+        reads.append({"chunk_bytes": chunk, "copies_in_flight_per_warp": depth, "gbs": nbytes / (ms * 1e-3) / 1e9})
+    if int(scratch[4096:4100].view(torch.int32).item()) != 0:
+        raise RuntimeError("the streaming probe reported a wait that ran out")
+    smem = 131200                                     # the streaming attention kernel's request at head_dim 128
+
+    def one():
+        ets.ets_probe_empty_launch(sms, smem, scratch, stream)
+    for _ in range(20):
+        one()
+    torch.cuda.synchronize()
+    single_us = _event_ms(torch, one, 51) * 1e3       # event, launch, event on an idle stream
+    n = 200
+    back_us = _event_ms(torch, lambda: [one() for _ in range(n)], 5) * 1e3 / n
+    empty_us = _event_ms(torch, lambda: None, 51) * 1e3
+    del buf
+    return {
+        "stream_read": reads,
+        "stream_read_best_gbs": max(r["gbs"] for r in reads),
+        "stream_read_attention_shape_gbs": reads[0]["gbs"],
+        "what": f"{nbytes >> 20} MiB read once per launch by {sms} CTAs x 8 warps through linear bulk copies, no arithmetic",
+        "launch": {"event_launch_event_us": single_us, "two_events_us": empty_us, "back_to_back_us_per_launch": back_us,
+                   "what": f"empty kernel, {sms} CTAs x 256 threads, {smem} B dynamic shared memory"},
+    }
+
+
+def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
+    """One row of the per-workload table: one tree, one layer per launch.  Cold protocol: the context holds R
+    layers with R x (a layer's K/V) >= 4 x L2 and the launches rotate over them back to back, so a layer's K/V
+    has left L2 when its turn comes again and launch latency hides behind the running kernels; for the two
+    smallest trees R is capped and the note says so.  Beside it the time of a single call on an idle stream
+    after L2 was overwritten."""
+    import math
+    import paper_2502_13575_b200 as ets
+    from workloads import make_workload
+    from workloads.loader import DecodeJob
+    wl = make_workload(name)
+    g, tree = wl.geometry, wl.tree
+    L = tree.n_leaves
+    U = int(tree.tokens.sum())
+    l2 = torch.cuda.get_device_properties(device).L2_cache_size
+    qo = 2 * L * g.num_q_heads * g.head_dim * 2
+    layer_bytes = U * g.kv_bytes_per_token + qo
+    R = int(min(32, max(2, math.ceil(4.0 * l2 / layer_bytes))))
+    # iterations per timed loop: enough launches to time, few enough that the tree (one more token per leaf and
+    # iteration) grows by a few percent only over the three loops
+    n_tok, warm = int(max(4, min(math.ceil(192 / R), 0.01 * U / L))), 3
+    job = DecodeJob(wl, headroom=3 * (n_tok + warm) + 8, device=device, layers=R, host_buffers=False, chain=chain)
+    ctx = job.ctx
+    # whole call (append + attention + merge) per layer: one decode iteration over the R layers captured into a
+    # CUDA graph and replayed, so the host's launch rate is not what is measured
+    replay = job.token_graph()
+    replay(warm)
+    torch.cuda.synchronize()
+
+    def loop():
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        replay(n_tok)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+    loops = []
+    for _ in range(3):
+        before = job.steps_done
+        loops.append((loop() * 1e3 / (n_tok * R), U + L * (before + 0.5 * n_tok)))   # (us per call, mean unique tokens)
+    call_us, u_call = min(loops)
+    ctx.poll_status()
+    # the same calls launched one by one with events around the attention kernels and the merge kernel
+    job.reset_lengths()
+    ctx.set_option(ets.ETS_OPT_TIMING, 1)
+    job.decode_tokens(warm)
+    torch.cuda.synchronize()
+    ctx.timing_read()
+    job.decode_tokens(n_tok)
+    torch.cuda.synchronize()
+    attn_ms, merge_ms, n_calls = ctx.timing_read()
+    ctx.set_option(ets.ETS_OPT_TIMING, 0)
+    attn_us, merge_us = attn_ms * 1e3 / n_calls, merge_ms * 1e3 / n_calls
+    # one call on an idle stream, L2 overwritten before it
+    flush = torch.empty(2 * l2, dtype=torch.uint8, device="cuda")
+    job.reset_lengths()
+    p = job._pointers()
+    stream = torch.cuda.current_stream().cuda_stream
+    singles = []
+    for i in range(9):
+        flush.zero_()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.tree_attn_decode(i % R, p["q"][i % R], p["out"][i % R], None, stream=stream)
+        e1.record()
+        torch.cuda.synchronize()
+        singles.append(e0.elapsed_time(e1) * 1e3)
+    ctx.poll_status()
+    t0 = time.perf_counter()
+    for _ in range(5):
+        ctx.tree_build(tree.parent, job.cap, tree.leaf_node, keep_pages_of=job.keep, stream=stream)
+    flatten_ms = (time.perf_counter() - t0) / 5 * 1e3
+    torch.cuda.synchronize()
+    st = ctx.get_stats()
+    u_mean = U + L * (warm + 0.5 * (n_tok + 1))                          # every iteration appends one token per leaf
+    alg = u_mean * g.kv_bytes_per_token + qo
+    gbs = alg / (attn_us * 1e-6) / 1e9
+    call_gbs = (u_call * g.kv_bytes_per_token + qo) / (call_us * 1e-6) / 1e9
+    row = {
+        "workload": name, "leaves": L, "unique_tokens": U, "algorithmic_bytes": alg,
+        "layers_rotated": R, "cold": bool(R * layer_bytes >= 4 * l2),
+        "attention_us": attn_us, "merge_us": merge_us, "gbs": gbs,
+        "frac_measured_copy": gbs / peak, "frac_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+        "frac_read_probe": (gbs / probe_gbs) if probe_gbs else None,
+        "call_us": call_us, "call_gbs": call_gbs, "call_frac_measured_copy": call_gbs / peak,
+        "leaf_queries_per_s": L / (call_us * 1e-6),
+        "single_call_after_flush_us": statistics.median(singles),
+        "flatten_host_ms": flatten_ms, "items": st["n_items"], "narrow_items": st["n_narrow_items"],
+        "launches_timed": int(n_calls),
+    }
+    del job, flush
+    torch.cuda.empty_cache()
+    return row
+
+
+def workload_table(torch, device, peak, probe_gbs, chain=None):
+    rows = [measure_workload(torch, n, device, peak, probe_gbs, chain) for n in TABLE_WORKLOADS]
+    by = {r["workload"]: r for r in rows}
+    # the paper's claim on this kernel (Section 3, Table 2): a tree with 1.8x less KV should take about 1.8x less
+    # time.  cfg3: the pair drawn with a keep fraction; search_*: the pairs grown by REBASE alone and by REBASE + the
+    # library's ets_select, with the KV size of the whole search (sum over its steps) from the generator.
+    from workloads import make_workload
+    pair = {}
+    for big, small, tag in (("cfg3_diverse", "cfg3_ets", "cfg3"), ("search_w64_rebase", "search_w64_ets", "search_w64"),
+                            ("search_w256_rebase", "search_w256_ets", "search_w256")):
+        d, e = by[big], by[small]
+        pair[tag + "_kv_ratio"] = d["unique_tokens"] / e["unique_tokens"]
+        pair[tag + "_time_ratio_attention"] = d["attention_us"] / e["attention_us"]
+        pair[tag + "_time_ratio_call"] = d["call_us"] / e["call_us"]
+        if tag != "cfg3":
+            pair[tag + "_search_kv_size_ratio"] = make_workload(small).notes["kv_ratio_vs_rebase"]
+    note = ("one layer per launch; attention_us / merge_us: events around the attention kernels and the merge kernel in a "
+            "back-to-back loop of ets_decode_step over layers_rotated layers (cold = those layers together exceed 4 x L2; the two "
+            "smallest trees stay L2-resident); gbs and the frac_* columns divide algorithmic_bytes by attention_us; call_us: "
+            "the whole call (append + attention + merge) per layer with the loop over the layers captured in a CUDA graph "
+            "and replayed, no events inside, call_gbs from it")
+    return {"rows": rows, "pair": pair, "note": note}
+
+
 # ----------------------------------------------------------------------------- ours
 def run_ours(args):
     import torch
@@ -426,15 +612,21 @@ def run_ours(args):
         ms = max_over_ranks(ms_local)
         return ms, float(np.mean(u_tokens))
 
-    # ---- device-resident throughput (the headline value) with clocks sampled during the region
+    # ---- device-resident throughput (the headline value) with clocks sampled during the region: the K-step
+    # loop is timed `repeats` times, each one exactly K steps between a barrier + synchronise on both sides;
+    # the reported step time is the median loop
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms_total, u_mean = timed_loop(job.step, sync_each=False)
+    loops = [timed_loop(job.step, sync_each=False) for _ in range(max(1, args.repeats))]
     clocks = sampler.stop() if rank == 0 else {}
     ctx.poll_status()
+    loops.sort(key=lambda x: x[0])
+    ms_total, u_mean = loops[len(loops) // 2]
     ms_step = ms_total / K
     value = aggregate_value(L, world, ms_step)
+    repeats = {"loops": len(loops), "ms_per_step_median": ms_step, "ms_per_step_min": loops[0][0] / K,
+               "ms_per_step_max": loops[-1][0] / K, "ms_per_step_all": [x[0] / K for x in loops]}
 
     # ---- same loop with the attention and merge kernels bracketed by events on their stream
     ctx.set_option(ets.ETS_OPT_TIMING, 1)
@@ -501,6 +693,16 @@ def run_ours(args):
                "ms_per_step": ms_e2e / K}
     ctx.poll_status()
 
+    # ---- the other workloads and the probes (default run only: one GPU, the headline workload)
+    table = probes = None
+    peak, peak_kind = measured_hbm_peak()
+    if rank == 0 and world == 1 and not args.no_table and args.workload == "cfg4":
+        del job
+        torch.cuda.empty_cache()
+        probes = run_probes(torch, local)
+        roofline["frac_of_read_probe"] = achieved / probes["stream_read_best_gbs"]
+        table = workload_table(torch, local, peak, probes["stream_read_best_gbs"], chain=args.chain)
+
     cpu = None
     if rank == 0 and not args.no_cpu_baseline and world == 1:
         res = oracle_sample(wl, layers, args.cpu_seconds)
@@ -522,7 +724,7 @@ def run_ours(args):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": cfg, "clocks": clocks, "e2e": e2e,
             "gpu_launches": K * layers * launches_per_layer, "roofline": roofline, "cpu_baseline": cpu,
-            "decode_loop": loop,
+            "decode_loop": loop, "repeats": repeats, "workloads": table, "probes": probes,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -595,9 +797,23 @@ def run_prefill(args):
     }), flush=True)
 
 
+def run_table_only(args):
+    """Only the per-workload table and the probes, on one GPU."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_hbm_peak()
+    probes = run_probes(torch, 0)
+    table = workload_table(torch, 0, peak, probes["stream_read_best_gbs"], chain=args.chain)
+    print(json.dumps({"workloads": table, "probes": probes, "peak": peak, "peak_kind": peak_kind + " copy bandwidth"}), flush=True)
+
+
 def main():
     args = parse_args()
-    if args.prefill:
+    if args.table_only:
+        run_table_only(args)
+    elif args.prefill:
         run_prefill(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -294,11 +294,15 @@ typedef struct ets_select_params {
     double temperature, lambda_b, lambda_d;
     int32_t width, reserved;
     int64_t node_limit;
+    const int32_t* node_tokens;   /* HOST, nullable: tokens held by each node, for the KV-size figures below */
 } ets_select_params;
 typedef struct ets_select_result {
     double objective;
     int64_t nodes_explored;
     int32_t proven_optimal, n_kept, n_nodes_kept, reserved;
+    /* "KV size" of Section 3 for this step, when params->node_tokens is given (else 0): tokens held by the    */
+    /* nodes of the retained tree V_S, and by all nodes that have a trajectory at or below them                */
+    int64_t kv_tokens_kept, kv_tokens_all;
 } ets_select_result;
 int32_t ets_select(int32_t n_nodes, const int32_t* parent, int32_t n_leaves, const int32_t* leaf_node,
                    const double* reward, const int32_t* cluster, const ets_select_params* params,
@@ -390,7 +394,7 @@ int32_t ets_poll_status(ets_ctx* ctx, void* cuda_stream);
  * memory (8 * depth * chunk_bytes must fit in 227 KiB).  Timed by the caller with events on cuda_stream.
  * ets_probe_empty_launch: a kernel that does nothing, n_ctas CTAs of 256 threads with smem_bytes of
  * dynamic shared memory: what a launch of that shape costs.
- *   scratch   DEVICE, 8 KiB, 1024-byte aligned, zeroed by the caller; the int32 at byte 4096 is set to
+ *   scratch   DEVICE, 8 KiB, 16-byte aligned, zeroed by the caller; the int32 at byte 4096 is set to
  *             ETS_ERR_DEVICE_TIMEOUT if a bounded wait of the probe ran out
  * Asynchronous.  Errors: ETS_ERR_INVALID_ARG, ETS_ERR_CUDA.
  */

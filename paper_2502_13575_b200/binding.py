@@ -88,12 +88,13 @@ class ets_stats(C.Structure):
 
 class ets_select_params(C.Structure):
     _fields_ = [("temperature", C.c_double), ("lambda_b", C.c_double), ("lambda_d", C.c_double),
-                ("width", C.c_int32), ("reserved", C.c_int32), ("node_limit", C.c_int64)]
+                ("width", C.c_int32), ("reserved", C.c_int32), ("node_limit", C.c_int64), ("node_tokens", _I32P)]
 
 
 class ets_select_result(C.Structure):
     _fields_ = [("objective", C.c_double), ("nodes_explored", C.c_int64), ("proven_optimal", C.c_int32),
-                ("n_kept", C.c_int32), ("n_nodes_kept", C.c_int32), ("reserved", C.c_int32)]
+                ("n_kept", C.c_int32), ("n_nodes_kept", C.c_int32), ("reserved", C.c_int32),
+                ("kv_tokens_kept", C.c_int64), ("kv_tokens_all", C.c_int64)]
 
 
 # every symbol include/ets.h declares, with its C signature
@@ -198,13 +199,14 @@ def ets_version() -> str:
 
 
 def ets_select(parent, leaf_node, reward, cluster=None, *, width: int, temperature: float = 0.2,
-               lambda_b: float = 0.0, lambda_d: float = 0.0, node_limit: int = 0) -> Dict[str, object]:
+               lambda_b: float = 0.0, lambda_d: float = 0.0, node_limit: int = 0, node_tokens=None) -> Dict[str, object]:
     """Selection step on the host (same name as the C call): REBASE weights, the kept set, the
     continuations per kept trajectory and the kept nodes of the tree."""
     parent, leaves = _i32(parent), _i32(leaf_node)
     r = np.ascontiguousarray(reward, dtype=np.float64)
     cl = None if cluster is None else _i32(cluster)
-    prm = ets_select_params(temperature, lambda_b, lambda_d, width, 0, node_limit)
+    tok = None if node_tokens is None else _i32(node_tokens)
+    prm = ets_select_params(temperature, lambda_b, lambda_d, width, 0, node_limit, _p(tok))
     res = ets_select_result()
     L, n = leaves.shape[0], parent.shape[0]
     weight, keep, cont, nodes = (np.zeros(L, np.int32), np.zeros(L, np.int32), np.zeros(L, np.int32),
@@ -215,7 +217,8 @@ def ets_select(parent, leaf_node, reward, cluster=None, *, width: int, temperatu
         raise EtsError(rc, "ets_select")
     return {"weight": weight, "keep": keep, "continuations": cont, "node_kept": nodes, "objective": res.objective,
             "proven_optimal": bool(res.proven_optimal), "nodes_explored": int(res.nodes_explored),
-            "n_kept": int(res.n_kept), "n_nodes_kept": int(res.n_nodes_kept)}
+            "n_kept": int(res.n_kept), "n_nodes_kept": int(res.n_nodes_kept),
+            "kv_tokens_kept": int(res.kv_tokens_kept), "kv_tokens_all": int(res.kv_tokens_all)}
 
 
 def ets_probe_stream_read(buf, nbytes: int, chunk_bytes: int, depth: int, n_ctas: int, scratch, stream=None):

@@ -85,7 +85,7 @@ int32_t ets_probe_stream_read(const void* buf, size_t bytes, int32_t chunk_bytes
                               void* scratch, void* cuda_stream) {
     if (!buf || !scratch || chunk_bytes < 1024 || chunk_bytes % 1024 || depth < 1 || depth > 8 || n_ctas < 1)
         return ETS_ERR_INVALID_ARG;
-    if (((uintptr_t)buf | (uintptr_t)scratch) & 1023) return ETS_ERR_INVALID_ARG;
+    if (((uintptr_t)buf & 1023) || ((uintptr_t)scratch & 15)) return ETS_ERR_INVALID_ARG;
     const size_t smem = (size_t)kProbeWarps * depth * chunk_bytes + kProbeWarps * depth * 8;
     if (smem > 227 * 1024) return ETS_ERR_INVALID_ARG;
     if (cudaFuncSetAttribute(stream_read_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -100,8 +100,12 @@ int32_t ets_probe_stream_read(const void* buf, size_t bytes, int32_t chunk_bytes
 
 int32_t ets_probe_empty_launch(int32_t n_ctas, size_t smem_bytes, void* scratch, void* cuda_stream) {
     if (n_ctas < 1 || smem_bytes > 227 * 1024 || !scratch) return ETS_ERR_INVALID_ARG;
-    if (cudaFuncSetAttribute(empty_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
-        return ETS_ERR_CUDA;
+    static size_t allowed = 0;   // raise the kernel's shared-memory limit only when a call needs more than before
+    if (smem_bytes > allowed) {
+        if (cudaFuncSetAttribute(empty_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
+            return ETS_ERR_CUDA;
+        allowed = smem_bytes;
+    }
     empty_kernel<<<n_ctas, kProbeWarps * 32, smem_bytes, (cudaStream_t)cuda_stream>>>(reinterpret_cast<int32_t*>(scratch));
     return cudaGetLastError() == cudaSuccess ? ETS_OK : ETS_ERR_CUDA;
 }

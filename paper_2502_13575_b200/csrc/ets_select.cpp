@@ -266,5 +266,16 @@ extern "C" int32_t ets_select(int32_t n_nodes, const int32_t* parent, int32_t n_
     result->proven_optimal = r.proven_optimal ? 1 : 0;
     result->n_kept = (int32_t)std::count(r.keep.begin(), r.keep.end(), 1);
     result->n_nodes_kept = (int32_t)std::count(r.node_kept.begin(), r.node_kept.end(), 1);
+    result->reserved = 0;
+    result->kv_tokens_kept = result->kv_tokens_all = 0;
+    if (params->node_tokens) {
+        std::vector<char> reached((size_t)n_nodes, 0);   // nodes with any trajectory at or below them
+        for (int32_t i = 0; i < n_leaves; ++i)
+            for (int32_t v = leaf_node[i]; v >= 0 && !reached[v]; v = parent[v]) reached[v] = 1;
+        for (int32_t v = 0; v < n_nodes; ++v) {
+            if (reached[v]) result->kv_tokens_all += params->node_tokens[v];
+            if (r.node_kept[v]) result->kv_tokens_kept += params->node_tokens[v];
+        }
+    }
     return ETS_OK;
 }

@@ -49,10 +49,11 @@ def test_cfg4_every_leaf_on_three_layers():
     assert np.array_equal(a, b)
 
 
-@pytest.mark.parametrize("name", ["cfg3_diverse", "cfg3_ets", "cfg5a", "cfg5b", "cfg5c", "forest_w64x8"])
+@pytest.mark.parametrize("name", ["cfg3_diverse", "cfg3_ets", "cfg5a", "cfg5b", "cfg5c", "forest_w64x8",
+                                  "search_w64_rebase", "search_w64_ets"])
 def test_other_configs_through_the_step_path(name):
     wl = make_workload(name)
-    job = DecodeJob(wl, headroom=3, device=0, host_buffers=False)
+    job = DecodeJob(wl, headroom=3, device=0, layers=1, host_buffers=False)
     job.step()
     torch.cuda.synchronize()
     job.ctx.poll_status()

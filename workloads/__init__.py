@@ -15,6 +15,7 @@ from .trees import (  # noqa: F401
     random_small_tree,
     tree_stats,
 )
+from .search import SEARCH_NAMES, run_search, make_search_workload  # noqa: F401
 from .values import (  # noqa: F401
     f32_to_bf16_bits,
     bf16_bits_to_f32,

@@ -76,7 +76,7 @@ class DecodeJob:
             self.ctx.set_option(ets.ETS_OPT_WIDE, wide)
         if chain is not None:
             self.ctx.set_option(ets.ETS_OPT_LAUNCH_CHAIN, chain)
-        # the step inputs below are resident before any call: appends may run under the preceding merge kernel
+        # the step inputs below are resident before any call: a call may start on them under the preceding merge kernel
         self.ctx.set_option(ets.ETS_OPT_OVERLAP_APPEND, overlap_append)
         self.ctx.set_option(ets.ETS_OPT_PACKED_INPUTS, 1)   # decode_tokens() packs k | v | q of a layer in one pinned buffer
         self.keep = np.arange(tree.n_nodes, dtype=np.int32)
@@ -162,8 +162,7 @@ class DecodeJob:
         stream = self.torch.cuda.current_stream().cuda_stream
         c.tree_build(t.parent, self.cap, t.leaf_node, keep_pages_of=self.keep, stream=stream)
         for layer in range(self.layers):
-            c.kv_append(layer, self.leaf_nodes, self.ones, p["nk"][layer], p["nv"][layer], stream=stream)
-            c.tree_attn_decode(layer, p["q"][layer], p["out"][layer], None, stream=stream)
+            c.decode_step(layer, p["nk"][layer], p["nv"][layer], p["q"][layer], p["out"][layer], None, stream=stream)
         self.steps_done += 1
 
     def decode_tokens(self, n_tokens: int):
@@ -178,6 +177,36 @@ class DecodeJob:
             for layer in range(self.layers):
                 c.decode_step(layer, p["nk"][layer], p["nv"][layer], p["q"][layer], p["out"][layer], None, stream=stream)
         self.steps_done += n_tokens
+
+    def token_graph(self):
+        """One decode iteration over all layers (ets_decode_step per layer) captured into a CUDA graph.  Returns
+        replay(n): n iterations with no host work per launch; the library's host-side lengths are kept in step
+        with ets_note_decode_steps.  Needs two iterations of head room for the capture itself."""
+        import gc
+        torch = self.torch
+        side = torch.cuda.Stream(device=self.dev)
+        with torch.cuda.stream(side):
+            self.decode_tokens(1)      # an ordinary call first: it leaves the append's descriptor list on the device
+        side.synchronize()
+        gc.collect()                   # a context collected during the capture would synchronise the device inside it
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            self.decode_tokens(1)      # counted on the host, runs nothing: the first replay makes up for it
+        state = {"owed": 1}
+
+        def replay(n: int):
+            if self.steps_done + n - state["owed"] > self.headroom:
+                raise RuntimeError("step budget of this job exhausted")
+            for _ in range(n):
+                graph.replay()
+            extra = n - state["owed"]
+            state["owed"] = 0
+            if extra > 0:
+                for layer in range(self.layers):
+                    self.ctx.note_decode_steps(layer, extra)
+                self.steps_done += extra
+        replay.graph = graph           # keeps the graph alive with the callable
+        return replay
 
     def step_host(self):
         """Host buffers in, host buffers out, through ets_decode_step_host (append + attention of one layer per

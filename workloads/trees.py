@@ -262,6 +262,9 @@ def make_workload(name: str) -> Workload:
     """Build one of CONFIG_NAMES.  Deterministic; results are cached per process."""
     if name in _CACHE:
         return _CACHE[name]
+    if name.startswith("search_"):
+        from .search import make_search_workload   # grown by a seeded search whose selection step is the library's
+        return make_search_workload(name)
     notes: Dict[str, float] = {}
     if name == "cfg1":
         cid, variant, tree = 1, 0, _cfg1()
