@@ -482,10 +482,18 @@ def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
         torch.cuda.synchronize()
         singles.append(e0.elapsed_time(e1) * 1e3)
     ctx.poll_status()
+    # host time of a rebuild: a changed tree (the capacities alternate between two values, pages kept, so every call
+    # flattens afresh and uploads), and the tree that is already current (recognised, nothing to do)
+    cap_b = job.cap.copy()
+    cap_b[tree.leaf_node] += 16
     t0 = time.perf_counter()
-    for _ in range(5):
+    for i in range(6):
+        ctx.tree_build(tree.parent, cap_b if i % 2 == 0 else job.cap, tree.leaf_node, keep_pages_of=job.keep, stream=stream)
+    flatten_ms = (time.perf_counter() - t0) / 6 * 1e3
+    t0 = time.perf_counter()
+    for _ in range(6):
         ctx.tree_build(tree.parent, job.cap, tree.leaf_node, keep_pages_of=job.keep, stream=stream)
-    flatten_ms = (time.perf_counter() - t0) / 5 * 1e3
+    flatten_same_ms = (time.perf_counter() - t0) / 6 * 1e3
     torch.cuda.synchronize()
     st = ctx.get_stats()
     u_mean = U + L * (warm + 0.5 * (n_tok + 1))                          # every iteration appends one token per leaf
@@ -501,7 +509,7 @@ def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
         "call_us": call_us, "call_gbs": call_gbs, "call_frac_measured_copy": call_gbs / peak,
         "leaf_queries_per_s": L / (call_us * 1e-6),
         "single_call_after_flush_us": statistics.median(singles),
-        "flatten_host_ms": flatten_ms, "items": st["n_items"], "narrow_items": st["n_narrow_items"],
+        "flatten_host_ms": flatten_ms, "flatten_same_tree_host_ms": flatten_same_ms, "items": st["n_items"], "narrow_items": st["n_narrow_items"],
         "launches_timed": int(n_calls),
     }
     del job, flush

@@ -226,6 +226,19 @@ int32_t ets_decode_step_host(ets_ctx* ctx, int32_t layer, const void* k_new, con
                              const void* q, void* out, float* lse, void* cuda_stream);
 
 /*
+ * The same for n_layers consecutive layers in one call, for callers that hold all layers' inputs of a decode
+ * iteration in host memory (a host-to-device copy of tens of MiB runs at about twice the rate of one of a few MiB):
+ *   inputs  HOST bf16, ONE allocation: n_layers records, record j = [k_new | v_new | q] of layer first_layer + j,
+ *           each part shaped as in ets_decode_step, the parts and the records packed without gaps
+ *   out     HOST bf16 [n_layers, n_leaves, num_q_heads, head_dim];  lse  HOST fp32 [n_layers, n_leaves, num_q_heads], nullable
+ * The inputs of up to four layers travel in one copy, their kernels run back to back, their outputs return in one
+ * copy, and groups of layers alternate between two staging areas.  Follows ETS_OPT_HOST_PIPELINE like the other
+ * *_host calls.  All capacity checks are made before anything is launched.
+ */
+int32_t ets_decode_step_host_layers(ets_ctx* ctx, int32_t first_layer, int32_t n_layers, const void* inputs,
+                                    void* out, float* lse, void* cuda_stream);
+
+/*
  * Attention of the tokens of newly generated steps: what prefilling a step, or scoring it with the
  * reward model, computes (Section 5.1: every new step is scored by a PRM; Section 4.1: the steps of a
  * trajectory share their ancestors' KV).  Every query token is a "leaf" sitting at its step's node

@@ -118,6 +118,7 @@ _SIGNATURES = {
     "ets_note_decode_steps": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),
     "ets_decode_step_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p]),
+    "ets_decode_step_host_layers": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_tree_attn_decode_host": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_tree_attn_decode_static": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ets_kv_read_debug": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -355,6 +356,10 @@ class EtsContext:
     def decode_step_host(self, layer: int, k_new, v_new, q, out, lse=None, stream=None):
         self._check(lib.ets_decode_step_host(self._h, layer, _dev_ptr(k_new), _dev_ptr(v_new), _dev_ptr(q),
                                              _dev_ptr(out), _dev_ptr(lse), _stream_ptr(stream)))
+
+    def decode_step_host_layers(self, first_layer: int, n_layers: int, inputs, out, lse=None, stream=None):
+        self._check(lib.ets_decode_step_host_layers(self._h, first_layer, n_layers, _dev_ptr(inputs), _dev_ptr(out),
+                                                    _dev_ptr(lse), _stream_ptr(stream)))
 
     def tree_attn_decode_host(self, layer: int, q, out, lse=None, stream=None):
         self._check(lib.ets_tree_attn_decode_host(self._h, layer, _dev_ptr(q), _dev_ptr(out), _dev_ptr(lse),

@@ -25,6 +25,7 @@ constexpr int kStages = 3;        // pinned staging buffers for table uploads
 constexpr int kDescSlots = 8;     // pinned/device descriptor slots for appends
 constexpr int kTimingCap = 8192;  // decode calls that can be timed between two reads
 constexpr int kMaxWorkers = 2048; // warp-workers of the attention kernel the tables are sized for
+constexpr int kGroupLayers = 4;   // layers whose host buffers travel in one copy (ets_decode_step_host_layers)
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -35,6 +36,7 @@ struct Layout {  // byte offsets inside the workspace
     size_t q_stage, out_stage, lse_stage, k_stage, v_stage;   // two of each, *_stride bytes apart
     size_t q_stride, lse_stride, kv_stride;
     size_t pk_stage, pk_stride;   // two areas for k_new | v_new | q of one call, contiguous
+    size_t grp_in, grp_in_stride, grp_out, grp_out_stride, grp_lse, grp_lse_stride;   // two areas each for a group of layers
     size_t status;
     size_t total;
     int64_t max_partial_slots, max_items, max_units;
@@ -110,6 +112,12 @@ Layout make_layout(const ets_config* c) {
     L.v_stage = off; off += 2 * L.kv_stride;
     L.pk_stride = align_up(2 * kvb + qbytes, A);
     L.pk_stage = off; off += 2 * L.pk_stride;
+    L.grp_in_stride = align_up((size_t)kGroupLayers * (2 * kvb + qbytes), A);
+    L.grp_in = off; off += 2 * L.grp_in_stride;
+    L.grp_out_stride = align_up((size_t)kGroupLayers * qbytes, A);
+    L.grp_out = off; off += 2 * L.grp_out_stride;
+    L.grp_lse_stride = align_up((size_t)kGroupLayers * c->max_leaves * c->num_q_heads * 4, A);
+    L.grp_lse = off; off += 2 * L.grp_lse_stride;
     L.status = off; off += A;
     L.total = off;
     return L;
@@ -127,6 +135,7 @@ struct ets_ctx {
     ets::FlattenParams fp{};
     Layout lay{};
     ets::Tree tree;
+    ets::FlattenParams built{};   // the options the current tree was built with
     bool has_tree = false;
     bool host_only = true;
     int sm_count = 148;
@@ -161,7 +170,9 @@ struct ets_ctx {
     cudaEvent_t ev_entry = nullptr, ev_q_in[2] = {}, ev_q_free[2] = {}, ev_comp[2] = {}, ev_out_free[2] = {};
     cudaEvent_t ev_kv_in[2] = {}, ev_kv_free[2] = {};
     bool q_used[2] = {false, false}, out_used[2] = {false, false}, kv_used[2] = {false, false};
-    uint64_t n_host_decode = 0, n_host_append = 0;
+    uint64_t n_host_decode = 0, n_host_append = 0, n_host_group = 0;
+    cudaEvent_t ev_g_in[2] = {}, ev_g_free[2] = {}, ev_g_comp[2] = {}, ev_g_out[2] = {};
+    bool g_used[2] = {false, false};
     bool opt_host_pipeline = false;   // host-buffer calls do not make the caller's stream wait; ets_host_join does
     bool host_pending = false;        // host-buffer work that the caller's stream has not been joined with yet
     cudaEvent_t ev_join_comp = nullptr, ev_join_out = nullptr;
@@ -328,7 +339,9 @@ int32_t ets_create(const ets_config* cfg, void* k_pool, void* v_pool, void* work
             {
                 cudaEvent_t* evs[] = {&c->cache_ev, &c->ev_join_comp, &c->ev_join_out, &c->ev_entry, &c->ev_q_in[0], &c->ev_q_in[1], &c->ev_q_free[0], &c->ev_q_free[1],
                                       &c->ev_comp[0], &c->ev_comp[1], &c->ev_out_free[0], &c->ev_out_free[1],
-                                      &c->ev_kv_in[0], &c->ev_kv_in[1], &c->ev_kv_free[0], &c->ev_kv_free[1]};
+                                      &c->ev_kv_in[0], &c->ev_kv_in[1], &c->ev_kv_free[0], &c->ev_kv_free[1],
+                                      &c->ev_g_in[0], &c->ev_g_in[1], &c->ev_g_free[0], &c->ev_g_free[1],
+                                      &c->ev_g_comp[0], &c->ev_g_comp[1], &c->ev_g_out[0], &c->ev_g_out[1]};
                 for (cudaEvent_t* ev : evs)
                     if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
             }
@@ -370,7 +383,8 @@ int32_t ets_destroy(ets_ctx* c) {
         {
             cudaEvent_t evs[] = {c->cache_ev, c->ev_join_comp, c->ev_join_out, c->ev_entry, c->ev_q_in[0], c->ev_q_in[1], c->ev_q_free[0], c->ev_q_free[1], c->ev_comp[0],
                                  c->ev_comp[1], c->ev_out_free[0], c->ev_out_free[1], c->ev_kv_in[0], c->ev_kv_in[1],
-                                 c->ev_kv_free[0], c->ev_kv_free[1]};
+                                 c->ev_kv_free[0], c->ev_kv_free[1], c->ev_g_in[0], c->ev_g_in[1], c->ev_g_free[0],
+                                 c->ev_g_free[1], c->ev_g_comp[0], c->ev_g_comp[1], c->ev_g_out[0], c->ev_g_out[1]};
             for (cudaEvent_t ev : evs)
                 if (ev) cudaEventDestroy(ev);
         }
@@ -437,6 +451,20 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
     fp.wide_min_rows = c->opt_wide;
     if (c->opt_wide_set) fp.wide_min_work = 0;
     fp.path_items = c->opt_path_items;
+    // A rebuild of the very tree that is current (same arrays, every node keeping its own pages, same options)
+    // changes nothing: tables, pages and lengths, on the host and on the device, already are what it would produce.
+    if (c->has_tree && keep_pages_of && n_nodes == c->tree.n_nodes && n_leaves == c->tree.n_leaves && n_nodes >= 0 &&
+        n_leaves >= 0 && (n_nodes == 0 || (parent && cap_tokens)) && (n_leaves == 0 || leaf_node) &&
+        fp.chunk_pages == c->built.chunk_pages && fp.wide_rows == c->built.wide_rows &&
+        fp.wide_min_rows == c->built.wide_min_rows && fp.wide_min_work == c->built.wide_min_work &&
+        fp.path_items == c->built.path_items &&
+        std::memcmp(parent, c->tree.parent.data(), (size_t)n_nodes * 4) == 0 &&
+        std::memcmp(cap_tokens, c->tree.cap.data(), (size_t)n_nodes * 4) == 0 &&
+        std::memcmp(leaf_node, c->tree.leaf_node.data(), (size_t)n_leaves * 4) == 0) {
+        bool identity = true;
+        for (int32_t i = 0; i < n_nodes && identity; ++i) identity = keep_pages_of[i] == i;
+        if (identity) return ETS_OK;
+    }
     ets::Tree next;
     std::string err;
     int32_t rc = ets::tree_build(c->tree, fp, n_nodes, parent, cap_tokens, keep_pages_of, n_leaves, leaf_node,
@@ -461,6 +489,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
     c->tree = std::move(next);
     c->bo = bo;
     c->has_tree = true;
+    c->built = fp;
     return ETS_OK;
 }
 
@@ -570,7 +599,7 @@ static ets::AppendArgs append_args(const ets_ctx* c, int32_t layer, const void* 
 
 static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int32_t* node_id,
                            const int32_t* n_new, const void* k_new, const void* v_new, bool host_src,
-                           cudaStream_t s) {
+                           cudaStream_t s, bool join = true) {
     if (!c) return ETS_ERR_INVALID_ARG;
     if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
     if (!c->has_tree) return fail(c, ETS_ERR_STATE, "no tree built");
@@ -601,7 +630,7 @@ static int32_t append_impl(ets_ctx* c, int32_t layer, int32_t n_items, const int
     ETS_CUDA(c, cudaSetDevice(c->cfg.device));
     const cudaStream_t user = s;
     const int hb = (int)(c->n_host_append & 1u);
-    if (!host_src) {
+    if (!host_src && join) {
         if (int32_t jrc = host_join(c, s)) return jrc;
     }
     if (host_src) {
@@ -987,6 +1016,91 @@ int32_t ets_decode_step_host(ets_ctx* c, int32_t layer, const void* k_new, const
     ++c->n_host_decode;
     ++c->n_host_append;
     for (int32_t l = 0; l < t.n_leaves; ++l) len[t.leaf_node[l]] += 1;
+    return ETS_OK;
+}
+
+// A decode step of several consecutive layers from host buffers.  A host-to-device copy of a few MiB runs at half
+// the rate of one of tens of MiB, so the inputs of kGroupLayers layers travel in one copy, the layers' kernels run
+// back to back on the compute stream, and their outputs come back in one copy; groups alternate between two
+// staging areas, so the copies of one group overlap the kernels of its neighbours.
+int32_t ets_decode_step_host_layers(ets_ctx* c, int32_t first_layer, int32_t n_layers, const void* inputs, void* out,
+                                    float* lse, void* cuda_stream) {
+    if (n_layers <= 0) return c ? fail(c, ETS_ERR_INVALID_ARG, "n_layers must be positive") : ETS_ERR_INVALID_ARG;
+    if (int32_t rc = decode_check(c, first_layer, inputs, out)) return rc;
+    if (int32_t rc = decode_check(c, first_layer + n_layers - 1, inputs, out)) return rc;
+    ets::Tree& t = c->tree;
+    if (t.n_leaves == 0) return ETS_OK;
+    if (t.n_leaves > c->lay.max_append_tokens) return fail(c, ETS_ERR_POOL_EXHAUSTED, "more leaves than max_append_tokens");
+    if ((int32_t)c->step_ones.size() != t.n_leaves) c->step_ones.assign((size_t)t.n_leaves, 1);
+    {   // everything that can fail is checked before the first launch: distinct leaf nodes, room in every layer
+        std::vector<char> seen((size_t)t.n_nodes, 0);
+        for (int32_t l = 0; l < t.n_leaves; ++l) {
+            if (seen[t.leaf_node[l]]) return fail(c, ETS_ERR_INVALID_ARG, "node named twice in one append");
+            seen[t.leaf_node[l]] = 1;
+        }
+        for (int32_t j = 0; j < n_layers; ++j) {
+            const std::vector<int32_t>& len = t.len[first_layer + j];
+            for (int32_t l = 0; l < t.n_leaves; ++l)
+                if (len[t.leaf_node[l]] + 1 > t.cap[t.leaf_node[l]]) return fail(c, ETS_ERR_POOL_EXHAUSTED, "append beyond cap_tokens");
+        }
+    }
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    const size_t rows = (size_t)t.n_leaves * c->cfg.num_q_heads;
+    const size_t qbytes = rows * c->cfg.head_dim * 2;
+    const size_t kvbytes = (size_t)t.n_leaves * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
+    const size_t rec = 2 * kvbytes + qbytes;
+    if (!c->host_epoch_open) {
+        ETS_CUDA(c, cudaEventRecord(c->ev_entry, s));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_entry, 0));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_entry, 0));
+        c->host_epoch_open = c->opt_host_pipeline;
+    }
+    // Group sizes: full groups in the middle, one and two layers at either end, so that the first kernels start
+    // after a short copy and the last copy back is a short one (with many layers the ends are what stays exposed).
+    std::vector<int32_t> sizes;
+    {
+        int32_t rem = n_layers;
+        const bool ramp = n_layers >= 2 * kGroupLayers;
+        if (ramp) { sizes.push_back(1); sizes.push_back(2); rem -= 6; }
+        for (; rem > 0; rem -= kGroupLayers) sizes.push_back(std::min(kGroupLayers, rem));
+        if (ramp) { sizes.push_back(2); sizes.push_back(1); }
+    }
+    int last = 0;
+    int32_t g0 = 0;
+    for (size_t gi = 0; gi < sizes.size(); g0 += sizes[gi], ++gi) {
+        const int32_t ng = sizes[gi];
+        const int b = (int)(c->n_host_group & 1u);
+        char* in_d = c->ws + c->lay.grp_in + (size_t)b * c->lay.grp_in_stride;
+        char* out_d = c->ws + c->lay.grp_out + (size_t)b * c->lay.grp_out_stride;
+        float* lse_d = reinterpret_cast<float*>(c->ws + c->lay.grp_lse + (size_t)b * c->lay.grp_lse_stride);
+        if (c->g_used[b]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_in, c->ev_g_free[b], 0));
+        ETS_CUDA(c, cudaMemcpyAsync(in_d, (const char*)inputs + (size_t)g0 * rec, (size_t)ng * rec, cudaMemcpyHostToDevice, c->st_in));
+        ETS_CUDA(c, cudaEventRecord(c->ev_g_in[b], c->st_in));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_g_in[b], 0));
+        if (c->g_used[b]) ETS_CUDA(c, cudaStreamWaitEvent(c->st_comp, c->ev_g_out[b], 0));
+        for (int32_t j = 0; j < ng; ++j) {
+            const int32_t layer = first_layer + g0 + j;
+            const char* kd = in_d + (size_t)j * rec;
+            if (int32_t rc = append_impl(c, layer, t.n_leaves, t.leaf_node.data(), c->step_ones.data(), kd, kd + kvbytes,
+                                         false, c->st_comp, false))
+                return rc;
+            if (int32_t rc = decode_impl(c, layer, kd + 2 * kvbytes, out_d + (size_t)j * qbytes,
+                                         lse ? lse_d + (size_t)j * rows : nullptr, c->st_comp))
+                return rc;
+        }
+        ETS_CUDA(c, cudaEventRecord(c->ev_g_free[b], c->st_comp));
+        ETS_CUDA(c, cudaEventRecord(c->ev_g_comp[b], c->st_comp));
+        ETS_CUDA(c, cudaStreamWaitEvent(c->st_out, c->ev_g_comp[b], 0));
+        ETS_CUDA(c, cudaMemcpyAsync((char*)out + (size_t)g0 * qbytes, out_d, (size_t)ng * qbytes, cudaMemcpyDeviceToHost, c->st_out));
+        if (lse) ETS_CUDA(c, cudaMemcpyAsync(lse + (size_t)g0 * rows, lse_d, (size_t)ng * rows * 4, cudaMemcpyDeviceToHost, c->st_out));
+        ETS_CUDA(c, cudaEventRecord(c->ev_g_out[b], c->st_out));
+        c->g_used[b] = true;
+        ++c->n_host_group;
+        last = b;
+    }
+    if (c->opt_host_pipeline) c->host_pending = true;
+    else ETS_CUDA(c, cudaStreamWaitEvent(s, c->ev_g_out[last], 0));   // st_out runs in order: the last group's copy is the last to finish
     return ETS_OK;
 }
 

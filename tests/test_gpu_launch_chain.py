@@ -108,3 +108,35 @@ def test_a_wait_that_runs_out_raises_the_status_and_leaves_the_context_usable(wi
         ctx.poll_status()
         ref, _ = tree_decode_attention(tree.parent, tree.tokens, tree.leaf_node, ks, vs, qb, g.num_q_heads, g.num_kv_heads)
         check_close(dev_to_bits(out), ref, "call after a timed-out launch")
+
+
+@pytest.mark.parametrize("pipeline", [0, 1])
+def test_layers_in_one_host_call_equal_one_host_call_per_layer(pipeline):
+    """ets_decode_step_host_layers over eleven layers (groups of four, four and three through both staging areas,
+    twice in a row) gives the bits and the lengths of one ets_decode_step_host per layer and of the device-pointer
+    step, and agrees with the oracle on the last layer."""
+    from workloads.loader import DecodeJob
+    wl = make_workload("cfg2")
+    g, tree = wl.geometry, wl.tree
+    layers = 11
+    jobs = {k: DecodeJob(wl, headroom=4, device=0, layers=layers, host_buffers=(k != "device")) for k in ("group", "single", "device")}
+    for j in jobs.values():
+        j.ctx.set_option(ets.ETS_OPT_HOST_PIPELINE, pipeline if j is not jobs["device"] else 0)
+    for step in range(2):
+        jobs["group"].step_host()
+        jobs["single"].step_host_per_layer()
+        jobs["device"].step()
+        torch.cuda.synchronize()
+        a = jobs["group"].out_h.numpy().view(np.uint16)
+        b = jobs["single"].out_h.numpy().view(np.uint16)
+        c = dev_to_bits(jobs["device"].out)
+        assert np.array_equal(a, b) and np.array_equal(a, c), step
+    for j in jobs.values():
+        j.ctx.poll_status()
+    for l in (0, 5, layers - 1):
+        assert jobs["group"].ctx.get_node_len(l).tolist() == jobs["device"].ctx.get_node_len(l).tolist()
+    leaves = list(range(tree.n_leaves))
+    node_len, ks, vs = jobs["group"].oracle_inputs(layers - 1, leaves)
+    ref, _ = tree_decode_attention(tree.parent, node_len, tree.leaf_node, ks, vs, jobs["group"].q_bits[layers - 1],
+                                   g.num_q_heads, g.num_kv_heads)
+    check_close(jobs["group"].out_h.numpy().view(np.uint16)[layers - 1], ref, "last layer through the grouped host call")

@@ -10,6 +10,7 @@ import pytest
 import paper_2502_13575_b200 as ets
 from oracle.flatten import ReferenceFlattener, BadTree, PoolExhausted
 from workloads import random_small_tree, make_workload, tree_stats, CONFIG_NAMES
+from paper_2502_13575_b200.runner import bounds_for_tree
 from _golden import read_golden
 
 TABLE_KEYS = ("node_page_off", "page_ids", "node_leaf_off", "node_leaves", "leaf_path_off",
@@ -332,3 +333,42 @@ def _path(tree, node):
         out.append(node)
         node = int(tree.parent[node])
     return out
+
+
+def test_rebuilding_the_current_tree_is_recognised_and_changes_nothing():
+    """A rebuild with the same arrays, every node keeping its own pages, is a no-op; any difference (a capacity, a
+    leaf, the keep list, an option) takes the ordinary path.  Either way the exported tables are what a fresh
+    flatten of those arrays gives."""
+    import time
+    wl = make_workload("cfg4")
+    t = wl.tree
+    cap = t.tokens.copy()
+    cap[t.leaf_node] += 20
+    n, l, mpt, mpe, pages = bounds_for_tree(t.parent, cap + 16, t.leaf_node)
+    cfg = ets.make_config(32, 8, 128, num_layers=2, max_nodes=n, max_leaves=l, max_path_tokens=mpt, max_path_entries=mpe,
+                          pages_per_layer=pages + 64, device=-1)
+    ctx = ets.EtsContext(cfg)
+    keep = np.arange(t.n_nodes, dtype=np.int32)
+    ctx.tree_build(t.parent, cap, t.leaf_node)
+    first = ctx.tree_export()
+    work = ctx.work_export()
+    t0 = time.perf_counter()
+    for _ in range(20):
+        ctx.tree_build(t.parent, cap, t.leaf_node, keep_pages_of=keep)
+    same = (time.perf_counter() - t0) / 20
+    again = ctx.tree_export()
+    for k in first:
+        assert np.array_equal(first[k], again[k]), k
+    assert np.array_equal(work["item"], ctx.work_export()["item"])
+    # a changed capacity is a real rebuild (more pages for the leaves' nodes), and going back restores the tables
+    cap2 = cap.copy()
+    cap2[t.leaf_node] += 16
+    t0 = time.perf_counter()
+    ctx.tree_build(t.parent, cap2, t.leaf_node, keep_pages_of=keep)
+    changed = time.perf_counter() - t0
+    assert ctx.tree_export()["page_ids"].shape[0] > first["page_ids"].shape[0]
+    assert same < changed
+    # a different keep list is not the identity: pages are reassigned
+    ctx.tree_build(t.parent, cap, t.leaf_node)
+    ctx.tree_build(t.parent, cap, t.leaf_node, keep_pages_of=np.full(t.n_nodes, -1, np.int32))
+    assert ctx.tree_export()["page_ids"].shape == first["page_ids"].shape

@@ -209,8 +209,20 @@ class DecodeJob:
         return replay
 
     def step_host(self):
-        """Host buffers in, host buffers out, through ets_decode_step_host (append + attention of one layer per
-        call); the caller synchronises to read the result."""
+        """Host buffers in, host buffers out: all layers of the step through one ets_decode_step_host_layers call
+        (the layers' [k_new | v_new | q] records are one pinned buffer); the caller synchronises to read the result."""
+        if self.steps_done >= self.headroom:
+            raise RuntimeError("step budget of this job exhausted; call reset_lengths()")
+        t = self.wl.tree
+        c = self.ctx
+        stream = self.torch.cuda.current_stream().cuda_stream
+        c.tree_build(t.parent, self.cap, t.leaf_node, keep_pages_of=self.keep, stream=stream)
+        c.decode_step_host_layers(0, self.layers, self.packed_h.data_ptr(), self.out_h.data_ptr(), None, stream=stream)
+        c.host_join(stream=stream)   # the step's results are complete once this stream has passed here
+        self.steps_done += 1
+
+    def step_host_per_layer(self):
+        """The same through one ets_decode_step_host call per layer."""
         if self.steps_done >= self.headroom:
             raise RuntimeError("step budget of this job exhausted; call reset_lengths()")
         t = self.wl.tree
@@ -221,7 +233,7 @@ class DecodeJob:
         for layer in range(self.layers):
             c.decode_step_host(layer, p["nk_h"][layer], p["nv_h"][layer], p["q_h"][layer], p["out_h"][layer], None,
                                stream=stream)
-        c.host_join(stream=stream)   # the step's results are complete once this stream has passed here
+        c.host_join(stream=stream)
         self.steps_done += 1
 
     # ---- what the oracle needs for a sample of leaves
