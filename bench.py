@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--repeats", type=int, default=5, help="times the K-step timed loop is repeated (median reported)")
     ap.add_argument("--no-table", action="store_true", help="skip the per-workload table and the probes of the default run")
     ap.add_argument("--table-only", action="store_true", help="only the per-workload table and the probes")
+    ap.add_argument("--table-workloads", default="", help="comma-separated subset of the table's workloads (with --table-only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time budget of the oracle sample")
@@ -485,7 +486,7 @@ def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
     # host time of a rebuild: a changed tree (the capacities alternate between two values, pages kept, so every call
     # flattens afresh and uploads), and the tree that is already current (recognised, nothing to do)
     cap_b = job.cap.copy()
-    cap_b[tree.leaf_node] += 16
+    cap_b[tree.leaf_node] -= 1      # inside the pages the context was sized for; the tokens appended so far still fit
     t0 = time.perf_counter()
     for i in range(6):
         ctx.tree_build(tree.parent, cap_b if i % 2 == 0 else job.cap, tree.leaf_node, keep_pages_of=job.keep, stream=stream)
@@ -517,8 +518,8 @@ def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
     return row
 
 
-def workload_table(torch, device, peak, probe_gbs, chain=None):
-    rows = [measure_workload(torch, n, device, peak, probe_gbs, chain) for n in TABLE_WORKLOADS]
+def workload_table(torch, device, peak, probe_gbs, chain=None, names=TABLE_WORKLOADS):
+    rows = [measure_workload(torch, n, device, peak, probe_gbs, chain) for n in names]
     by = {r["workload"]: r for r in rows}
     # the paper's claim on this kernel (Section 3, Table 2): a tree with 1.8x less KV should take about 1.8x less
     # time.  cfg3: the pair drawn with a keep fraction; search_*: the pairs grown by REBASE alone and by REBASE + the
@@ -527,6 +528,8 @@ def workload_table(torch, device, peak, probe_gbs, chain=None):
     pair = {}
     for big, small, tag in (("cfg3_diverse", "cfg3_ets", "cfg3"), ("search_w64_rebase", "search_w64_ets", "search_w64"),
                             ("search_w256_rebase", "search_w256_ets", "search_w256")):
+        if big not in by or small not in by:
+            continue
         d, e = by[big], by[small]
         pair[tag + "_kv_ratio"] = d["unique_tokens"] / e["unique_tokens"]
         pair[tag + "_time_ratio_attention"] = d["attention_us"] / e["attention_us"]
@@ -707,9 +710,12 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_table and args.workload == "cfg4":
         del job
         torch.cuda.empty_cache()
-        probes = run_probes(torch, local)
-        roofline["frac_of_read_probe"] = achieved / probes["stream_read_best_gbs"]
-        table = workload_table(torch, local, peak, probes["stream_read_best_gbs"], chain=args.chain)
+        try:   # the headline line is printed whatever happens here
+            probes = run_probes(torch, local)
+            roofline["frac_of_read_probe"] = achieved / probes["stream_read_best_gbs"]
+            table = workload_table(torch, local, peak, probes["stream_read_best_gbs"], chain=args.chain)
+        except Exception as exc:   # noqa: BLE001
+            table = {"error": f"{type(exc).__name__}: {exc}"}
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline and world == 1:
@@ -812,8 +818,9 @@ def run_table_only(args):
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(0)
     peak, peak_kind = measured_hbm_peak()
+    names = tuple(n for n in args.table_workloads.split(",") if n) or TABLE_WORKLOADS
     probes = run_probes(torch, 0)
-    table = workload_table(torch, 0, peak, probes["stream_read_best_gbs"], chain=args.chain)
+    table = workload_table(torch, 0, peak, probes["stream_read_best_gbs"], chain=args.chain, names=names)
     print(json.dumps({"workloads": table, "probes": probes, "peak": peak, "peak_kind": peak_kind + " copy bandwidth"}), flush=True)
 
 
