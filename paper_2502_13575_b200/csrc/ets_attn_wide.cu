@@ -244,6 +244,7 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
     auto produce = [&](uint32_t st) -> int {
         const uint32_t s = st % kStages;
         int n = 0;
+        int my_pg = 0, my_vl = 0, my_nd = -1, my_t0 = 0;
         const uint32_t kdst = ring + s * 2 * STAGE_HALF, vdst = kdst + STAGE_HALF;
         while (n < kStageUnits && u < it.unit_count) {
             if (u >= win_base + 32) {
@@ -269,19 +270,27 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
             const int vl = __shfl_sync(0xffffffffu, w_valid, src);
             const int nd = __shfl_sync(0xffffffffu, w_node, src);
             const int t0 = __shfl_sync(0xffffffffu, w_tok0, src);
-            if (lane == 0) {
-                sh->info[s].valid[n] = vl;
-                sh->info[s].node[n] = nd;
-                sh->info[s].tok0[n] = t0;
-                const char* tile = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, pg, h, TB);
-                // raise the byte count first; the producer's single arrival comes after the
-                // last copy of the stage has been started, so the phase cannot end early
-                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"(2 * TB) : "memory");
-                bulk_g2s(kdst + n * TB, tile, TB, smem_u32(&sh->full[s]));
-                bulk_g2s(vdst + n * TB, tile + TB, TB, smem_u32(&sh->full[s]));
-            }
+            if ((lane >> 1) == n) { my_pg = pg; my_vl = vl; my_nd = nd; my_t0 = t0; }   // lanes 2n, 2n+1: the slot's K and V copy
             ++n;
         }
+        // All copies of the stage are started by one instruction, one lane per tile (a bulk copy occupies the
+        // lane that starts it for some hundred cycles; eight of them one after the other from a single lane
+        // were the longest link of the stage's ring of waits).  The byte count is raised first; the producer's
+        // single arrival comes after the copies have been started, so the phase cannot end early.
+        if (lane == 0 && n > 0)
+            asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"((uint32_t)n * 2 * TB) : "memory");
+        __syncwarp();
+        if (lane < 2 * n) {
+            const int slot = lane >> 1, kind = lane & 1;
+            if (kind == 0) {
+                sh->info[s].valid[slot] = my_vl;
+                sh->info[s].node[slot] = my_nd;
+                sh->info[s].tok0[slot] = my_t0;
+            }
+            const char* tile = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, my_pg, h, TB);
+            bulk_g2s((kind ? vdst : kdst) + slot * TB, tile + (kind ? TB : 0u), TB, smem_u32(&sh->full[s]));
+        }
+        __syncwarp();
         if (u > it.unit_count) u = it.unit_count;
         if (lane == 0) {
             sh->info[s].n_units = n;                 // n == 0: end marker
