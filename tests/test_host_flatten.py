@@ -372,3 +372,34 @@ def test_rebuilding_the_current_tree_is_recognised_and_changes_nothing():
     ctx.tree_build(t.parent, cap, t.leaf_node)
     ctx.tree_build(t.parent, cap, t.leaf_node, keep_pages_of=np.full(t.n_nodes, -1, np.int32))
     assert ctx.tree_export()["page_ids"].shape == first["page_ids"].shape
+
+
+def test_new_entry_points_refuse_a_host_only_context_and_bad_arguments():
+    """Every device entry point is refused on a context without a device, before anything is attempted; options
+    outside their range are refused; the probes check their arguments before any launch."""
+    ctx = host_ctx()
+    ctx.tree_build([-1, 0], [4, 4], [1])
+    for call in (lambda: ctx.decode_step_host_layers(0, 1, 1024, 1024),
+                 lambda: ctx.decode_step(0, 1024, 1024, 1024, 1024),
+                 lambda: ctx.tree_attn_decode_static(0, 1024, 1024)):
+        with pytest.raises(ets.EtsError) as e:
+            call()
+        assert e.value.code == ets.ETS_ERR_STATE
+    with pytest.raises(ets.EtsError) as e:
+        ctx.decode_step_host_layers(0, 0, 1024, 1024)
+    assert e.value.code == ets.ETS_ERR_INVALID_ARG
+    ctx.set_option(ets.ETS_OPT_LAUNCH_CHAIN, 0)
+    ctx.set_option(ets.ETS_OPT_LAUNCH_CHAIN, 1)
+    ctx.set_option(ets.ETS_OPT_TEST_FIRST_WAIT_POLLS, 0)
+    ctx.set_option(ets.ETS_OPT_TEST_FIRST_WAIT_POLLS, -1)
+    with pytest.raises(ets.EtsError) as e:
+        ctx.set_option(ets.ETS_OPT_TEST_FIRST_WAIT_POLLS, 1 << 40)
+    assert e.value.code == ets.ETS_ERR_INVALID_ARG
+    for args in ((0, 1 << 20, 8192, 2, 148, 0), (4096, 1 << 20, 1000, 2, 148, 4096), (4096, 1 << 20, 8192, 9, 148, 4096),
+                 (4096, 1 << 20, 16384, 2, 148, 4096), (4096, 1 << 20, 8192, 2, 0, 4096)):
+        with pytest.raises(ets.EtsError) as e:   # null buffer, odd chunk, depth, shared memory, grid
+            ets.ets_probe_stream_read(*args)
+        assert e.value.code == ets.ETS_ERR_INVALID_ARG
+    with pytest.raises(ets.EtsError) as e:
+        ets.ets_probe_empty_launch(0, 0, 4096)
+    assert e.value.code == ets.ETS_ERR_INVALID_ARG
