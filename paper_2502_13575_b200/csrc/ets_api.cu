@@ -176,7 +176,7 @@ struct ets_ctx {
     bool opt_host_pipeline = false;   // host-buffer calls do not make the caller's stream wait; ets_host_join does
     bool host_pending = false;        // host-buffer work that the caller's stream has not been joined with yet
     cudaEvent_t ev_join_comp = nullptr, ev_join_out = nullptr;
-    // second stream on which the wide-group kernel runs beside the narrow kernel
+    // second stream on which the wide-group kernel runs beside the narrow kernel when launches are not chained
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // options

@@ -21,7 +21,7 @@
 // stage s, the copies of stage s + 1 land and its S = Q K^T is already issued; the maximum pass of stage
 // s + 1 overlaps the product O += P V of stage s.  The rest of a stage is serial (softmax -> PV), so a CTA
 // alone does not saturate anything; it is sized (97 KB of shared memory, 256 TMEM columns) to sit on an SM
-// next to a CTA of the narrow kernel, launched on a second stream, and the two overlap.
+// next to a CTA of the narrow kernel, launched behind it as its programmatic dependent, and the two overlap.
 // Every wait is bounded.  A wait that runs out sets an abort flag that all roles poll, the status
 // word is raised, copies in flight are waited for (again boundedly), TMEM is released, and the CTA
 // returns.

@@ -190,9 +190,9 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     const int32_t leaves_per_tile = std::max(1, p.rows_per_item / std::max(1, p.gqa));
     const int32_t n_workers = std::max(1, p.n_workers);
     const int32_t max_run = std::min(32, p.chunk_pages > 0 ? p.chunk_pages : 32);
-    // A very small tree is left to the narrow kernel alone: the second kernel costs a fork and a join of
-    // streams, a few microseconds, which is more than it saves when a warp has only a handful of page
-    // slots to read anyway (measured on a width-16 tree: 16.8 us without, 20.5 us with the second kernel).
+    // A very small tree is left to the narrow kernel alone: a second kernel and the latency of its items cost
+    // more than the re-reads they save when a warp has only a handful of page slots to read anyway (measured on a
+    // width-16 tree with chained launches: 24.7 us per step without, 27.8 us with the second kernel).
     bool wide_pays = p.wide_rows > 0;
     if (wide_pays && !p.path_items) {
         int64_t all_narrow = 0;   // (page slot, kv head, leaf tile) visits if every segment were narrow
