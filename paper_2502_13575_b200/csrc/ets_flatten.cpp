@@ -100,7 +100,8 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         int32_t got = 0;
         if (keep_pages_of && keep_pages_of[i] >= 0) {
             int32_t o = keep_pages_of[i];
-            for (; got < claimed_old[o]; ++got) t.page_ids[w + got] = prev.page_ids[prev.node_page_off[o] + got];
+            got = claimed_old[o];
+            std::copy_n(prev.page_ids.data() + prev.node_page_off[o], got, t.page_ids.data() + w);
         }
         for (; got < need[i]; ++got) {
             if (t.free_heap.empty()) { err = "page pool exhausted at node " + std::to_string(i); return F_EXHAUSTED; }
@@ -170,14 +171,16 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     const int64_t n_units = seg_unit_off[n_seg];
     t.unit.resize((size_t)n_units * 4);
     for (int32_t s = 0; s < n_seg; ++s) {
-        int32_t u = seg_unit_off[s];
-        for (int32_t v = seg_head[s]; v >= 0; v = seg_next[v])
-            for (int32_t j = 0; j < need[v]; ++j, ++u) {
-                t.unit[4 * (size_t)u + 0] = t.page_ids[t.node_page_off[v] + j];
-                t.unit[4 * (size_t)u + 1] = v;
-                t.unit[4 * (size_t)u + 2] = j * p.page_size;
-                t.unit[4 * (size_t)u + 3] = 0;
+        int32_t* u = t.unit.data() + 4 * (size_t)seg_unit_off[s];
+        for (int32_t v = seg_head[s]; v >= 0; v = seg_next[v]) {
+            const int32_t* pg = t.page_ids.data() + t.node_page_off[v];
+            for (int32_t j = 0, nv = need[v]; j < nv; ++j, u += 4) {
+                u[0] = pg[j];
+                u[1] = v;
+                u[2] = j * p.page_size;
+                u[3] = 0;
             }
+        }
     }
 
     // ---- narrow work queue.  A run is the page slots of one segment for one (kv head, leaf tile).
@@ -245,9 +248,13 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         static const int32_t kCaps[] = {32, 24, 16, 12, 8, 6, 4, 3, 2, 1};
         double best = 0.0;
         int32_t prev_c = 0;
+        int32_t longest_seg = 0;
+        for (const SegInfo& q : narrow) longest_seg = std::max(longest_seg, q.nu);
         for (int32_t cand : kCaps) {
             const int32_t c = std::min(cand, max_run);
             if (c == prev_c) continue;
+            // a piece length at or above the longest segment cuts nothing: the same queue as the previous candidate
+            if (prev_c != 0 && c >= longest_seg && prev_c >= longest_seg) continue;
             prev_c = c;
             const int32_t tc = p.tail_pages > 0 ? p.tail_pages : std::max(8, c / 4);
             int64_t need_slots = 0;
@@ -298,27 +305,37 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         }
     }
     int64_t slots = 0;
+    // Every run of items made below covers one query group (gn leaves, listed from leaf_list_begin) for all kv
+    // heads: head h, leaf position i gets partial slot base + h * gn + i.  The runs are remembered and the
+    // per-(leaf, kv head) slot lists are written from them at the end, once per leaf instead of once per item.
+    struct GroupRun { int32_t leaf_list_begin, gn; int64_t base; };
+    std::vector<GroupRun> runs;
     {
         size_t n_items_narrow = 0;
         for (const Part& q : best_parts) n_items_narrow += (size_t)p.num_kv_heads * ceil_div(g[seg_head[q.seg]], leaves_per_tile);
         t.items.reserve(n_items_narrow + 64);
     }
+    runs.reserve(best_parts.size() + 64);
     for (const Part& q : best_parts) {
         const int32_t head_node = seg_head[q.seg];
         const int32_t gn = g[head_node];
+        const int32_t tiles = ceil_div(gn, leaves_per_tile);
+        runs.push_back({t.node_leaf_off[head_node], gn, slots});
+        const size_t first = t.items.size();
+        t.items.resize(first + (size_t)p.num_kv_heads * tiles);
+        Item* it = t.items.data() + first;
+        const int32_t unit_begin = seg_unit_off[q.seg] + q.begin, list = t.node_leaf_off[head_node];
         for (int32_t h = 0; h < p.num_kv_heads; ++h)
-            for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile) {
-                Item it;
-                it.unit_begin = seg_unit_off[q.seg] + q.begin;
-                it.unit_count = q.len;
-                it.kv_head = h;
-                it.leaf_list_begin = t.node_leaf_off[head_node] + l0;
-                it.n_leaves_tile = std::min(leaves_per_tile, gn - l0);
-                it.slot_first = (int32_t)slots;
-                it.segment = q.seg;
-                it.reserved = (l0 + leaves_per_tile < gn) ? 1 : 0;   // bit 0: the next tile re-reads these pages
-                t.items.push_back(it);
-                slots += it.n_leaves_tile;
+            for (int32_t l0 = 0; l0 < gn; l0 += leaves_per_tile, ++it) {
+                it->unit_begin = unit_begin;
+                it->unit_count = q.len;
+                it->kv_head = h;
+                it->leaf_list_begin = list + l0;
+                it->n_leaves_tile = std::min(leaves_per_tile, gn - l0);
+                it->slot_first = (int32_t)slots;
+                it->segment = q.seg;
+                it->reserved = (l0 + leaves_per_tile < gn) ? 1 : 0;   // bit 0: the next tile re-reads these pages
+                slots += it->n_leaves_tile;
             }
     }
     if (slots > p.max_partial_slots) { err = "partial-result slots exceed the workspace bound"; return F_EXHAUSTED; }
@@ -355,6 +372,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             const int32_t n_pieces = ceil_div(nu, piece);
             for (int32_t pc = 0; pc < n_pieces; ++pc) {
                 const int32_t ub = (int32_t)((int64_t)nu * pc / n_pieces), ue = (int32_t)((int64_t)nu * (pc + 1) / n_pieces);
+                runs.push_back({t.node_leaf_off[head_node], gn, slots});
                 for (int32_t h = 0; h < p.num_kv_heads; ++h)
                     for (int32_t l0 = 0; l0 < gn; l0 += wide_leaves) {
                         Item it;
@@ -380,6 +398,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     t.path_items = p.path_items;
     if (p.path_items) {
         t.items.clear();
+        runs.clear();
         slots = 0;
         std::vector<int32_t> at_off((size_t)n_nodes + 1, 0);
         for (int32_t l = 0; l < n_leaves; ++l) ++at_off[leaf_node[l] + 1];
@@ -411,6 +430,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
                 const int32_t uc = (int32_t)(t.unit.size() / 4) - ub;
                 if (uc == 0) continue;
                 const int32_t per_tile = dense ? wide_leaves : leaves_per_tile;
+                runs.push_back({ext + at_off[v], nl, slots});
                 for (int32_t h = 0; h < p.num_kv_heads; ++h)
                     for (int32_t l0 = 0; l0 < nl; l0 += per_tile) {
                         Item it;
@@ -435,19 +455,35 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
     t.n_partial_slots = slots;
     if ((int64_t)t.items.size() > p.max_items) { err = "work items exceed the workspace bound"; return F_EXHAUSTED; }
 
-    // ---- per (leaf, kv head): the partial slots to merge
+    // ---- per (leaf, kv head): the partial slots to merge, in item order.  A leaf meets the same runs for every
+    // kv head, so its count is taken once and the H lists of a leaf lie one behind the other.
     const int32_t H = p.num_kv_heads;
-    t.leaf_slot_off.assign((size_t)n_leaves * H + 1, 0);
-    for (const Item& it : t.items)
-        for (int32_t i = 0; i < it.n_leaves_tile; ++i)
-            ++t.leaf_slot_off[(size_t)t.node_leaves[it.leaf_list_begin + i] * H + it.kv_head + 1];
-    for (size_t k = 0; k < (size_t)n_leaves * H; ++k) t.leaf_slot_off[k + 1] += t.leaf_slot_off[k];
-    t.leaf_slots.assign((size_t)t.leaf_slot_off[(size_t)n_leaves * H], 0);
+    std::vector<int32_t> per_leaf((size_t)n_leaves, 0);
+    for (const GroupRun& r : runs) {
+        const int32_t* lv = t.node_leaves.data() + r.leaf_list_begin;
+        for (int32_t i = 0; i < r.gn; ++i) ++per_leaf[lv[i]];
+    }
+    t.leaf_slot_off.resize((size_t)n_leaves * H + 1);
     {
-        std::vector<int32_t> cur(t.leaf_slot_off.begin(), t.leaf_slot_off.end() - 1);
-        for (const Item& it : t.items)
-            for (int32_t i = 0; i < it.n_leaves_tile; ++i)
-                t.leaf_slots[(size_t)cur[(size_t)t.node_leaves[it.leaf_list_begin + i] * H + it.kv_head]++] = it.slot_first + i;
+        int32_t off = 0;
+        for (int32_t l = 0; l < n_leaves; ++l)
+            for (int32_t h = 0; h < H; ++h) {
+                t.leaf_slot_off[(size_t)l * H + h] = off;
+                off += per_leaf[l];
+            }
+        t.leaf_slot_off[(size_t)n_leaves * H] = off;
+        t.leaf_slots.resize((size_t)off);
+    }
+    {
+        std::vector<int32_t> cur((size_t)n_leaves, 0);
+        for (const GroupRun& r : runs) {
+            const int32_t* lv = t.node_leaves.data() + r.leaf_list_begin;
+            for (int32_t i = 0; i < r.gn; ++i) {
+                const int32_t l = lv[i], k = cur[l]++, n = per_leaf[l];
+                int32_t* dst = t.leaf_slots.data() + t.leaf_slot_off[(size_t)l * H] + k;
+                for (int32_t h = 0; h < H; ++h) dst[(size_t)h * n] = (int32_t)(r.base + (int64_t)h * r.gn + i);
+            }
+        }
     }
     return F_OK;
 }
