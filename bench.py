@@ -353,7 +353,7 @@ def aggregate_value(leaves_per_rank: int, world: int, ms_per_step: float) -> flo
 
 
 # ----------------------------------------------------------------------------- probes and the per-workload table
-TABLE_WORKLOADS = ("cfg1", "cfg2", "cfg3_diverse", "cfg3_ets", "cfg5a", "cfg5b", "cfg5c", "forest_w16x8", "forest_w64x8",
+TABLE_WORKLOADS = ("cfg1", "cfg2", "cfg3_diverse", "cfg3_ets", "cfg4", "cfg5a", "cfg5b", "cfg5c", "forest_w16x8", "forest_w64x8",
                    "search_w64_rebase", "search_w64_ets", "search_w256_rebase", "search_w256_ets")
 NOMINAL_HBM_GBS = 8000.0
 
@@ -414,6 +414,37 @@ def run_probes(torch, device):
     }
 
 
+def timeline_from_stamps(st, max_launches=64):
+    """Mean timeline of a call from the library's device time stamps (ets_stamps_read), in microseconds relative to the
+    start of the streaming attention kernel: when the append ahead of it ended, when its wait for that append returned,
+    when it ended, the tcgen05 kernel's start and end (None without wide groups), the merge's end, and the period
+    (merge end to merge end)."""
+    cnt, s0, e0 = st["count"], st["start_ns"], st["end_ns"]
+    n = int(min(cnt[1], cnt[3], cnt[4]))
+    if n < 3:
+        return None
+    k = min(n - 1, max_launches)
+    rows = []
+    for j in range(n - k, n):
+        def at(kind, arr):   # the launch of `kind` that belongs to the j-th launch counted from the end of the narrow series
+            i = int(cnt[kind]) - (int(cnt[1]) - j)
+            return None if i < 0 or i >= int(cnt[kind]) else int(arr[kind][i])
+        base = at(1, s0)
+        rec = {"append_start": at(0, s0), "append_end": at(0, e0), "narrow_wait_returned": at(4, s0), "narrow_end": at(1, e0),
+               "wide_start": at(2, s0), "wide_end": at(2, e0), "merge_start": at(3, s0), "merge_end": at(3, e0)}
+        rows.append({key: (None if v is None else (v - base) / 1e3) for key, v in rec.items()} | {"_merge_end_abs": at(3, e0)})
+    out = {}
+    for key in rows[0]:
+        if key.startswith("_"):
+            continue
+        vals = [r[key] for r in rows if r[key] is not None]
+        out[key] = float(np.mean(vals)) if len(vals) == len(rows) else None
+    ends = [r["_merge_end_abs"] for r in rows]
+    out["period"] = float(np.mean(np.diff(ends))) / 1e3
+    out["launches"] = len(rows)
+    return out
+
+
 def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
     """One row of the per-workload table: one tree, one layer per launch.  Cold protocol: the context holds R
     layers with R x (a layer's K/V) >= 4 x L2 and the launches rotate over them back to back, so a layer's K/V
@@ -435,7 +466,7 @@ def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
     # iterations per timed loop: enough launches to time, few enough that the tree (one more token per leaf and
     # iteration) grows by a few percent only over the three loops
     n_tok, warm = int(max(4, min(math.ceil(192 / R), 0.01 * U / L))), 3
-    job = DecodeJob(wl, headroom=3 * (n_tok + warm) + 8, device=device, layers=R, host_buffers=False, chain=chain)
+    job = DecodeJob(wl, headroom=4 * (n_tok + warm) + 16, device=device, layers=R, host_buffers=False, chain=chain)
     ctx = job.ctx
     # whole call (append + attention + merge) per layer: one decode iteration over the R layers captured into a
     # CUDA graph and replayed, so the host's launch rate is not what is measured
@@ -456,6 +487,15 @@ def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
         loops.append((loop() * 1e3 / (n_tok * R), U + L * (before + 0.5 * n_tok)))   # (us per call, mean unique tokens)
     call_us, u_call = min(loops)
     ctx.poll_status()
+    # where a call's time goes: the same replayed loop with the kernels recording device time stamps
+    ctx.set_option(ets.ETS_OPT_TIMING, 2)
+    replay_stamped = job.token_graph()
+    replay_stamped(warm)
+    ctx.stamps_read()
+    replay_stamped(n_tok)
+    timeline = timeline_from_stamps(ctx.stamps_read(), max_launches=max(2, n_tok * R - 1))
+    ctx.set_option(ets.ETS_OPT_TIMING, 0)
+    del replay_stamped
     # the same calls launched one by one with events around the attention kernels and the merge kernel
     job.reset_lengths()
     ctx.set_option(ets.ETS_OPT_TIMING, 1)
@@ -509,7 +549,7 @@ def measure_workload(torch, name, device, peak, probe_gbs, chain=None):
         "frac_read_probe": (gbs / probe_gbs) if probe_gbs else None,
         "call_us": call_us, "call_gbs": call_gbs, "call_frac_measured_copy": call_gbs / peak,
         "leaf_queries_per_s": L / (call_us * 1e-6),
-        "single_call_after_flush_us": statistics.median(singles),
+        "single_call_after_flush_us": statistics.median(singles), "timeline_us": timeline,
         "flatten_host_ms": flatten_ms, "flatten_same_tree_host_ms": flatten_same_ms, "items": st["n_items"], "narrow_items": st["n_narrow_items"],
         "launches_timed": int(n_calls),
     }
@@ -540,7 +580,9 @@ def workload_table(torch, device, peak, probe_gbs, chain=None, names=TABLE_WORKL
             "back-to-back loop of ets_decode_step over layers_rotated layers (cold = those layers together exceed 4 x L2; the two "
             "smallest trees stay L2-resident); gbs and the frac_* columns divide algorithmic_bytes by attention_us; call_us: "
             "the whole call (append + attention + merge) per layer with the loop over the layers captured in a CUDA graph "
-            "and replayed, no events inside, call_gbs from it")
+            "and replayed, no events inside, call_gbs from it; timeline_us: mean device time stamps of a call in the replayed "
+            "loop, relative to the start of the streaming attention kernel (ETS_OPT_TIMING = 2); the cfg4 row is one layer "
+            "of the headline workload in a context of layers_rotated layers")
     return {"rows": rows, "pair": pair, "note": note}
 
 

@@ -365,7 +365,9 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
                                  /* results are valid after ets_host_join + synchronising that stream;  */
                                  /* the calls are ordered after cuda_stream's work only as of the first */
                                  /* *_host call following a join                                        */
-#define ETS_OPT_TIMING        3  /* 1: bracket the attention and merge kernels with events      */
+#define ETS_OPT_TIMING        3  /* 1: bracket the attention and merge kernels with events (ets_timing_read);   */
+                                 /* 2: the kernels record device time stamps instead (ets_stamps_read), which  */
+                                 /* leaves the launches chained as they are; 0: neither                        */
 #define ETS_OPT_LAUNCH_CHAIN 10  /* 1 (default): the kernels of a call go to cuda_stream as a chain of programmatic  */
                                  /* dependent launches: each may become resident and run its set-up (barriers,      */
                                  /* table reads) under the tail of the one before, and waits for it before it       */
@@ -391,6 +393,24 @@ int32_t ets_host_join(ets_ctx* ctx, void* cuda_stream);
 
 /* With ETS_OPT_TIMING on: waits for the recorded events, returns and clears the sums. */
 int32_t ets_timing_read(ets_ctx* ctx, double* attn_ms, double* merge_ms, int64_t* n_calls);
+
+/*
+ * With ETS_OPT_TIMING = 2: per kind of kernel (0 append, 1 streaming attention, 2 tcgen05 attention, 3 merge, 4 the
+ * moment the streaming kernel's wait for the kernel ahead of it returned) and launch since the last read, the
+ * earliest start and the latest end over the kernel's CTAs on the GPU's global nanosecond timer.  count[k] launches
+ * of kind k were recorded (at most ETS_STAMP_LAUNCHES; further ones are dropped).  Synchronises the device, copies
+ * the table to `out` (HOST) and clears it.  Launches captured into a CUDA graph record stamps if the option was on
+ * at capture time.  A measurement aid: the paper has no counterpart.
+ */
+#define ETS_STAMP_KINDS 5
+#define ETS_STAMP_LAUNCHES 4096
+typedef struct ets_stamps_host {
+    uint32_t count[8];
+    uint32_t reserved[8];
+    uint64_t start_ns[ETS_STAMP_KINDS][ETS_STAMP_LAUNCHES];
+    uint64_t end_ns[ETS_STAMP_KINDS][ETS_STAMP_LAUNCHES];
+} ets_stamps_host;
+int32_t ets_stamps_read(ets_ctx* ctx, ets_stamps_host* out);
 
 /*
  * Synchronise cuda_stream and report the device-side status word: ETS_OK, or

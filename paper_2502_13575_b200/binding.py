@@ -86,6 +86,14 @@ class ets_stats(C.Structure):
         "attended_tokens", "n_narrow_items")]
 
 
+STAMP_KINDS, STAMP_LAUNCHES = 5, 4096
+
+
+class ets_stamps_host(C.Structure):
+    _fields_ = [("count", C.c_uint32 * 8), ("reserved", C.c_uint32 * 8),
+                ("start_ns", C.c_uint64 * (STAMP_KINDS * STAMP_LAUNCHES)), ("end_ns", C.c_uint64 * (STAMP_KINDS * STAMP_LAUNCHES))]
+
+
 class ets_select_params(C.Structure):
     _fields_ = [("temperature", C.c_double), ("lambda_b", C.c_double), ("lambda_d", C.c_double),
                 ("width", C.c_int32), ("reserved", C.c_int32), ("node_limit", C.c_int64), ("node_tokens", _I32P)]
@@ -126,6 +134,7 @@ _SIGNATURES = {
     "ets_set_option": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int64]),
     "ets_host_join": (C.c_int32, [C.c_void_p, C.c_void_p]),
     "ets_timing_read": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "ets_stamps_read": (C.c_int32, [C.c_void_p, C.POINTER(ets_stamps_host)]),
     "ets_poll_status": (C.c_int32, [C.c_void_p, C.c_void_p]),
     "ets_probe_stream_read": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "ets_probe_empty_launch": (C.c_int32, [C.c_int32, C.c_size_t, C.c_void_p, C.c_void_p]),
@@ -390,6 +399,15 @@ class EtsContext:
         a, m, n = C.c_double(), C.c_double(), C.c_int64()
         self._check(lib.ets_timing_read(self._h, C.byref(a), C.byref(m), C.byref(n)))
         return a.value, m.value, n.value
+
+    def stamps_read(self) -> Dict[str, np.ndarray]:
+        """Device time stamps since the last read: counts [5] and, per kind, start / end in ns ([5, launches])."""
+        st = ets_stamps_host()
+        self._check(lib.ets_stamps_read(self._h, C.byref(st)))
+        count = np.array(list(st.count)[:STAMP_KINDS], dtype=np.int64)
+        start = np.ctypeslib.as_array(st.start_ns).reshape(STAMP_KINDS, STAMP_LAUNCHES).astype(np.int64)
+        end = np.ctypeslib.as_array(st.end_ns).reshape(STAMP_KINDS, STAMP_LAUNCHES).astype(np.int64)
+        return {"count": count, "start_ns": start.copy(), "end_ns": end.copy()}
 
     def poll_status(self, stream=None):
         self._check(lib.ets_poll_status(self._h, _stream_ptr(stream)))

@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <cstddef>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -38,6 +39,7 @@ struct Layout {  // byte offsets inside the workspace
     size_t pk_stage, pk_stride;   // two areas for k_new | v_new | q of one call, contiguous
     size_t grp_in, grp_in_stride, grp_out, grp_out_stride, grp_lse, grp_lse_stride;   // two areas each for a group of layers
     size_t status;
+    size_t stamps;
     size_t total;
     int64_t max_partial_slots, max_items, max_units;
     int32_t max_append_tokens;
@@ -119,6 +121,7 @@ Layout make_layout(const ets_config* c) {
     L.grp_lse_stride = align_up((size_t)kGroupLayers * c->max_leaves * c->num_q_heads * 4, A);
     L.grp_lse = off; off += 2 * L.grp_lse_stride;
     L.status = off; off += A;
+    L.stamps = off; off += align_up(sizeof(ets::Stamps), A);
     L.total = off;
     return L;
 }
@@ -196,6 +199,7 @@ struct ets_ctx {
     // narrow kernel that it saves); 49 gives the shortest whole step on the width-256 tree.
     int32_t opt_wide = 49;
     bool opt_timing = false;
+    bool opt_stamps = false;          // device time stamps per kernel launch (ETS_OPT_TIMING = 2)
     // timing
     std::vector<cudaEvent_t> tev;   // 3 per timed call
     int64_t timed_calls = 0;
@@ -261,6 +265,15 @@ const T* blob_ptr(const ets_ctx* c, size_t off) { return reinterpret_cast<const 
 extern "C" {
 
 static int32_t host_join(ets_ctx* c, cudaStream_t s);
+
+// all starts to "never", all ends and counters to zero (synchronises the device: only used around measurements)
+static int32_t stamps_clear(ets_ctx* c) {
+    char* base = c->ws + c->lay.stamps;
+    ETS_CUDA(c, cudaDeviceSynchronize());
+    ETS_CUDA(c, cudaMemset(base, 0, sizeof(ets::Stamps)));
+    ETS_CUDA(c, cudaMemset(base + offsetof(ets::Stamps, start_ns), 0xFF, sizeof(((ets::Stamps*)nullptr)->start_ns)));
+    return ETS_OK;
+}
 
 const char* ets_version(void) { return "ets-b200 0.1"; }
 
@@ -434,7 +447,13 @@ int32_t ets_set_option(ets_ctx* c, int32_t key, int64_t value) {
             return ETS_OK;
         case ETS_OPT_TIMING:
             if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
-            c->opt_timing = value != 0;
+            if (value < 0 || value > 2) return fail(c, ETS_ERR_INVALID_ARG, "timing mode must be 0, 1 or 2");
+            c->opt_timing = value == 1;
+            if (value == 2 && !c->opt_stamps) {
+                ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+                if (int32_t rc = stamps_clear(c)) return rc;
+            }
+            c->opt_stamps = value == 2;
             return ETS_OK;
         default:
             return fail(c, ETS_ERR_INVALID_ARG, "unknown option");
@@ -594,6 +613,7 @@ static ets::AppendArgs append_args(const ets_ctx* c, int32_t layer, const void* 
     a.Hkv = c->cfg.num_kv_heads;
     a.D = c->cfg.head_dim;
     a.overlap = 0;
+    a.stamps = c->opt_stamps ? reinterpret_cast<ets::Stamps*>(c->ws + c->lay.stamps) : nullptr;
     return a;
 }
 
@@ -794,6 +814,7 @@ static ets::DecodeArgs decode_args(const ets_ctx* c, int32_t layer, const void* 
     a.scale_log2 = c->scale_log2;
     a.first_wait_polls = c->opt_first_wait_polls;
     a.wide_behind_narrow = 0;
+    a.stamps = c->opt_stamps ? reinterpret_cast<ets::Stamps*>(c->ws + c->lay.stamps) : nullptr;
     return a;
 }
 
@@ -1212,6 +1233,17 @@ int32_t ets_timing_read(ets_ctx* c, double* attn_ms, double* merge_ms, int64_t* 
     c->timed_calls = 0;
     *attn_ms = a; *merge_ms = m; *n_calls = n;
     return ETS_OK;
+}
+
+int32_t ets_stamps_read(ets_ctx* c, ets_stamps_host* out) {
+    if (!c || !out) return ETS_ERR_INVALID_ARG;
+    if (c->host_only) return fail(c, ETS_ERR_STATE, "host-only context");
+    static_assert(sizeof(ets_stamps_host) == sizeof(ets::Stamps) && ETS_STAMP_LAUNCHES == ets::kStampLaunches &&
+                      ETS_STAMP_KINDS == ets::kStampKinds, "stamp tables out of sync");
+    ETS_CUDA(c, cudaSetDevice(c->cfg.device));
+    ETS_CUDA(c, cudaDeviceSynchronize());
+    ETS_CUDA(c, cudaMemcpy(out, c->ws + c->lay.stamps, sizeof(ets::Stamps), cudaMemcpyDeviceToHost));
+    return stamps_clear(c);
 }
 
 int32_t ets_poll_status(ets_ctx* c, void* cuda_stream) {

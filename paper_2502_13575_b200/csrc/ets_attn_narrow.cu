@@ -309,6 +309,21 @@ __device__ __forceinline__ void store_partials(const DecodeArgs& a, const DevIte
 template <int N>
 struct IntTag { static constexpr int value = N; };
 
+// Device time stamps of the narrow kernel, out of line so that they do not weigh on the register allocation of the
+// streaming loop: what = 0 at kernel entry, 1 when the wait for the kernel ahead has returned, 2 when a warp is done.
+__device__ __noinline__ void narrow_stamp(Stamps* s, int what, int n_warps) {
+    if (what == 0) {
+        if (threadIdx.x == 0) stamp_start(s, 1);
+    } else if (what == 1) {
+        if (threadIdx.x == 0) stamp_start(s, 4);
+    } else if ((threadIdx.x & 31) == 0) {
+        // no warp of this launch has finished yet when any of them reads the index, so all read the same one
+        const unsigned int i = min(*((volatile unsigned int*)&s->count[1]), (unsigned int)kStampLaunches);
+        if (threadIdx.x == 0 && blockIdx.x == 0) stamp_end(s, 4, i, 1);   // the "wait returned" series advances with the launch
+        stamp_end(s, 1, i, (unsigned int)n_warps);
+    }
+}
+
 template <int D>
 // 168 registers x 256 threads leave room in the register file for a wide-kernel CTA (80 x 192)
 __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
@@ -322,6 +337,7 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
     const int grp = lane >> 2;
     const int G = a.G;
 
+    if (a.stamps) narrow_stamp(a.stamps, 0, 0);
     const bool aligned = (base & 127u) == 0;   // the swizzled tile rows must start on 128-byte boundaries
     const bool active = aligned && worker < a.n_narrow;
     if (!aligned && threadIdx.x == 0) atomicExch(a.status, -1);
@@ -445,6 +461,7 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
         }
         pdl_wait();
         pdl_launch_dependents();
+        if (a.stamps) narrow_stamp(a.stamps, 1, 0);
         if (active) fetch_finish();
 
         bool dead = false;
@@ -532,6 +549,7 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
     // Every warp of the grid reports here; the last one rewinds the queue for the next launch.  A warp's
     // claims have all returned before it gets here, so nobody touches the counter after the last report.
     __syncwarp();
+    if (a.stamps) narrow_stamp(a.stamps, 2, n_warps);
     if (lane == 0 && atomicAdd(a.queue + 1, 1) == n_warps - 1) {
         a.queue[0] = 0;
         a.queue[1] = 0;

@@ -222,6 +222,8 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
     // needs none then: the narrow kernel lets it start only after its own wait, i.e. when everything
     // earlier in the stream has completed.  Completion stays transitive because the CTA that finishes
     // last waits for the narrow kernel before it leaves (at the end of this function).
+    unsigned int stamp = 0;
+    if (a.stamps && threadIdx.x == 0) stamp = stamp_start(a.stamps, 2);
     pdl_launch_dependents();
     if (!a.wide_behind_narrow) pdl_wait();
     if (base & 1023u) {   // the swizzled operand layout needs 1024-byte aligned tiles
@@ -612,6 +614,7 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
     }
     // behind the narrow kernel: the CTA that finishes last waits for that kernel, so that this grid
     // completes after it (the others leave at once and free their SM for the CTAs still queued)
+    if (a.stamps && threadIdx.x == 0) stamp_end(a.stamps, 2, stamp, gridDim.x);
     if (a.wide_behind_narrow && threadIdx.x == 0) {
         if (atomicAdd(a.queue + 2, 1) == (int)gridDim.x - 1) {
             a.queue[2] = 0;

@@ -38,6 +38,40 @@ __host__ __device__ inline P* kv_tile(P* pool_even, P* pool_odd, int64_t pages_p
     return pool + ((size_t)head * pool_pairs(pages_per_layer) + (size_t)(page >> 1)) * 2 * tb;
 }
 
+// Device time stamps (ETS_OPT_TIMING = 2): per kind of kernel and launch, the earliest start and the latest end over
+// its CTAs, read from the GPU's global nanosecond timer.  Kinds: 0 append, 1 narrow attention, 2 wide attention,
+// 3 merge, 4 the moment the narrow kernel's wait for the kernel ahead returned (start only).  The launch index of a
+// kind is a counter that the last CTA (warp, for the narrow kernel) of a launch to finish advances; launches of one
+// kind never overlap each other here, so every CTA of a launch reads the same index.  Costs one predicate per kernel
+// when switched off (null pointer).
+constexpr int kStampKinds = 5;
+constexpr int kStampLaunches = 4096;
+struct Stamps {
+    unsigned int count[8];
+    unsigned int done[8];
+    unsigned long long start_ns[kStampKinds][kStampLaunches];
+    unsigned long long end_ns[kStampKinds][kStampLaunches];
+};
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// returns the launch index (or kStampLaunches when the table is full)
+__device__ __forceinline__ unsigned int stamp_start(Stamps* s, int kind) {
+    const unsigned int i = min(*((volatile unsigned int*)&s->count[kind]), (unsigned int)kStampLaunches);
+    if (i < (unsigned int)kStampLaunches) atomicMin(&s->start_ns[kind][i], global_ns());
+    return i;
+}
+__device__ __forceinline__ void stamp_end(Stamps* s, int kind, unsigned int i, unsigned int n_reports) {
+    if (i < (unsigned int)kStampLaunches) atomicMax(&s->end_ns[kind][i], global_ns());
+    __threadfence();
+    if (atomicAdd(&s->done[kind], 1u) == n_reports - 1) {
+        s->done[kind] = 0;
+        atomicAdd(&s->count[kind], 1u);
+    }
+}
+
 struct DevItem {
     int32_t unit_begin, unit_count, kv_head, leaf_list_begin;
     int32_t n_leaves_tile, slot_first, segment, reserved;
@@ -69,6 +103,7 @@ struct DecodeArgs {
     float scale_log2;              // sm_scale * log2(e)
     uint32_t first_wait_polls;     // give-up limit of each worker's first wait for data (kWaitPolls unless a test lowers it)
     int32_t wide_behind_narrow;    // wide kernel: launched as the narrow kernel's programmatic dependent (see launch_attention)
+    Stamps* stamps;                // nullable: device time stamps
 };
 
 constexpr uint32_t kWaitPolls = 1u << 22;   // polls after which a device-side wait gives up
@@ -97,6 +132,7 @@ struct AppendArgs {
     int64_t pages_per_layer;
     int32_t Hkv, D;
     int32_t overlap;               // 1: copy first, wait for the preceding kernel at the end (see launch_kv_append)
+    Stamps* stamps;                // nullable: device time stamps
 };
 
 void launch_kv_append(const AppendArgs& a, int n_items, int max_new, bool chained, cudaStream_t s);

@@ -64,10 +64,16 @@ __device__ __forceinline__ void kv_append_block(const AppendArgs& a) {
 // by the caller's promise; the wait at the end keeps completion transitive, so that the attention
 // kernel behind this append cannot overwrite partial results the merge kernel is still reading.
 __global__ void __launch_bounds__(256) kv_append_kernel(AppendArgs a) {
+    unsigned int stamp = 0;
+    if (a.stamps && threadIdx.x == 0) stamp = stamp_start(a.stamps, 0);
     pdl_launch_dependents();
     if (!a.overlap) pdl_wait();
     kv_append_block(a);
     if (a.overlap) pdl_wait();
+    if (a.stamps) {
+        __syncthreads();
+        if (threadIdx.x == 0) stamp_end(a.stamps, 0, stamp, gridDim.x * gridDim.y);
+    }
 }
 
 void launch_kv_append(const AppendArgs& a, int n_items, int max_new, bool chained, cudaStream_t s) {
@@ -248,11 +254,17 @@ __global__ void __launch_bounds__(kMergeWarps * 32) lse_merge_kernel(DecodeArgs 
     // dependent, the CTA may be resident while the attention kernels still run; it reads partial results
     // only after the wait, and only then lets the kernel behind it (the next append) start, so that
     // kernel runs when the attention kernels have completed.
+    unsigned int stamp = 0;
+    if (a.stamps && threadIdx.x == 0) stamp = stamp_start(a.stamps, 3);
     MergeList ml{};
     if (active) ml = merge_list(a, (int)(row / a.Hq), (int)(row % a.Hq), lane);
     pdl_wait();
     pdl_launch_dependents();
     if (active) merge_row<D>(a, (int)(row / a.Hq), (int)(row % a.Hq), lane, ml);
+    if (a.stamps) {
+        __syncthreads();
+        if (threadIdx.x == 0) stamp_end(a.stamps, 3, stamp, gridDim.x);
+    }
 }
 
 void launch_merge(const DecodeArgs& a, int D, bool chained, cudaStream_t s) {

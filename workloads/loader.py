@@ -184,7 +184,11 @@ class DecodeJob:
         with ets_note_decode_steps.  Needs two iterations of head room for the capture itself."""
         import gc
         torch = self.torch
-        side = torch.cuda.Stream(device=self.dev)
+        # one capture stream per job: the library orders its cached append list against the stream that uploaded it,
+        # and a wait on that upload's event from another stream has no place inside a capture
+        if getattr(self, "_graph_stream", None) is None:
+            self._graph_stream = torch.cuda.Stream(device=self.dev)
+        side = self._graph_stream
         with torch.cuda.stream(side):
             self.decode_tokens(1)      # an ordinary call first: it leaves the append's descriptor list on the device
         side.synchronize()
