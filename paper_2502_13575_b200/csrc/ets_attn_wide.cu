@@ -17,11 +17,15 @@
 //               reference lazily, only after it is outgrown by 2^8, saves most rescales but leaves
 //               the dominant weight off a power of two, and its bf16 rounding then shows in peaked
 //               rows whose output nearly cancels; the exact policy keeps that weight at 1.)
-// A CTA holds two stages of 64 tokens and two S buffers in tensor memory: while the softmax warps work on
-// stage s, the copies of stage s + 1 land and its S = Q K^T is already issued; the maximum pass of stage
-// s + 1 overlaps the product O += P V of stage s.  The rest of a stage is serial (softmax -> PV), so a CTA
-// alone does not saturate anything; it is sized (97 KB of shared memory, 256 TMEM columns) to sit on an SM
-// next to a CTA of the narrow kernel, launched behind it as its programmatic dependent, and the two overlap.
+// A CTA holds two stages of 64 tokens and two S buffers in tensor memory.  The K half and the V half of a
+// stage are tracked separately: a K half is free again as soon as its S = Q K^T has run, one whole stage
+// before the V half (free after O += P V), so K of stage s + 2 is already on its way while the softmax warps
+// work on stage s, and S of stage s + 1 is in tensor memory before they are done.  The tensor pipe runs
+// QK(0) QK(1) PV(0) QK(2) PV(1) QK(3) ...: a product never waits for a copy that was started less than a
+// stage ago, and what is left on the critical path of a stage is the softmax itself (maximum pass, rescale of
+// O, exponentials) plus the hand-over to PV.  A CTA alone does not saturate anything; it is sized (97 KB of
+// shared memory, 256 TMEM columns) to sit on an SM next to a CTA of the narrow kernel, launched behind it as
+// its programmatic dependent, and the two overlap.
 // Every wait is bounded.  A wait that runs out sets an abort flag that all roles poll, the status
 // word is raised, copies in flight are waited for (again boundedly), TMEM is released, and the CTA
 // returns.
@@ -33,7 +37,8 @@ namespace {
 
 constexpr int kWideThreads = 192;
 constexpr int kStageUnits = 4;                 // page slots (16 tokens each) per stage
-constexpr int kStages = 2;                     // two 64-token stages: the next one loads while this one is computed; same footprint as one of 128
+constexpr int kStages = 2;                     // two 64-token stages in shared memory (K half and V half each)
+constexpr int kInfoRing = 4;                   // stage descriptions outlive the K half they were written with (see Shared)
 constexpr uint32_t kSpin = kWaitPolls;
 constexpr uint32_t kTmemCols = 256;
 // P (bf16, 8 columns per 16 tokens) is written over the S columns it was computed from: chunk c of P
@@ -170,20 +175,26 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 struct StageInfo {
     int32_t n_units;                 // page slots in the stage (0 = end of item)
+    int32_t page[kStageUnits];       // page of each (the V copies are started later than the K copies)
     int32_t valid[kStageUnits];      // tokens held by each
     int32_t node[kStageUnits];       // node it belongs to and index of its first token there: a query that
     int32_t tok0[kStageUnits];       // is limited inside its own node (step prefill) needs them
 };
 
 struct Shared {
-    uint64_t full[kStages];          // copies of a stage have landed (producer -> MMA warp)
-    uint64_t empty[kStages];         // stage may be overwritten (PV product done -> producer)
+    uint64_t full_k[kStages];        // K copies of a stage have landed (producer -> MMA warp)
+    uint64_t full_v[kStages];        // V copies of a stage have landed
+    uint64_t empty_k[kStages];       // K half may be overwritten (QK product done -> producer)
+    uint64_t empty_v[kStages];       // V half may be overwritten (PV product done -> producer)
     uint64_t s_ready[2];             // S = Q K^T of an even / odd stage is in tensor memory (MMA -> softmax)
     uint64_t p_ready;                // P is in tensor memory (softmax -> MMA), 4 arrivals
     uint64_t o_ready;                // O += P V done (MMA -> softmax)
     uint32_t tmem_base;
     volatile int32_t abort;
-    StageInfo info[kStages];
+    // Stage st is described in info[st % 4]: it is written when the K copies of st start (QK(st - 2) done,
+    // which is before the softmax of st - 2 has read its own description) and read until PV(st) is issued;
+    // entry st % 4 is next written for st + 4, after QK(st + 2), which the tensor pipe runs after PV(st).
+    StageInfo info[kInfoRing];
 };
 
 // Called by all 32 lanes of a warp together; the answer is the same in every lane, so that the
@@ -235,19 +246,21 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
     const int G = a.G, h = it.kv_head;
     const int rows = it.n_leaves_tile * G;
 
-    // Producer step: take the next page slots of the item that hold tokens (up to kStageUnits), start their
-    // copies into stage st % kStages and publish the stage.  Returns the number of slots (0 = end marker).
-    // Called by all lanes of warp 0.  The descriptors of 32 consecutive page slots, one per lane, are kept in
-    // registers between calls: the two dependent table loads behind them are paid once per 32 slots, not once
-    // per stage.
+    // Producer step, K part: take the next page slots of the item that hold tokens (up to kStageUnits),
+    // describe stage st in info[st % kInfoRing], start the copies of their K tiles into stage st % kStages and
+    // publish.  Returns the number of slots (0 = end marker).  Called by all lanes of warp 0.  The descriptors
+    // of 32 consecutive page slots, one per lane, are kept in registers between calls: the two dependent table
+    // loads behind them are paid once per 32 slots, not once per stage.
     int u = 0, win_base = -32;
     int w_page = 0, w_valid = 0, w_node = -1, w_tok0 = 0;
     uint32_t w_live = 0;
-    auto produce = [&](uint32_t st) -> int {
+    uint32_t prod_k = 0, prod_v = 0;   // stages whose K / V copies were started
+    auto produce_k = [&](uint32_t st) -> int {
         const uint32_t s = st % kStages;
+        StageInfo* inf = &sh->info[st % kInfoRing];
         int n = 0;
         int my_pg = 0, my_vl = 0, my_nd = -1, my_t0 = 0;
-        const uint32_t kdst = ring + s * 2 * STAGE_HALF, vdst = kdst + STAGE_HALF;
+        const uint32_t kdst = ring + s * 2 * STAGE_HALF;
         while (n < kStageUnits && u < it.unit_count) {
             if (u >= win_base + 32) {
                 win_base = u;
@@ -272,40 +285,58 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
             const int vl = __shfl_sync(0xffffffffu, w_valid, src);
             const int nd = __shfl_sync(0xffffffffu, w_node, src);
             const int t0 = __shfl_sync(0xffffffffu, w_tok0, src);
-            if ((lane >> 1) == n) { my_pg = pg; my_vl = vl; my_nd = nd; my_t0 = t0; }   // lanes 2n, 2n+1: the slot's K and V copy
+            if (lane == n) { my_pg = pg; my_vl = vl; my_nd = nd; my_t0 = t0; }   // lane n: the slot's copies
             ++n;
         }
-        // All copies of the stage are started by one instruction, one lane per tile (a bulk copy occupies the
-        // lane that starts it for some hundred cycles; eight of them one after the other from a single lane
-        // were the longest link of the stage's ring of waits).  The byte count is raised first; the producer's
+        // All copies of the half stage are started by one instruction, one lane per tile (a bulk copy occupies
+        // the lane that starts it for some hundred cycles).  The byte count is raised first; the producer's
         // single arrival comes after the copies have been started, so the phase cannot end early.
         if (lane == 0 && n > 0)
-            asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full[s])), "r"((uint32_t)n * 2 * TB) : "memory");
+            asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full_k[s])), "r"((uint32_t)n * TB) : "memory");
         __syncwarp();
-        if (lane < 2 * n) {
-            const int slot = lane >> 1, kind = lane & 1;
-            if (kind == 0) {
-                sh->info[s].valid[slot] = my_vl;
-                sh->info[s].node[slot] = my_nd;
-                sh->info[s].tok0[slot] = my_t0;
-            }
-            const char* tile = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, my_pg, h, TB);
-            bulk_g2s((kind ? vdst : kdst) + slot * TB, tile + (kind ? TB : 0u), TB, smem_u32(&sh->full[s]));
+        if (lane < n) {
+            inf->page[lane] = my_pg;
+            inf->valid[lane] = my_vl;
+            inf->node[lane] = my_nd;
+            inf->tok0[lane] = my_t0;
+            bulk_g2s(kdst + lane * TB, kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, my_pg, h, TB), TB, smem_u32(&sh->full_k[s]));
         }
         __syncwarp();
         if (u > it.unit_count) u = it.unit_count;
         if (lane == 0) {
-            sh->info[s].n_units = n;                 // n == 0: end marker
-            mbar_arrive(smem_u32(&sh->full[s]));      // publishes the stage info with release semantics
+            inf->n_units = n;                         // n == 0: end marker
+            mbar_arrive(smem_u32(&sh->full_k[s]));    // publishes the stage info with release semantics
         }
         __syncwarp();
+        if (n > 0) ++prod_k;
         return n;
+    };
+    // V part of a stage that produce_k described: its V tiles follow the K tiles in the page image.
+    auto produce_v = [&](uint32_t st) {
+        const uint32_t s = st % kStages;
+        const StageInfo* inf = &sh->info[st % kInfoRing];
+        const int n = inf->n_units;
+        const uint32_t vdst = ring + s * 2 * STAGE_HALF + STAGE_HALF;
+        if (lane == 0)
+            asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh->full_v[s])), "r"((uint32_t)n * TB) : "memory");
+        __syncwarp();
+        if (lane < n)
+            bulk_g2s(vdst + lane * TB, kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, inf->page[lane], h, TB) + TB, TB, smem_u32(&sh->full_v[s]));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh->full_v[s]));
+        __syncwarp();
+        ++prod_v;
     };
 
     int n_first = 0;
     if (warp == 0) {
         if (lane == 0) {
-            for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
+            for (int s = 0; s < kStages; ++s) {
+                mbar_init(smem_u32(&sh->full_k[s]), 1);
+                mbar_init(smem_u32(&sh->full_v[s]), 1);
+                mbar_init(smem_u32(&sh->empty_k[s]), 1);
+                mbar_init(smem_u32(&sh->empty_v[s]), 1);
+            }
             mbar_init(smem_u32(&sh->s_ready[0]), 1);
             mbar_init(smem_u32(&sh->s_ready[1]), 1);
             mbar_init(smem_u32(&sh->p_ready), 4);
@@ -319,7 +350,8 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         // the first stage's copies start before anybody else is ready for them
-        n_first = produce(0);
+        n_first = produce_k(0);
+        if (n_first > 0) produce_v(0);
     } else {
         // Q tile: query row r = (leaf r / G of the tile, head h*G + r % G), K-major with the 128-byte
         // swizzle.  The producer warp is already fetching K/V meanwhile.  Leaf ids are fetched once
@@ -361,17 +393,19 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
     asm volatile("bar.sync 1, %0;" ::"r"(kWideThreads) : "memory");   // barriers, TMEM address, Q tile: visible to all
     tc_fence_after();
     const uint32_t tmem = sh->tmem_base;
-    uint32_t prod_stages = 0;   // producer only: stages whose copies were started
-
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
-        if (n_first > 0) {
-            prod_stages = 1;
-            for (uint32_t st = 1;; ++st) {
-                const uint32_t s = st % kStages;
-                if (st >= (uint32_t)kStages && !wait_or_abort(smem_u32(&sh->empty[s]), ((st / kStages) - 1) & 1u, sh)) break;
-                if (produce(st) == 0) break;
-                ++prod_stages;
+        // Order of the copies: K0 V0 K1 V1 K2, then K(j+1), V(j) for j = 2, 3, ...: a K half is refilled when
+        // the product that read it has run, which is a whole stage before the V half of the same stage is free.
+        if (n_first > 0 && produce_k(1) > 0) {
+            produce_v(1);
+            int n_next = 0;
+            if (wait_or_abort(smem_u32(&sh->empty_k[0]), 0u, sh)) n_next = produce_k(2);            // QK(0) has run
+            for (uint32_t j = 2; n_next > 0; ++j) {    // stage j: K on its way, V not yet
+                if (!wait_or_abort(smem_u32(&sh->empty_k[(j + 1) % kStages]), (((j + 1) / kStages) - 1) & 1u, sh)) break;   // QK(j - 1)
+                n_next = produce_k(j + 1);
+                if (!wait_or_abort(smem_u32(&sh->empty_v[j % kStages]), ((j / kStages) - 1) & 1u, sh)) break;               // PV(j - 2)
+                produce_v(j);
             }
         }
     } else if (warp == 1) {
@@ -380,27 +414,13 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
         // S = Q K^T of stage st into S buffer st % 2 (or the end marker); returns the stage's page slots, -1 on abort
         auto issue_qk = [&](uint32_t st) -> int {
             const uint32_t s = st % kStages;
-            if (!wait_or_abort(smem_u32(&sh->full[s]), (st / kStages) & 1u, sh, st == 0 ? a.first_wait_polls : kSpin)) return -1;
-            const int n = sh->info[s].n_units;
+            if (!wait_or_abort(smem_u32(&sh->full_k[s]), (st / kStages) & 1u, sh, st == 0 ? a.first_wait_polls : kSpin)) return -1;
+            const int n = sh->info[st % kInfoRing].n_units;
             if (n == 0) {   // end of item: wake the softmax warps, which then see the same marker
                 if (lane == 0) mbar_arrive(smem_u32(&sh->s_ready[st & 1u]));
                 return 0;
             }
-            const uint32_t kst = ring + s * 2 * STAGE_HALF, vst = kst + STAGE_HALF;
-            // rows past a page's length hold stale bytes; zero them in V (0 * garbage could be NaN)
-            bool wrote = false;
-            for (int k = 0; k < n; ++k) {
-                const int valid = sh->info[s].valid[k];
-                if (valid < 16) {
-                    for (int i = lane; i < (16 - valid) * (D / 8); i += 32) {
-                        const int t = valid + i / (D / 8), c = i % (D / 8);
-                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vst + k * TB + tile_offset(D, t, c * 8)), "r"(0u) : "memory");
-                    }
-                    wrote = true;
-                }
-            }
-            if (wrote) fence_proxy_async();
-            __syncwarp();
+            const uint32_t kst = ring + s * 2 * STAGE_HALF;
             tc_fence_after();
             if (lane == 0) {
                 const uint32_t idesc_qk = instr_desc(16u * n, false);
@@ -411,18 +431,34 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
                             smem_desc(kst + koff, 16, 1024u * (D / 64)), idesc_qk, ks > 0);
                 }
                 umma_commit(smem_u32(&sh->s_ready[st & 1u]));
+                umma_commit(smem_u32(&sh->empty_k[s]));
             }
             __syncwarp();
             return n;
         };
-        // The S buffer of stage st + 1 held stage st - 1, whose second product was issued by this thread
-        // before: the tensor pipe runs a thread's products in order, so the buffer is free by then.
+        // The S buffer of stage st + 2 held S and P of stage st, whose second product was issued by this
+        // thread just before: the tensor pipe runs a thread's products in order, so the buffer is free by then.
         int n = issue_qk(0);
-        for (uint32_t st = 0; n > 0; ++st) {
+        int n_next = n > 0 ? issue_qk(1) : 0;
+        for (uint32_t st = 0; n > 0 && n_next >= 0; ++st) {
             const uint32_t s = st % kStages;
-            const int n_next = issue_qk(st + 1);
-            if (n_next < 0) break;
+            const StageInfo* inf = &sh->info[st % kInfoRing];
             const uint32_t vst = ring + s * 2 * STAGE_HALF + STAGE_HALF;
+            if (!wait_or_abort(smem_u32(&sh->full_v[s]), (st / kStages) & 1u, sh)) break;
+            // rows past a page's length hold stale bytes; zero them in V (0 * garbage could be NaN)
+            bool wrote = false;
+            for (int k = 0; k < n; ++k) {
+                const int valid = inf->valid[k];
+                if (valid < 16) {
+                    for (int i = lane; i < (16 - valid) * (D / 8); i += 32) {
+                        const int t = valid + i / (D / 8), c = i % (D / 8);
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vst + k * TB + tile_offset(D, t, c * 8)), "r"(0u) : "memory");
+                    }
+                    wrote = true;
+                }
+            }
+            if (wrote) fence_proxy_async();
+            __syncwarp();
             if (!wait_or_abort(smem_u32(&sh->p_ready), st & 1u, sh)) break;
             tc_fence_after();
             if (lane == 0) {
@@ -433,11 +469,14 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
                 for (int k = 0; k < n; ++k)
                     umma_ts(tmem + kColO, tmem + kColP + kColPLo + kColSBuf * (st & 1u) + p_col(k), smem_desc(vst + k * TB, 1024, 1024u * (D / 64)),
                             idesc_pv, true);
-                umma_commit(smem_u32(&sh->empty[s]));
+                umma_commit(smem_u32(&sh->empty_v[s]));
                 umma_commit(smem_u32(&sh->o_ready));
             }
             __syncwarp();
+            int n_after = 0;
+            if (n_next > 0) n_after = issue_qk(st + 2);
             n = n_next;
+            n_next = n_after;
         }
     } else {
         // ------------------------------------------------------------------ softmax, one row per thread
@@ -462,9 +501,9 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
             return v;
         };
         for (uint32_t st = 0;; ++st) {
-            const uint32_t s = st % kStages;
+            const uint32_t s = st % kInfoRing;
             if (!wait_or_abort(smem_u32(&sh->s_ready[st & 1u]), (st >> 1) & 1u, sh)) { ok = false; break; }
-            // s_ready can only complete after the MMA warp saw full[s]: the stage info is visible
+            // s_ready can only complete after the MMA warp saw full_k of the stage: the stage info is visible
             const int n = sh->info[s].n_units;
             if (n == 0) break;   // end marker passed on by the MMA warp
             tc_fence_after();
@@ -600,9 +639,12 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
         if (threadIdx.x == 0) atomicExch(a.status, -7);
         // copies that were started still target this CTA's shared memory: give them time to land
         if (warp == 0) {
-            const uint32_t lo = prod_stages > (uint32_t)kStages ? prod_stages - kStages : 0u;
-            for (uint32_t st = lo; st < prod_stages; ++st) {
-                const uint32_t bar = smem_u32(&sh->full[st % kStages]), par = (st / kStages) & 1u;
+            for (uint32_t st = prod_k > (uint32_t)kStages ? prod_k - kStages : 0u; st < prod_k; ++st) {
+                const uint32_t bar = smem_u32(&sh->full_k[st % kStages]), par = (st / kStages) & 1u;
+                for (uint32_t i = 0; i < kSpin && !mbar_try_wait(bar, par); ++i) {}
+            }
+            for (uint32_t st = prod_v > (uint32_t)kStages ? prod_v - kStages : 0u; st < prod_v; ++st) {
+                const uint32_t bar = smem_u32(&sh->full_v[st % kStages]), par = (st / kStages) & 1u;
                 for (uint32_t i = 0; i < kSpin && !mbar_try_wait(bar, par); ++i) {}
             }
         }
