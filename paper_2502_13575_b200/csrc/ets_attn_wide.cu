@@ -363,7 +363,7 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
         const int leaf_hi = (lane + 32 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 32] : 0;
         const int leaf_h2 = (lane + 64 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 64] : 0;
         const int leaf_h3 = (lane + 96 < it.n_leaves_tile) ? a.node_leaves[it.leaf_list_begin + lane + 96] : 0;
-        constexpr int kBatch = 7;   // loads in flight per thread; bounded to keep registers low
+        constexpr int kBatch = kPer;   // all of a thread's loads in flight at once: the roles' registers are not live yet
 #pragma unroll 1
         for (int k0 = 0; k0 < kPer; k0 += kBatch) {
             uint4 v[kBatch];
@@ -614,6 +614,15 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
             a.part_ml[prow] = make_float2(m_ref, l);
         }
         if (ok) {
+            // O goes out through shared memory: a thread owns a row, so stores straight from its registers would
+            // touch 32 different 512-byte rows per instruction.  Each thread lays its row down in the (now idle)
+            // Q tile and K/V ring, rows 16 bytes apart from a multiple of 512 so that the 16-byte stores of a
+            // warp spread over all banks, and sends it with one bulk copy.  Nothing else uses that memory any
+            // more: the wait for the last product above covers every product of this CTA, and every copy that
+            // was started has been consumed by one of them.
+            constexpr uint32_t kRowBytes = D * 4 + 16;
+            static_assert(128u * kRowBytes <= 128u * D * 2u + kStages * 2u * STAGE_HALF, "O staging fits in the Q tile and the ring");
+            const uint32_t row_smem = base + (uint32_t)row * kRowBytes;
             float* po = a.part_o + ((size_t)(it.slot_first + row / G) * G + row % G) * D;
 #pragma unroll 1
             for (int c = 0; c < D; c += 32) {
@@ -623,11 +632,17 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = 0.f;
                 }
-                if (row < rows) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        *reinterpret_cast<float4*>(po + c + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                }
+                for (int i = 0; i < 32; i += 4)
+                    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(row_smem + (uint32_t)(c + i) * 4u), "f"(v[i]), "f"(v[i + 1]),
+                                 "f"(v[i + 2]), "f"(v[i + 3])
+                                 : "memory");
+            }
+            if (row < rows) {
+                fence_proxy_async();   // the row was written by ordinary stores and is read by the copy engine
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(po), "r"(row_smem), "r"((uint32_t)(D * 4)) : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // own copy only; it reads this CTA's shared memory
             }
         }
     }
