@@ -341,7 +341,7 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
 #define ETS_OPT_KERNEL        2  /* 0 tensor-core attention kernels (default), 1 scalar-FMA kernel;  */
                                  /* rebuild the tree after changing it                             */
 #define ETS_OPT_WIDE          4  /* smallest query group, in rows (leaves * Hq/Hkv, at least 17), that */
-                                 /* goes to the tcgen05 kernel (default 49); 0: none.  Next build.      */
+                                 /* goes to the tcgen05 kernel (default 33); 0: none.  Next build.      */
                                  /* While the option is untouched, a tree so small that a warp of the    */
                                  /* streaming kernel would read four page slots or fewer gets no such    */
                                  /* items (the second kernel's launch costs more than it saves there).   */

@@ -193,11 +193,11 @@ struct ets_ctx {
     // ets_device.cuh); 0: ordinary launches, the wide kernel on a second stream forked from the caller's.
     bool opt_chain = true;
     uint32_t opt_first_wait_polls = ets::kWaitPolls;
-    // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on the width-256 tree and on
-    // eight width-64 trees: 33, 49 and 65 are within a microsecond of each other per layer, 17 and "never" are
-    // 20 % slower (below ~32 rows the per-item latency of the wide kernel costs more than the re-reads by the
-    // narrow kernel that it saves); 49 gives the shortest whole step on the width-256 tree.
-    int32_t opt_wide = 49;
+    // smallest query group (rows) sent to the wide kernel; 0 = never.  Measured on width-256 trees and on
+    // eight width-64 trees: 33 is 1-2 % ahead of 49 and 65 per layer, 25 is 2-12 % and 17 15-20 % slower (below
+    // ~32 rows the per-item latency of the wide kernel costs more than the re-reads by the narrow kernel that
+    // it saves).
+    int32_t opt_wide = 33;
     bool opt_timing = false;
     bool opt_stamps = false;          // device time stamps per kernel launch (ETS_OPT_TIMING = 2)
     // timing
