@@ -168,6 +168,12 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// maximum of three (one instruction on sm_100)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -518,9 +524,9 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
                 float m0 = -INFINITY, m1 = -INFINITY;
                 if (v0 == 16 && v1 == 16) {   // two full pages, the usual case: no per-token test
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        m0 = fmaxf(m0, v[i]);
-                        m1 = fmaxf(m1, v[16 + i]);
+                    for (int i = 0; i < 16; i += 2) {
+                        m0 = max3(m0, v[i], v[i + 1]);
+                        m1 = max3(m1, v[16 + i], v[16 + i + 1]);
                     }
                 } else {
 #pragma unroll
@@ -551,8 +557,13 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
                     for (int c = 0; c < D; c += 32) {
                         float v[32];
                         tmem_ld32(tlane + kColO + c, v);
+                        const float2 f2 = make_float2(f, f);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] *= f;
+                        for (int i = 0; i < 32; i += 2) {   // packed fp32 multiplies: half the instructions
+                            const float2 r = __fmul2_rn(make_float2(v[i], v[i + 1]), f2);
+                            v[i] = r.x;
+                            v[i + 1] = r.y;
+                        }
                         tmem_st32(tlane + kColO + c, v);
                     }
                     tmem_wait_st();
@@ -565,8 +576,11 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
             // value and the rounded rest: with one term the weights would be off by up to 2^-8 each,
             // which on a path of a few tokens with values of opposite sign exceeds the output's
             // tolerance.  Both terms of a pair go where the pair's S was.
-            float l0 = 0.f, l1 = 0.f;
-            const float neg_ref = -m_ref;
+            // The scaling, the rests and the row sums use the packed fp32 instructions (two lanes per
+            // instruction): the softmax warps are bound by the number of instructions they issue.
+            float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+            const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), nr2 = make_float2(-m_ref, -m_ref);
+            const float2 minus1 = make_float2(-1.f, -1.f);
             for (int c = 0; c < n; c += 2) {
                 float v[32];
                 tmem_ld32(tlane + kColS + kColSBuf * (st & 1u) + 16u * c, v);
@@ -578,16 +592,22 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
                 for (int i = 0; i < 16; i += 2) {
                     // weights are at most 1 and are rounded to bf16 next: the approximate exponential
                     // (2 ulp, tiny results flushed to zero) loses nothing
-                    const float a0 = (full || i < v0) ? ex2_approx(fmaf(v[i], a.scale_log2, neg_ref)) : 0.f;
-                    const float a1 = (full || i + 1 < v0) ? ex2_approx(fmaf(v[i + 1], a.scale_log2, neg_ref)) : 0.f;
-                    const float b0 = (full || i < v1) ? ex2_approx(fmaf(v[16 + i], a.scale_log2, neg_ref)) : 0.f;
-                    const float b1 = (full || i + 1 < v1) ? ex2_approx(fmaf(v[16 + i + 1], a.scale_log2, neg_ref)) : 0.f;
-                    const __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1);
-                    const __nv_bfloat162 pb = __floats2bfloat162_rn(b0, b1);
-                    const __nv_bfloat162 qa = __floats2bfloat162_rn(a0 - __low2float(pa), a1 - __high2float(pa));
-                    const __nv_bfloat162 qb = __floats2bfloat162_rn(b0 - __low2float(pb), b1 - __high2float(pb));
-                    l0 += a0 + a1;
-                    l1 += b0 + b1;
+                    const float2 xa = __ffma2_rn(make_float2(v[i], v[i + 1]), sc2, nr2);
+                    const float2 xb = __ffma2_rn(make_float2(v[16 + i], v[16 + i + 1]), sc2, nr2);
+                    float2 wa, wb;
+                    wa.x = (full || i < v0) ? ex2_approx(xa.x) : 0.f;
+                    wa.y = (full || i + 1 < v0) ? ex2_approx(xa.y) : 0.f;
+                    wb.x = (full || i < v1) ? ex2_approx(xb.x) : 0.f;
+                    wb.y = (full || i + 1 < v1) ? ex2_approx(xb.y) : 0.f;
+                    const __nv_bfloat162 pa = __floats2bfloat162_rn(wa.x, wa.y);
+                    const __nv_bfloat162 pb = __floats2bfloat162_rn(wb.x, wb.y);
+                    // rest = weight - rounded weight (exact in fp32)
+                    const float2 ra = __ffma2_rn(make_float2(__low2float(pa), __high2float(pa)), minus1, wa);
+                    const float2 rb = __ffma2_rn(make_float2(__low2float(pb), __high2float(pb)), minus1, wb);
+                    const __nv_bfloat162 qa = __floats2bfloat162_rn(ra.x, ra.y);
+                    const __nv_bfloat162 qb = __floats2bfloat162_rn(rb.x, rb.y);
+                    la = __fadd2_rn(la, wa);
+                    lb = __fadd2_rn(lb, wb);
                     pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pa);
                     pk[8 + (i >> 1)] = *reinterpret_cast<const uint32_t*>(&pb);
                     plo[i >> 1] = *reinterpret_cast<const uint32_t*>(&qa);
@@ -596,6 +616,7 @@ __global__ void __maxnreg__(88) attn_partial_wide_kernel(DecodeArgs a, int first
                 tmem_st16(tlane + kColP + kColSBuf * (st & 1u) + p_col(c), pk);
                 tmem_st16(tlane + kColP + kColPLo + kColSBuf * (st & 1u) + p_col(c), plo);
             }
+            const float l0 = la.x + la.y, l1 = lb.x + lb.y;
             l += l0 + l1;
             tmem_wait_st();
             tc_fence_before();
