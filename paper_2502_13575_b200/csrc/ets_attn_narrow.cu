@@ -119,9 +119,10 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
     return y;
 }
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 // The page slots of one narrow item, one per lane (an item has at most 32): page id and the number
@@ -222,46 +223,62 @@ __device__ __forceinline__ void tile_step(uint32_t kt, uint32_t vt, int valid, f
         for (int i = 0; i < 4; ++i) s[0][i] += s2[0][i];
     }
 
-    // online softmax (log2 units); this lane holds tokens grp and grp+8 of rows 2quad, 2quad+1
+    // online softmax (log2 units); this lane holds tokens grp and grp+8 of rows 2quad, 2quad+1.  The two rows
+    // go through the packed fp32 instructions together (one instruction for both): the warp is a chain of
+    // dependent instructions and their number is what a tile costs.
     uint32_t pf[NT][2], pg[NT][2];
 #pragma unroll
     for (int j = 0; j < NT; ++j) {
-        float sv[4];
+        const float2 sc2 = make_float2(scale_log2, scale_log2);
+        // (row 2quad, row 2quad+1) of token grp and of token grp+8; tokens past the node's length are masked
+        float2 sa = __fmul2_rn(make_float2(s[j][0], s[j][1]), sc2);
+        float2 sb = __fmul2_rn(make_float2(s[j][2], s[j][3]), sc2);
+        if (grp >= valid) sa = make_float2(-INFINITY, -INFINITY);
+        if (grp + 8 >= valid) sb = make_float2(-INFINITY, -INFINITY);
+        float2 mx = make_float2(fmaxf(sa.x, sb.x), fmaxf(sa.y, sb.y));
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int tok = grp + (i >> 1) * 8;
-            sv[i] = tok < valid ? s[j][i] * scale_log2 : -INFINITY;
+        for (int d = 4; d <= 16; d <<= 1) {
+            mx.x = fmaxf(mx.x, __shfl_xor_sync(0xffffffffu, mx.x, d));
+            mx.y = fmaxf(mx.y, __shfl_xor_sync(0xffffffffu, mx.y, d));
         }
-        float p[4], pl[4];
+        // finite: token 0 of the tile is valid
+        const float2 mn = make_float2(fmaxf(acc.m[j][0], mx.x), fmaxf(acc.m[j][1], mx.y));
+        const float2 neg = make_float2(-mn.x, -mn.y);
+        const float2 corr = make_float2(ex2_approx(acc.m[j][0] + neg.x), ex2_approx(acc.m[j][1] + neg.y));
+        const float2 da = __fadd2_rn(sa, neg), db = __fadd2_rn(sb, neg);
+        // weights are at most 1 and are rounded to bf16 next: the approximate exponential (2 ulp, tiny results
+        // flushed to zero) loses nothing
+        const float2 ea = make_float2(ex2_approx(da.x), ex2_approx(da.y));
+        const float2 eb = make_float2(ex2_approx(db.x), ex2_approx(db.y));
+        // A weight enters the product as two bf16 terms, its rounded value and the rounded rest
+        // (16 bits of it in all): with one term the weights would be off by up to 2^-8 each, which
+        // on a path of a few tokens with values of opposite sign exceeds the output's tolerance.
+        const __nv_bfloat162 pa = __floats2bfloat162_rn(ea.x, ea.y);
+        const __nv_bfloat162 pb = __floats2bfloat162_rn(eb.x, eb.y);
+        const float2 minus1 = make_float2(-1.f, -1.f);
+        const float2 ra = __ffma2_rn(make_float2(__low2float(pa), __high2float(pa)), minus1, ea);
+        const float2 rb = __ffma2_rn(make_float2(__low2float(pb), __high2float(pb)), minus1, eb);
+        const __nv_bfloat162 qa = __floats2bfloat162_rn(ra.x, ra.y);
+        const __nv_bfloat162 qb = __floats2bfloat162_rn(rb.x, rb.y);
+        const float2 l2 = __fadd2_rn(__ffma2_rn(make_float2(acc.l[j][0], acc.l[j][1]), corr, ea), eb);
+        acc.l[j][0] = l2.x;
+        acc.l[j][1] = l2.y;
+        acc.m[j][0] = mn.x;
+        acc.m[j][1] = mn.y;
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            float mx = fmaxf(sv[r], sv[r + 2]);
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-            const float mn = fmaxf(acc.m[j][r], mx);     // finite: token 0 of the tile is valid
-            const float corr = exp2f(acc.m[j][r] - mn);
-            // A weight enters the product as two bf16 terms, its rounded value and the rounded rest
-            // (16 bits of it in all): with one term the weights would be off by up to 2^-8 each, which
-            // on a path of a few tokens with values of opposite sign exceeds the output's tolerance.
-            const float e0 = exp2f(sv[r] - mn), e1 = exp2f(sv[r + 2] - mn);
-            p[r] = __bfloat162float(__float2bfloat16_rn(e0));
-            p[r + 2] = __bfloat162float(__float2bfloat16_rn(e1));
-            pl[r] = e0 - p[r];
-            pl[r + 2] = e1 - p[r + 2];
-            acc.l[j][r] = acc.l[j][r] * corr + e0 + e1;
-            acc.m[j][r] = mn;
-#pragma unroll
-            for (int mt = 0; mt < KS; ++mt) {
-                acc.o[mt][j][r] *= corr;
-                acc.o[mt][j][r + 2] *= corr;
-            }
+        for (int mt = 0; mt < KS; ++mt) {
+            const float2 o01 = __fmul2_rn(make_float2(acc.o[mt][j][0], acc.o[mt][j][1]), corr);
+            const float2 o23 = __fmul2_rn(make_float2(acc.o[mt][j][2], acc.o[mt][j][3]), corr);
+            acc.o[mt][j][0] = o01.x;
+            acc.o[mt][j][1] = o01.y;
+            acc.o[mt][j][2] = o23.x;
+            acc.o[mt][j][3] = o23.y;
         }
         // P^T as B operand: transpose the two 8x8 (token x row) blocks
-        pf[j][0] = movmatrix_trans(pack_bf16(p[0], p[1]));
-        pf[j][1] = movmatrix_trans(pack_bf16(p[2], p[3]));
-        pg[j][0] = movmatrix_trans(pack_bf16(pl[0], pl[1]));
-        pg[j][1] = movmatrix_trans(pack_bf16(pl[2], pl[3]));
+        pf[j][0] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pa));
+        pf[j][1] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pb));
+        pg[j][0] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&qa));
+        pg[j][1] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&qb));
     }
 
     // O^T += V_tile^T . P^T
