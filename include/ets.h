@@ -344,7 +344,9 @@ int32_t ets_get_stats(const ets_ctx* ctx, ets_stats* out);
                                  /* goes to the tcgen05 kernel (default 33); 0: none.  Next build.      */
                                  /* While the option is untouched, a tree so small that a warp of the    */
                                  /* streaming kernel would read four page slots or fewer gets no such    */
-                                 /* items (the second kernel's launch costs more than it saves there).   */
+                                 /* items (the second kernel's launch costs more than it saves there),   */
+                                 /* and a tree on which the tcgen05 kernel would end after the streaming */
+                                 /* kernel (most of its K/V under large query groups) is built with 49.  */
 #define ETS_OPT_PATH_ITEMS    7  /* 1: the next builds serve ets_tree_attn_prefill only: a work item is one   */
                                  /* (node that leaves sit at, kv head, tile of its leaves) and walks the node's */
                                  /* whole path, so a dense tile keeps its accumulator resident and leaves one  */

@@ -469,6 +469,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
     fp.wide_rows = (c->opt_wide > 0 && c->opt_kernel == 0) ? 128 : 0;
     fp.wide_min_rows = c->opt_wide;
     if (c->opt_wide_set) fp.wide_min_work = 0;
+    fp.wide_alt_rows = c->opt_wide_set ? 0 : 49;   // see ets_flatten.cpp: where the limit sits when the wide kernel would end last
     fp.path_items = c->opt_path_items;
     // A rebuild of the very tree that is current (same arrays, every node keeping its own pages, same options)
     // changes nothing: tables, pages and lengths, on the host and on the device, already are what it would produce.
@@ -476,6 +477,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
         n_leaves >= 0 && (n_nodes == 0 || (parent && cap_tokens)) && (n_leaves == 0 || leaf_node) &&
         fp.chunk_pages == c->built.chunk_pages && fp.wide_rows == c->built.wide_rows &&
         fp.wide_min_rows == c->built.wide_min_rows && fp.wide_min_work == c->built.wide_min_work &&
+        fp.wide_alt_rows == c->built.wide_alt_rows &&
         fp.path_items == c->built.path_items &&
         std::memcmp(parent, c->tree.parent.data(), (size_t)n_nodes * 4) == 0 &&
         std::memcmp(cap_tokens, c->tree.cap.data(), (size_t)n_nodes * 4) == 0 &&

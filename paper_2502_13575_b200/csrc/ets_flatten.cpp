@@ -203,9 +203,28 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             all_narrow += (int64_t)(seg_unit_off[s + 1] - seg_unit_off[s]) * p.num_kv_heads * ceil_div(g[seg_head[s]], leaves_per_tile);
         wide_pays = all_narrow > (int64_t)p.wide_min_work * n_workers;
     }
+    // Which of the two kernels ends last decides where the limit should sit: a tree whose bytes are under
+    // large query groups keeps the wide kernel busy after the narrow one has finished, and every group the
+    // narrow kernel takes over shortens the call; a tree with little sharing has the narrow kernel on the
+    // critical path and the wide kernel idle at the end.  Run times of both at the lower limit, from counts
+    // (fits to device time stamps on a 148-SM GPU: a narrow warp needs 1.5 us per page-slot visit, a wide
+    // item 7 us per 64-token stage including its share of prologue and epilogue, one item per SM at a time).
+    int32_t wide_min_rows = p.wide_min_rows;
+    if (wide_pays && !p.path_items && p.wide_alt_rows > wide_min_rows) {
+        const int32_t wide_leaves = std::max(1, p.wide_rows / std::max(1, p.gqa));
+        int64_t visits = 0, stages = 0;
+        for (int32_t s = 0; s < n_seg; ++s) {
+            const int32_t nu = seg_unit_off[s + 1] - seg_unit_off[s], gn = g[seg_head[s]], r = gn * p.gqa;
+            if (r > p.rows_per_item && r >= wide_min_rows) stages += (int64_t)ceil_div(nu, 4) * p.num_kv_heads * ceil_div(gn, wide_leaves);
+            else visits += (int64_t)nu * p.num_kv_heads * ceil_div(gn, leaves_per_tile);
+        }
+        const double t_narrow = 5.0 + 1.5 * (double)visits / n_workers;
+        const double t_wide = 7.0 + 7.0 * (double)stages / std::max(1, n_workers / 8);
+        if (t_wide > t_narrow) wide_min_rows = p.wide_alt_rows;
+    }
     auto is_wide = [&](int32_t s) {
         const int32_t r = g[seg_head[s]] * p.gqa;
-        return wide_pays && r > p.rows_per_item && r >= p.wide_min_rows;
+        return wide_pays && r > p.rows_per_item && r >= wide_min_rows;
     };
     struct Part { int32_t seg, begin, len; };
     // per narrow segment: page slots, pieces per part (heads x leaf tiles), mean weight of a page slot

@@ -32,6 +32,7 @@ struct FlattenParams {
     int32_t wide_rows = 0;      // query rows one wide (tcgen05) item covers; 0 = no wide items
     int32_t wide_min_rows = 17; // smallest query group (in rows) that is treated as wide
     int32_t wide_min_work = 4;   // no wide items below this many page-slot visits per warp (counted as if all were narrow)
+    int32_t wide_alt_rows = 0;   // if larger than wide_min_rows: the limit used instead when the wide kernel would end after the narrow one
     int32_t wide_max_units = 32; // longest page run of a wide item
     int32_t wide_piece = 0;      // page run of a wide item (0 = chosen by the builder)
     bool path_items = false;     // step prefill: items walk whole root-to-node paths (see tree_build)

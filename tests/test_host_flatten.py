@@ -282,6 +282,23 @@ def test_small_trees_get_no_wide_items_unless_asked():
     assert n_narrow < n_items
 
 
+def test_wide_limit_follows_the_kernel_that_would_end_last():
+    """While ETS_OPT_WIDE is untouched the limit is 33 rows where the streaming kernel is on the critical path
+    (little sharing: the width-256 tree) and 49 where the tcgen05 kernel would end last (most K/V under large
+    query groups: the random-sharing tree, an ETS-pruned width-256 tree)."""
+    def counts(name, wide=None):
+        wl = make_workload(name)
+        g = wl.geometry
+        ctx = host_ctx(g.num_q_heads, g.num_kv_heads, g.head_dim, pages=1 << 16, max_path_tokens=1 << 16, max_path_entries=1 << 20, max_nodes=4096, max_leaves=1024)
+        if wide is not None:
+            ctx.set_option(ets.ETS_OPT_WIDE, wide)
+        ctx.tree_build(wl.tree.parent, wl.tree.tokens, wl.tree.leaf_node)
+        return ctx.get_stats()["n_narrow_items"], len(ctx.work_export()["item"])
+    assert counts("cfg4") == counts("cfg4", wide=33) != counts("cfg4", wide=49)
+    assert counts("cfg5c") == counts("cfg5c", wide=49) != counts("cfg5c", wide=33)
+    assert counts("search_w256_ets") == counts("search_w256_ets", wide=49) != counts("search_w256_ets", wide=33)
+
+
 def test_path_items_cover_every_path_once():
     """ETS_OPT_PATH_ITEMS: one item per (node that leaves sit at, kv head, tile of those leaves); its page slots
     are the node's whole path in root-to-node order; every leaf gets exactly one partial slot per kv head; the
