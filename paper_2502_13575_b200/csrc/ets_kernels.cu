@@ -245,7 +245,7 @@ void launch_partial_fma(const DecodeArgs& a, int D, int n_items, cudaStream_t s)
 #endif
 constexpr int kMergeWarps = ETS_MERGE_WARPS;
 
-template <int D>
+template <int D, int kEarly>
 __global__ void __launch_bounds__(kMergeWarps * 32) lse_merge_kernel(DecodeArgs a) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * kMergeWarps + warp;
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kMergeWarps * 32) lse_merge_kernel(DecodeArgs 
     if (active) ml = merge_list(a, (int)(row / a.Hq), (int)(row % a.Hq), lane);
     pdl_wait();
     pdl_launch_dependents();
-    if (active) merge_row<D>(a, (int)(row / a.Hq), (int)(row % a.Hq), lane, ml);
+    if (active) merge_row<D, kEarly>(a, (int)(row / a.Hq), (int)(row % a.Hq), lane, ml);
     if (a.stamps) {
         __syncthreads();
         if (threadIdx.x == 0) stamp_end(a.stamps, 3, stamp, gridDim.x);
@@ -272,8 +272,17 @@ void launch_merge(const DecodeArgs& a, int D, bool chained, cudaStream_t s) {
     if (rows <= 0) return;
     const int blocks = (int)((rows + kMergeWarps - 1) / kMergeWarps);
     ChainLaunch l(dim3(blocks), dim3(kMergeWarps * 32), 0, s, chained);
-    if (D == 128) cudaLaunchKernelEx(&l.cfg, lse_merge_kernel<128>, a);
-    else cudaLaunchKernelEx(&l.cfg, lse_merge_kernel<64>, a);
+    // A row usually has 8 to 12 partials.  With 12 of them fetched in the first round trip a warp needs more
+    // registers and fewer CTAs fit on an SM: taken when the whole grid is resident at once even so (one
+    // width-64 tree), where it saves the second round trip; larger grids keep 8 and the higher occupancy.
+    const bool small_grid = blocks <= 148 * 4;
+    if (D == 128) {
+        if (small_grid) cudaLaunchKernelEx(&l.cfg, lse_merge_kernel<128, 12>, a);
+        else cudaLaunchKernelEx(&l.cfg, lse_merge_kernel<128, 8>, a);
+    } else {
+        if (small_grid) cudaLaunchKernelEx(&l.cfg, lse_merge_kernel<64, 12>, a);
+        else cudaLaunchKernelEx(&l.cfg, lse_merge_kernel<64, 8>, a);
+    }
 }
 
 }  // namespace ets

@@ -26,7 +26,8 @@ __device__ __forceinline__ MergeList merge_list(const DecodeArgs& a, int leaf, i
     return m;
 }
 
-template <int D>
+// kEarly: o rows whose loads are started together with the (m, l) loads (registers: kEarly * D / 32)
+template <int D, int kEarly = 8>
 __device__ __forceinline__ void merge_row(const DecodeArgs& a, int leaf, int head, int lane, const MergeList& list) {
     constexpr int EPL = D / 32;  // features per lane
     const int G = a.G, sub = head % G;
@@ -35,7 +36,6 @@ __device__ __forceinline__ void merge_row(const DecodeArgs& a, int leaf, int hea
     float acc[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-    constexpr int kEarly = 8;   // o rows whose loads are started together with the (m, l) loads
     for (int base = s0; base < s1; base += 32) {
         const int cnt = min(32, s1 - base);
         const int my_slot = base == s0 ? list.first_slot : (lane < cnt ? a.leaf_slots[base + lane] : -1);
