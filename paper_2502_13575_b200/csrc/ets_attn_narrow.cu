@@ -125,10 +125,10 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// The page slots of one narrow item, one per lane (an item has at most 32): page id and the number
+// The page slots of one narrow item, one per lane (an item has at most 32): where the page's tiles are and the number
 // of tokens the slot holds now (0 = skip: empty, or a page id outside the pool, which is also flagged).
 struct SlotView {
-    int page = 0;
+    int page = 0;       // bit 0: which pool buffer holds the page; bits 1..: index of its (K tile, V tile) pair there, for the item's kv head
     int valid = 0;
     uint32_t live = 0;  // bit i: lane i's slot has tokens
 };
@@ -375,7 +375,7 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
         int cur_leaf[2] = {0, 0};
         bool f_on_next = false;     // the issue side has moved on to the next item
         uint32_t f_live = 0;        // slots of its item that it has not started yet
-        int f_page = 0, f_head = 0; // its item: page id per lane, kv head
+        int f_page = 0;             // its item: per lane, where the slot's tile pair sits (see SlotView::page)
         bool f_reread = false;      // its item's pages are read again by the next leaf tile
         NextItem nx;
 
@@ -415,7 +415,9 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
                             v = 0;
                         }
                     }
-                    nx.v.page = nx.un.x;
+                    // tile pair index inside its pool buffer, and which buffer (see kv_tile), worked out here by all
+                    // lanes at once instead of by the one lane that later starts the copy
+                    nx.v.page = (int)((((uint32_t)nx.it.kv_head * (uint32_t)pool_pairs(a.pages_per_layer) + (uint32_t)(nx.un.x >> 1)) << 1) | (uint32_t)(nx.un.x & 1));
                     nx.v.valid = v;
                     nx.v.live = __ballot_sync(FULL, v > 0);
                     nx.stage = 4;
@@ -436,12 +438,12 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
                 if (f_live) {
                     const int b = __ffs(f_live) - 1;
                     f_live &= f_live - 1;
-                    const int page = __shfl_sync(FULL, f_page, b);
+                    const uint32_t where = (uint32_t)__shfl_sync(FULL, f_page, b);
                     if (lane == 0) {
                         const uint32_t slot = n_issued % kDepth;
                         const uint32_t bar = bars + slot * 8;
                         const uint32_t dst = ring + slot * 2 * TB;
-                        const char* src = kv_tile(a.k_pool, a.v_pool, a.pages_per_layer, page, f_head, TB);
+                        const char* src = ((where & 1u) ? a.v_pool : a.k_pool) + (size_t)(where >> 1) * (2 * TB);
                         mbar_expect_tx(bar, 2 * TB);
                         if (f_reread) bulk_g2s(dst, src, 2 * TB, bar);   // K tile and V tile in one copy
                         else bulk_g2s_hint(dst, src, 2 * TB, bar, pol_stream);
@@ -457,7 +459,6 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
                 f_on_next = true;
                 f_live = nx.v.live;
                 f_page = nx.v.page;
-                f_head = nx.it.kv_head;
                 f_reread = (nx.it.reserved & 1) != 0;
             }
         };
@@ -494,7 +495,6 @@ __global__ void __maxnreg__(168) attn_partial_narrow_kernel(DecodeArgs a) {
             } else {
                 f_live = cv.live;
                 f_page = cv.page;
-                f_head = cur.kv_head;
                 f_reread = (cur.reserved & 1) != 0;
             }
             nx.stage = 0;
