@@ -138,6 +138,7 @@ struct ets_ctx {
     ets::FlattenParams fp{};
     Layout lay{};
     ets::Tree tree;
+    ets::Tree spare;   // the tree before the current one: the next build writes into it, reusing its memory
     ets::FlattenParams built{};   // the options the current tree was built with
     bool has_tree = false;
     bool host_only = true;
@@ -486,7 +487,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
         for (int32_t i = 0; i < n_nodes && identity; ++i) identity = keep_pages_of[i] == i;
         if (identity) return ETS_OK;
     }
-    ets::Tree next;
+    ets::Tree& next = c->spare;
     std::string err;
     int32_t rc = ets::tree_build(c->tree, fp, n_nodes, parent, cap_tokens, keep_pages_of, n_leaves, leaf_node,
                                  next, err);
@@ -507,7 +508,7 @@ int32_t ets_tree_build(ets_ctx* c, int32_t n_nodes, const int32_t* parent, const
         c->stage_used[i] = true;
         c->stage_next = (i + 1) % kStages;
     }
-    c->tree = std::move(next);
+    std::swap(c->tree, c->spare);
     c->bo = bo;
     c->has_tree = true;
     c->built = fp;

@@ -57,14 +57,21 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         }
     }
 
-    t = Tree();
+    // `t` may be an object that an earlier build filled: everything is set again below, and vectors that keep
+    // their capacity save the allocations (and the page faults of fresh memory) of a rebuild.
+    t.items.clear();
+    t.n_narrow_items = 0;
+    t.n_segments = t.n_chunks = t.n_partial_slots = 0;
+    t.chunk_pages_used = 0;
+    t.path_items = false;
     t.n_nodes = n_nodes;
     t.n_leaves = n_leaves;
     t.parent.assign(parent, parent + n_nodes);
     t.cap.assign(cap_tokens, cap_tokens + n_nodes);
     t.leaf_node.assign(leaf_node, leaf_node + n_leaves);
     const int32_t L = p.num_layers;
-    t.len.assign((size_t)L, std::vector<int32_t>((size_t)n_nodes, 0));
+    t.len.resize((size_t)L);
+    for (auto& v : t.len) v.assign((size_t)n_nodes, 0);
 
     // ---- pages: release what nobody keeps, then allocate in node order (lowest ids first)
     std::vector<int32_t> need((size_t)n_nodes);
@@ -242,18 +249,36 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             wsum += (std::min(leaves_per_tile, gn - l0) * p.gqa > 8 ? p.cost_rows16 : 1.0) * (l0 > 0 ? p.cost_reread : 1.0);
         narrow.push_back({s, nu, p.num_kv_heads * tiles, gn, wsum / tiles});
     }
+    // The estimate below is evaluated for up to ten piece lengths; segments with the same number of page slots
+    // behave alike in it, so they are summed up once (a tree has a thousand segments and a few dozen lengths).
+    struct Bucket { int32_t nu; int64_t mult, gn; double w_mult, w_max, w_min; };
+    std::vector<Bucket> buckets;
+    {
+        int32_t max_nu = 0;
+        for (const SegInfo& q : narrow) max_nu = std::max(max_nu, q.nu);
+        std::vector<int32_t> at((size_t)max_nu + 1, -1);
+        for (const SegInfo& q : narrow) {
+            if (at[q.nu] < 0) { at[q.nu] = (int32_t)buckets.size(); buckets.push_back({q.nu, 0, 0, 0.0, q.w, q.w}); }
+            Bucket& k = buckets[at[q.nu]];
+            k.mult += q.mult;
+            k.gn += q.gn;
+            k.w_mult += q.w * q.mult;
+            k.w_max = std::max(k.w_max, q.w);
+            k.w_min = std::min(k.w_min, q.w);
+        }
+    }
     // Estimated time of the queue for a piece length, in page-slot units: the mean load of a warp plus
     // half of a late piece, or the longest piece when that is more or when there are no more pieces than warps.
     auto estimate = [&](int32_t cap, int32_t tail_cap, int64_t& slots_needed) {
         double total = 0.0, longest = 0.0, shortest = 1e30;
         slots_needed = 0;
         int64_t pieces = 0;
-        for (const SegInfo& q : narrow) {
+        for (const Bucket& q : buckets) {
             const int32_t np_ = ceil_div(q.nu, cap);
             const double len = (double)q.nu / np_;
-            total += ((double)np_ * p.cost_item + q.nu * q.w) * q.mult;
-            longest = std::max(longest, p.cost_item + std::ceil(len) * q.w);
-            shortest = std::min(shortest, p.cost_item + std::min<double>(len, tail_cap) * q.w);
+            total += (double)np_ * p.cost_item * q.mult + q.nu * q.w_mult;
+            longest = std::max(longest, p.cost_item + std::ceil(len) * q.w_max);
+            shortest = std::min(shortest, p.cost_item + std::min<double>(len, tail_cap) * q.w_min);
             pieces += (int64_t)np_ * q.mult;
             slots_needed += (int64_t)np_ * p.num_kv_heads * q.gn;
         }
@@ -281,7 +306,7 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
             // returns; measured 32.1 -> 30.9 and 39.7 -> 38.1 us per call on the two width-64 trees, while the
             // width-256 tree, 4.5 pieces per warp, loses 0.6 % with 12).
             int64_t pieces_c = 0;
-            for (const SegInfo& q : narrow) pieces_c += (int64_t)ceil_div(q.nu, c) * q.mult;
+            for (const Bucket& q : buckets) pieces_c += (int64_t)ceil_div(q.nu, c) * q.mult;
             const int32_t tc = p.tail_pages > 0 ? p.tail_pages : std::max(pieces_c < 3 * (int64_t)n_workers ? 12 : 8, c / 4);
             int64_t need_slots = 0;
             const double est = estimate(c, tc, need_slots);

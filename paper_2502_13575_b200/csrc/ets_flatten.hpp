@@ -70,7 +70,8 @@ enum : int32_t { F_OK = 0, F_INVALID = -1, F_BAD_TREE = -2, F_EXHAUSTED = -3 };
 // Fresh state: all pages free, no nodes.
 void tree_init(Tree& t, const FlattenParams& p, int64_t pages_per_layer);
 
-// Builds `next` from `prev` (which is left untouched).  On failure `next` is unspecified and
+// Builds `next` from `prev` (which is left untouched; `next` must be another object).  `next` may hold an earlier
+// build: all of it is overwritten and its vectors' capacity is reused.  On failure `next` is unspecified and
 // `err` holds a message.
 int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, const int32_t* parent,
                    const int32_t* cap_tokens, const int32_t* keep_pages_of, int32_t n_leaves,
