@@ -12,7 +12,7 @@ namespace ets {
 void tree_init(Tree& t, const FlattenParams& p, int64_t pages_per_layer) {
     t = Tree();
     t.free_heap.resize((size_t)pages_per_layer);
-    std::iota(t.free_heap.begin(), t.free_heap.end(), 0);  // ascending = a valid min-heap
+    for (int64_t i = 0; i < pages_per_layer; ++i) t.free_heap[(size_t)i] = (int32_t)(pages_per_layer - 1 - i);   // falling: the lowest id is at the back
     t.len.assign((size_t)p.num_layers, {});
     t.node_page_off.assign(1, 0);
     t.node_leaf_off.assign(1, 0);
@@ -90,13 +90,20 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
                 if (keep_pages_of[i] >= 0) dst[i] = std::min(src[keep_pages_of[i]], cap_tokens[i]);
         }
     }
-    t.free_heap = prev.free_heap;
-    auto heap_cmp = std::greater<int32_t>();
-    for (int32_t o = 0; o < n_prev; ++o) {
-        int32_t keepn = std::max(claimed_old[o], 0);
-        for (int32_t j = prev.node_page_off[o] + keepn; j < prev.node_page_off[o + 1]; ++j) {
-            t.free_heap.push_back(prev.page_ids[j]);
-            std::push_heap(t.free_heap.begin(), t.free_heap.end(), heap_cmp);
+    // free pages, ids falling, so that the lowest is taken from the back; what this build releases is merged in
+    {
+        std::vector<int32_t> released;
+        for (int32_t o = 0; o < n_prev; ++o) {
+            int32_t keepn = std::max(claimed_old[o], 0);
+            for (int32_t j = prev.node_page_off[o] + keepn; j < prev.node_page_off[o + 1]; ++j) released.push_back(prev.page_ids[j]);
+        }
+        if (released.empty()) {
+            t.free_heap = prev.free_heap;
+        } else {
+            std::sort(released.begin(), released.end(), std::greater<int32_t>());
+            t.free_heap.resize(prev.free_heap.size() + released.size());
+            std::merge(prev.free_heap.begin(), prev.free_heap.end(), released.begin(), released.end(), t.free_heap.begin(),
+                       std::greater<int32_t>());
         }
     }
     t.node_page_off.assign((size_t)n_nodes + 1, 0);
@@ -112,7 +119,6 @@ int32_t tree_build(const Tree& prev, const FlattenParams& p, int32_t n_nodes, co
         }
         for (; got < need[i]; ++got) {
             if (t.free_heap.empty()) { err = "page pool exhausted at node " + std::to_string(i); return F_EXHAUSTED; }
-            std::pop_heap(t.free_heap.begin(), t.free_heap.end(), heap_cmp);
             t.page_ids[w + got] = t.free_heap.back();
             t.free_heap.pop_back();
         }

@@ -52,7 +52,7 @@ struct Tree {
     std::vector<int32_t> node_leaf_off, node_leaves;
     std::vector<int32_t> leaf_path_off, leaf_path, leaf_path_pos;
     std::vector<std::vector<int32_t>> len;  // [layer][node]
-    std::vector<int32_t> free_heap;         // min-heap of free page ids (std::greater)
+    std::vector<int32_t> free_heap;         // free page ids in falling order: the lowest id is handed out first, from the back
     // work decomposition
     std::vector<int32_t> unit;              // 4 per unit: page, node, tok0, 0
     std::vector<Item> items;                // narrow items in queue order, then wide items
