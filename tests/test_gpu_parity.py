@@ -203,6 +203,21 @@ def test_short_paths_with_cancelling_values_keep_the_tolerance(seed, aligned_q):
     run_and_check(tree, geom, 5000 + seed + 1, cap=tree.tokens, lengths=lengths, wide=wide, aligned_q=aligned_q)
 
 
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("leaves,root_tokens,filled", [(40, 523, 523), (33, 1100, 1093), (9, 300, 297)])
+def test_long_shared_prefix_on_the_tcgen05_kernel(d, leaves, root_tokens, filled):
+    """One long shared root under many leaves: its query group spans one full and one partly filled 128-row
+    tile (or a single small one), and its page slots make items of more than four 64-token stages (the stage
+    descriptions are a ring of four), a last stage with fewer than four page slots and a last page that is
+    partly filled, once with the root shorter than its capacity.  Every leaf against the oracle."""
+    parent = np.array([-1] + [0] * leaves, np.int32)
+    tokens = np.array([root_tokens] + [5 + 3 * (i % 7) for i in range(leaves)], np.int32)
+    tree = Tree(parent, tokens, np.arange(1, leaves + 1, dtype=np.int32))
+    lengths = tokens.copy()
+    lengths[0] = filled
+    run_and_check(tree, Geometry(8 * 4, 8, d) if leaves > 9 else Geometry(16, 1, d), 7700 + leaves, cap=tokens, lengths=lengths, wide=17)
+
+
 def test_single_token_tree_returns_v():
     g = Geometry(4, 2, 64)
     tree = Tree(np.array([-1], np.int32), np.array([1], np.int32), np.array([0], np.int32))
